@@ -1,0 +1,442 @@
+#!/usr/bin/env python
+"""Benchmark of the SBW hot path on B200.
+
+    python bench.py --gpus N --steps K --warmup W            # this library (CUDA kernels)
+    python bench.py --impl reference --steps K --warmup W    # the CPU oracle, as it stands
+
+One "step" is one decode step of the headline workload: `sbw_bias_logits` (context-hash seeding,
+gamma 0.5, delta 2.0, key 0x5EED) on a fresh [64, 128256] bf16 logits tensor with fresh context
+tokens -- 256 distinct step inputs (4.2 GB) are resident and visited in turn, so no step finds its
+input in L2.  `value` is bias throughput in Gelem/s (B*V logits per second, all GPUs).  The same
+JSON line carries the roofline placement of the bias kernel, the end-to-end figure through the
+host-buffer entry point, the oracle timed on the host cores, and (under "extra") the self-salt
+bias, detection and fused-sampling workloads with their own roofline fractions.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+KEY = 0x5EED
+B2, V2 = 64, 128256                 # headline workload: bf16, context scheme
+GAMMA2, DELTA2 = 0.5, 2.0
+POOL = 256                          # distinct step inputs kept resident
+# Algorithmic work per logit (what the method itself needs, not what the kernel spends):
+#   context scheme: Philox4x32-10 word 0 = 20 32x32->64 multiplies + 20 three-input xors, and one
+#   compare = 41 integer operations; 2 bytes read + 2 bytes written (bf16).
+INT_OPS = {"context": 41, "selfsalt": 80, "detect_context": 62, "detect_selfsalt": 100}
+# Integer ceiling of one B200: 148 SMs x 4 schedulers x 32 lanes = 18944 thread-operations per
+# clock (one warp instruction per scheduler per clock) at the 1965 MHz maximum SM clock.
+SMS, LANES_PER_SM_CLK, SM_MAX_MHZ = 148, 128, 1965.0
+INT_PEAK_TOPS = SMS * LANES_PER_SM_CLK * SM_MAX_MHZ * 1e6 / 1e12
+# DRAM bytes per bias launch of the headline workload from the ncu capture summarised under
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
+NCU_TRAFFIC_BYTES = None
+
+
+def measured_peaks() -> dict:
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return {"hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples = []
+        self._stop = threading.Event()
+        self._thread = None
+        self.max_mhz = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                self.samples.append((time.perf_counter(), float(mhz), int(reasons)))
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self, t0: float, t1: float) -> dict:
+        if self.nv is None or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        inside = [s for s in self.samples if t0 <= s[0] <= t1] or \
+            sorted(self.samples, key=lambda s: min(abs(s[0] - t0), abs(s[0] - t1)))[:3]
+        mhz = sorted(s[1] for s in inside)
+        bits = 0
+        for s in inside:
+            bits |= s[2]
+        names = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap",
+                 0x8: "hw_slowdown", 0x10: "sync_boost", 0x20: "sw_thermal_slowdown",
+                 0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+                 0x100: "display_clock_setting"}
+        return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": self.max_mhz, "samples": len(inside),
+                "reasons": [n for b, n in names.items() if bits & b and n != "gpu_idle"]}
+
+
+def dist_env():
+    return (int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)),
+            int(os.environ.get("WORLD_SIZE", 1)))
+
+
+def shard_rows(total_rows: int, rank: int, world: int) -> tuple[int, int]:
+    """Rows [lo, hi) of a batch owned by `rank` when a batch is sharded over `world` ranks (the
+    path has no cross-row dependency, so sharding needs no collective)."""
+    base, rem = divmod(total_rows, world)
+    lo = rank * base + min(rank, rem)
+    return lo, lo + base + (1 if rank < rem else 0)
+
+
+def max_over_ranks(x: float, world: int, device=None) -> float:
+    if world == 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# ------------------------------------------------------------------------------- reference arm
+def run_reference(args) -> None:
+    """Times the CPU oracle, as it stands, on the host cores: each step is one headline decode
+    step (64 x 128256 bf16, context scheme).  Rank 0 only."""
+    rank, _, _ = dist_env()
+    if rank != 0:
+        return
+    import torch
+    import oracle
+    from paper_2609_03844_b200 import inputs
+
+    cores = os.cpu_count() or 1
+    n_in = min(max(args.steps, 1), 4)
+    xs = [inputs.as_oracle_array(inputs.logits_normal(B2, V2, 4.0, torch.bfloat16, seed=1000 + i))
+          for i in range(n_in)]
+    cs = [inputs.uniform_tokens((B2, 1), V2, seed=2000 + i).numpy() for i in range(n_in)]
+    for i in range(args.warmup):
+        oracle.bias_logits(xs[i % n_in], V2, cs[i % n_in], KEY, GAMMA2, DELTA2, oracle.SCHEME_CONTEXT,
+                           threads=cores)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        oracle.bias_logits(xs[i % n_in], V2, cs[i % n_in], KEY, GAMMA2, DELTA2, oracle.SCHEME_CONTEXT,
+                           threads=cores)
+    dt = time.perf_counter() - t0
+    value = B2 * V2 * args.steps / dt / 1e9
+    line = {"impl": "reference", "metric": "sbw_bias_throughput", "value": value, "unit": "Gelem/s",
+            "n_gpus": 0, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": workload_config(),
+            "cpu_baseline": {"value": value, "unit": "Gelem/s", "cores": cores, "kind": "oracle",
+                             "sample": f"{args.steps} full decode steps of the headline workload"},
+            "e2e": {"value": value, "unit": "Gelem/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def workload_config() -> dict:
+    return {"workload": "config 2: sbw_bias_logits, B=64, V=128256, bf16 logits N(0,4^2), "
+                        "context-hash seeding on 1 preceding token, gamma=0.5, delta=2.0, key=0x5EED",
+            "B": B2, "V": V2, "scheme": "context", "gamma": GAMMA2, "delta": DELTA2,
+            "l2": f"{POOL} distinct step inputs (4.2 GB) visited in turn, far larger than the 126 MB L2"}
+
+
+# ------------------------------------------------------------------------------------ our arm
+def time_region(fn_enqueue, stream, world, device):
+    """barrier + sync, events around fn_enqueue() on `stream`, sync + barrier; max over ranks."""
+    import torch
+    import torch.distributed as dist
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    e0.record(stream)
+    fn_enqueue()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    t1 = time.perf_counter()
+    if world > 1:
+        dist.barrier()
+    ms = max_over_ranks(e0.elapsed_time(e1), world, device)
+    return ms, t0, t1
+
+
+def run_ours(args) -> None:
+    import torch
+    import paper_2609_03844_b200 as sbw
+    from paper_2609_03844_b200 import inputs
+
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the SBW path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    sbw.lib()
+    peaks = measured_peaks()
+    K, W = args.steps, args.warmup
+    stream = torch.cuda.current_stream()
+
+    # ---- headline workload: every rank holds its own POOL step inputs (weak scaling) ----
+    pool = min(POOL, max(K, 16))
+    logits = [inputs.logits_normal(B2, V2, 4.0, torch.bfloat16, seed=10_000 * rank + i, device=dev)
+              for i in range(pool)]
+    ctxs = [inputs.uniform_tokens((B2, 1), V2, seed=5_000_000 + 10_000 * rank + i, device=dev)
+            for i in range(pool)]
+    torch.cuda.synchronize()
+
+    def step(i):
+        j = i % pool
+        sbw.sbw_bias_logits(logits[j], ctxs[j], KEY, GAMMA2, DELTA2, sbw.SCHEME_CONTEXT)
+
+    for i in range(max(W, 3)):
+        step(i)
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.02)
+
+    launch_mode = "stream"
+    graph = None
+    if not args.no_graph:
+        try:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                for i in range(K):
+                    step(W + i)
+            launch_mode = "cuda_graph"
+        except Exception as exc:    # capture unsupported: keep the plain stream launches
+            graph = None
+            launch_mode = f"stream (graph capture failed: {type(exc).__name__})"
+    stream = torch.cuda.current_stream()
+    if graph is not None:
+        graph.replay()              # one untimed replay: graph upload
+        ms, t0, t1 = time_region(graph.replay, stream, world, dev)
+    else:
+        ms, t0, t1 = time_region(lambda: [step(W + i) for i in range(K)], stream, world, dev)
+    # the same K steps as plain stream launches, for the record
+    ms_stream, _, _ = time_region(lambda: [step(W + i) for i in range(K)], stream, world, dev)
+    time.sleep(0.01)
+    sampler.stop()
+    clocks = sampler.summary(t0, t1)
+
+    elems_step = B2 * V2
+    value = world * elems_step * K / (ms * 1e-3) / 1e9
+    launch_s = ms * 1e-3 / K
+    int_ops = INT_OPS["context"] * elems_step
+    ach_tops = int_ops / launch_s / 1e12
+    hbm_gbs = 4 * elems_step / launch_s / 1e9
+    roofline = {"bound": "alu", "achieved": ach_tops, "peak": INT_PEAK_TOPS, "unit": "Tint-op/s",
+                "frac": ach_tops / INT_PEAK_TOPS, "traffic": NCU_TRAFFIC_BYTES,
+                "peak_source": "derived: 148 SMs x 4 schedulers x 32 lanes x 1965 MHz",
+                "kernel": "bias_kernel<bf16, context, vector>", "avg_launch_us": launch_s * 1e6,
+                "int_ops_per_elem": INT_OPS["context"],
+                "hbm": {"achieved": hbm_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": hbm_gbs / peaks["hbm_gbs"], "of": peaks["source"],
+                        "bytes_per_elem": 4},
+                "binding": "alu" if int_ops / (INT_PEAK_TOPS * 1e12) > 4 * elems_step / (peaks["hbm_gbs"] * 1e9)
+                else "hbm"}
+
+    # ---- end to end: host buffers through the C ABI, copies inside the timed region ----
+    n_host = 4
+    h_logits = [inputs.logits_normal(B2, V2, 4.0, torch.bfloat16, seed=77 + i).pin_memory() for i in range(n_host)]
+    h_ctx = [inputs.uniform_tokens((B2, 1), V2, seed=88 + i).pin_memory() for i in range(n_host)]
+    staging = torch.empty(sbw.sbw_bias_logits_host_staging_bytes(torch.bfloat16, B2, V2, 1),
+                          dtype=torch.uint8, device=dev)
+    K_e2e = max(1, min(K, 64))
+
+    def e2e_steps():
+        for i in range(K_e2e):
+            sbw.sbw_bias_logits_host(h_logits[i % n_host], h_ctx[i % n_host], KEY, GAMMA2, DELTA2,
+                                     sbw.SCHEME_CONTEXT, staging)
+
+    e2e_steps()
+    ms_e2e, _, _ = time_region(e2e_steps, torch.cuda.current_stream(), world, dev)
+    e2e = {"value": world * elems_step * K_e2e / (ms_e2e * 1e-3) / 1e9, "unit": "Gelem/s",
+           "h2d_bytes_per_step": elems_step * 2 + B2 * 4, "d2h_bytes_per_step": elems_step * 2,
+           "steps": K_e2e, "ms_per_step": ms_e2e / K_e2e,
+           "api": "sbw_bias_logits_host (pinned host logits and context tokens)"}
+    del h_logits, staging
+
+    line = {"metric": "sbw_bias_throughput", "value": value, "unit": "Gelem/s", "n_gpus": world,
+            "steps": K, "warmup": W, "ms_per_step": ms / K, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {**workload_config(), "launch": launch_mode, "parallelism": f"replicas x{world}",
+                       "l2": f"{pool} distinct step inputs ({pool * elems_step * 2 / 1e9:.1f} GB) visited in "
+                             "turn, far larger than the 126 MB L2"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": K, "roofline": roofline,
+            "stream_launch": {"value": world * elems_step * K / (ms_stream * 1e-3) / 1e9,
+                              "ms_per_step": ms_stream / K}}
+
+    if rank == 0 and world == 1 and not args.no_extra:
+        del logits, ctxs
+        torch.cuda.empty_cache()
+        line["extra"] = run_extra(sbw, inputs, dev, peaks)
+        line["cpu_baseline"] = cpu_baseline()
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def cpu_baseline() -> dict:
+    """The oracle, untouched, on the host cores: a bounded sample of the headline workload."""
+    import torch
+    import oracle
+    from paper_2609_03844_b200 import inputs
+
+    cores = os.cpu_count() or 1
+    x = inputs.as_oracle_array(inputs.logits_normal(B2, V2, 4.0, torch.bfloat16, seed=4242))
+    c = inputs.uniform_tokens((B2, 1), V2, seed=4243).numpy()
+    oracle.bias_logits(x, V2, c, KEY, GAMMA2, DELTA2, oracle.SCHEME_CONTEXT, threads=cores)
+    t0 = time.perf_counter()
+    n = 0
+    while True:
+        oracle.bias_logits(x, V2, c, KEY, GAMMA2, DELTA2, oracle.SCHEME_CONTEXT, threads=cores)
+        n += 1
+        dt = time.perf_counter() - t0
+        if dt * cores > 12.0 or n >= 64:       # about 12 core-seconds of work
+            break
+    t1 = time.perf_counter()
+    oracle.bias_logits(x[:8], V2, c[:8], KEY, GAMMA2, DELTA2, oracle.SCHEME_CONTEXT, threads=1)
+    single = 8 * V2 / (time.perf_counter() - t1) / 1e9
+    return {"value": B2 * V2 * n / dt / 1e9, "unit": "Gelem/s", "cores": cores, "kind": "oracle",
+            "sample": f"{n} decode steps of the headline workload ({n * B2 * V2 / 1e6:.0f} M logits)",
+            "single_thread_value": single}
+
+
+def _time_calls(fn, n, warm=3):
+    import torch
+    for i in range(warm):
+        fn(i)
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(n):
+        fn(warm + i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e-3 / n
+
+
+def run_extra(sbw, inputs, dev, peaks) -> dict:
+    """The other workloads of the hot path, each timed on its own (inputs larger than L2 or
+    rotating), and the integer-throughput probe."""
+    import torch
+    out = {}
+    hbm = peaks["hbm_gbs"]
+
+    def place(int_ops, nbytes, seconds):
+        t_alu = int_ops / (INT_PEAK_TOPS * 1e12)
+        t_hbm = nbytes / (hbm * 1e9)
+        return {"bound": "alu" if t_alu >= t_hbm else "hbm", "frac": max(t_alu, t_hbm) / seconds,
+                "alu_frac": t_alu / seconds, "hbm_frac": t_hbm / seconds,
+                "achieved_tint_ops": int_ops / seconds / 1e12, "achieved_gbs": nbytes / seconds / 1e9}
+
+    # config 3: full-vocabulary self-salt, fp32, B=256, V=151936, gamma .25, delta 4
+    B3, V3 = 256, 151936
+    p3 = [inputs.add_zipf_spike_(inputs.logits_normal(B3, V3, 4.0, torch.float32, seed=300 + i, device=dev),
+                                 V3, seed=310 + i) for i in range(4)]
+    c3 = [inputs.uniform_tokens((B3, 1), V3, seed=320 + i, device=dev) for i in range(4)]
+    for name, scheme in (("selfsalt", sbw.SCHEME_SELFSALT), ("context", sbw.SCHEME_CONTEXT)):
+        s = _time_calls(lambda i: sbw.sbw_bias_logits(p3[i % 4], c3[i % 4], KEY, 0.25, 4.0, scheme), 128)
+        n = B3 * V3
+        out[f"bias_fp32_{name}_B256_V151936"] = {"gelem_s": n / s / 1e9, "ms": s * 1e3,
+                                                 **place(INT_OPS[name] * n, 8 * n, s)}
+    del p3, c3
+    # config 2 shape under the self-salt scheme
+    p2 = [inputs.logits_normal(B2, V2, 4.0, torch.bfloat16, seed=400 + i, device=dev) for i in range(16)]
+    c2 = [inputs.uniform_tokens((B2, 1), V2, seed=420 + i, device=dev) for i in range(16)]
+    s = _time_calls(lambda i: sbw.sbw_bias_logits(p2[i % 16], c2[i % 16], KEY, 0.5, 2.0, sbw.SCHEME_SELFSALT), 256)
+    out["bias_bf16_selfsalt_B64_V128256"] = {"gelem_s": B2 * V2 / s / 1e9, "ms": s * 1e3,
+                                             **place(INT_OPS["selfsalt"] * B2 * V2, 4 * B2 * V2, s)}
+    del p2, c2
+    # config 5 (null half shape): 100000 sequences, lengths uniform in [64, 1024], 218 MB of ids
+    N = 100000
+    tokens, lengths = inputs.null_token_streams(N, 64, 1024, V2, seed=500, device=dev)
+    counts = torch.empty(N, dtype=torch.int32, device=dev)
+    z = torch.empty(N, dtype=torch.float64, device=dev)
+    ws = torch.empty(sbw.sbw_detect_workspace_bytes(N), dtype=torch.uint8, device=dev)
+    ntok = tokens.numel()
+    for name, scheme in (("context", sbw.SCHEME_CONTEXT), ("selfsalt", sbw.SCHEME_SELFSALT)):
+        s = _time_calls(lambda i: sbw.sbw_detect(tokens, lengths, KEY, 0.25, scheme, counts, z, workspace=ws), 30)
+        out[f"detect_{name}_N100000"] = {"tokens_per_s": ntok / s, "ms": s * 1e3, "tokens": ntok,
+                                         **place(INT_OPS[f"detect_{name}"] * ntok, 4 * ntok + 24 * N, s)}
+    del tokens
+    # config 4: fused sampling sweep, bf16, V=128256, tau 0.7
+    for B in (1, 8, 32, 128, 512, 1024):
+        x = inputs.logits_normal(B, V2, 4.0, torch.bfloat16, seed=600 + B, device=dev)
+        c = inputs.uniform_tokens((B, 1), V2, seed=700 + B, device=dev)
+        ids = torch.empty(B, dtype=torch.int32, device=dev)
+        wsb = torch.empty(sbw.sbw_sample_workspace_bytes(B, V2), dtype=torch.uint8, device=dev)
+        for name, scheme in (("context", sbw.SCHEME_CONTEXT), ("selfsalt", sbw.SCHEME_SELFSALT)):
+            s = _time_calls(lambda i: sbw.sbw_bias_sample(x, c, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, wsb), 20)
+            out[f"sample_bf16_{name}_B{B}"] = {"gelem_s": B * V2 / s / 1e9, "ms": s * 1e3,
+                                               "l2_resident": B * V2 * 2 < 100e6}
+    # integer-throughput probe
+    probes = {}
+    for kind in ("mulwide", "lop3", "iadd3", "imad", "philox", "ffma"):
+        r = sbw.sbw_int_probe(kind, steps=8192, blocks_per_sm=4, threads=256)
+        probes[kind] = {"ops_per_clk_per_sm": r["ops_per_clk_per_sm"], "tops": r["ops_per_s"] / 1e12,
+                        "sm_mhz": r["sm_mhz_implied"]}
+    out["int_probe"] = probes
+    return out
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2048)
+    ap.add_argument("--warmup", type=int, default=16)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-graph", action="store_true", help="time plain stream launches only")
+    ap.add_argument("--no-extra", action="store_true", help="skip the secondary workloads and the CPU baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps == 2048:
+            args.steps, args.warmup = 32, 3
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,167 @@
+/*
+ * sbw.h -- C ABI of the B200 (sm_100a) library for Stateless Bernoulli Watermarking (SBW).
+ *
+ * The library is the data-parallel hot path of the method: the per-decode-step logits bias
+ * (Section 2.2, Eq. 1 and Eq. 2 of the paper), the same bias fused with temperature softmax and
+ * Gumbel-max sampling, and batch detection (Section 2.2 "Detection", Eq. 5).  Every step runs
+ * in hand-written CUDA kernels; there is no CPU fallback and no other backend.
+ *
+ * Conventions for every call
+ *   - Pointers are DEVICE pointers owned by the caller unless a parameter says "host".
+ *   - The library allocates nothing, frees nothing and never synchronises: work is enqueued on
+ *     `stream` (a cudaStream_t passed as void*, NULL = the legacy default stream) and the call
+ *     returns at once.  Scratch memory, where a call needs it, is passed in as `workspace`.
+ *   - Return value: SBW_OK or a negative SBW_ERR_* code.  Nothing is enqueued when an argument
+ *     is rejected.  After SBW_ERR_CUDA, sbw_last_cuda_error() returns the cudaError_t seen by
+ *     the calling thread.  No exceptions, no exit(), no device-side traps.
+ *   - Token ids are reinterpreted as unsigned 32-bit values; any bit pattern gives a
+ *     deterministic result and is never used as an address.
+ *   - B == 0 or N == 0 is SBW_OK and launches nothing.
+ *
+ * Readings taken where the paper names an operation without printing it ("SBW-spec v1"):
+ *   Jenkins hash J      (Section 2.3)  a=(a+0x7ed55d16)+(a<<12); a=(a^0xc761c23c)^(a>>19);
+ *                                      a=(a+0x165667b1)+(a<<5);  a=(a+0xd3a2646c)^(a<<9);
+ *                                      a=(a+0xfd7046c5)+(a<<3);  a=(a^0xb55a4f09)^(a>>16)
+ *   CBRNG               (Section 2.2)  x = word 0 of Philox4x32-10(counter (v,0,0,0),
+ *                                      key (lo32 r, hi32 r)), v = vocab_offset + column
+ *   green               (Eq. 1)        x < ceil(gamma * 2^32)   (strict, integer compare)
+ *   seed r, CONTEXT     (Table 12, "additive")          r = key * (sum of the ctx ids)  mod 2^64
+ *   seed r, SELFSALT    (Table 12, "anchored minhash";  r = key * J(v) * min(J(v), min_i J(ctx_i))
+ *                        Section 5.2, every candidate)      mod 2^64, J(.)J(.) taken in 64 bits
+ *   bias                (Eq. 2)        green: one round-to-nearest-even add of delta in the
+ *                                      logits' precision (bf16: delta rounded to bf16 first);
+ *                                      not green: value unchanged
+ */
+#ifndef SBW_H
+#define SBW_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SBW_OK 0
+#define SBW_ERR_INVALID_ARG (-1) /* null required pointer, size < 0, ld < V, gamma outside (0,1), ... */
+#define SBW_ERR_UNSUPPORTED (-2) /* a value the ABI reserves but this build does not implement */
+#define SBW_ERR_WORKSPACE (-3)   /* workspace missing, misaligned or too small */
+#define SBW_ERR_CUDA (-4)        /* a CUDA runtime call failed; see sbw_last_cuda_error() */
+
+#define SBW_SCHEME_CONTEXT 0  /* seed from the preceding tokens only (SBW-1, SBW-4) */
+#define SBW_SCHEME_SELFSALT 1 /* seed from the preceding tokens and the candidate (SBW-ss-V) */
+
+#define SBW_DTYPE_F32 0  /* IEEE binary32 logits */
+#define SBW_DTYPE_BF16 1 /* bfloat16 logits */
+
+#define SBW_MAX_CTX_WIDTH 8
+
+/* Library version string (static storage, host). */
+const char *sbw_version(void);
+
+/* cudaError_t recorded by the calling thread's last call that returned SBW_ERR_CUDA, else 0. */
+int sbw_last_cuda_error(void);
+
+/*
+ * sbw_bias_logits -- Eq. 1 + Eq. 2, one decode step, in place, one pass, no mask tensor
+ * (Section 5.1: in-place mutation, a single CBRNG evaluation per token, no CPU synchronisation).
+ *
+ *   logits       in/out, device, [B, ld] row-major, element type `dtype`; columns 0..V-1 of each
+ *                row are biased, columns V..ld-1 are neither read nor written.  Any alignment is
+ *                accepted; rows that start on 16-byte boundaries take the vectorised path.
+ *   B, V, ld     rows, vocabulary columns, row stride in elements (ld >= V > 0, B >= 0).
+ *   vocab_offset global id of column 0 (>= 0; non-zero when the vocabulary is sharded).
+ *   ctx_tokens   device, [B, ctx_width] int32: the ctx_width tokens preceding the one being
+ *                generated, per row.  1 <= ctx_width <= SBW_MAX_CTX_WIDTH.
+ *   key          64-bit secret key.      gamma  green fraction, 0 < gamma < 1.
+ *   delta        bias added to green logits (any finite float; 0 leaves every bit unchanged).
+ *   scheme       SBW_SCHEME_*.           stream cudaStream_t.
+ * NaN logits stay NaN (payload unspecified); +-inf follow IEEE addition.
+ */
+int sbw_bias_logits(void *logits, int dtype, int64_t B, int64_t V, int64_t ld, int64_t vocab_offset,
+                    const int32_t *ctx_tokens, int ctx_width, uint64_t key, double gamma,
+                    float delta, int scheme, void *stream);
+
+/*
+ * sbw_bias_logits_host -- the same step for callers whose logits live in HOST memory: copies
+ * B*ld elements and the context tokens to the device staging buffer, runs sbw_bias_logits on
+ * it, and copies the logits back, all enqueued on `stream` (the copies are asynchronous only if
+ * the host buffers are page-locked).  The paper has the logits on the GPU already; this entry
+ * exists so that end-to-end cost including the PCIe transfers can be measured.
+ *
+ *   logits_host  in/out, HOST, [B, ld].        ctx_tokens_host  HOST, [B, ctx_width] int32.
+ *   staging      device scratch of at least sbw_bias_logits_host_staging_bytes(...) bytes,
+ *                256-byte aligned; owned by the caller, contents undefined afterwards.
+ * The results are in logits_host once `stream` has been synchronised by the caller.
+ */
+size_t sbw_bias_logits_host_staging_bytes(int dtype, int64_t B, int64_t ld, int ctx_width);
+int sbw_bias_logits_host(void *logits_host, int dtype, int64_t B, int64_t V, int64_t ld,
+                         int64_t vocab_offset, const int32_t *ctx_tokens_host, int ctx_width,
+                         uint64_t key, double gamma, float delta, int scheme, void *staging,
+                         size_t staging_bytes, void *stream);
+
+/*
+ * sbw_bias_sample -- the bias of Eq. 1 + Eq. 2 fused with temperature softmax statistics and
+ * Gumbel-max sampling, one pass over read-only logits.  The paper leaves sampling to the
+ * serving engine (Section 5.1 speaks of absorbing the watermark into existing logit
+ * post-processing); this call is that absorption.  Per row b, with l'_v the biased logit in the
+ * logits' own precision and tau = temperature:
+ *     m  = max_v l'_v                      Z = sum_v exp((l'_v - m) / tau)
+ *     id = argmax_v fmaf(l'_v, 1/tau, g_v)  (fp32, 1/tau rounded once; ties -> lowest v)
+ *     p  = exp((l'_id - m) / tau) / Z
+ * g_v = -L(-L(u_v)) is a standard Gumbel variate from a counter-based stream of its own:
+ *     y   = word (vg & 3) of Philox4x32-10(counter (vg >> 2, b, lo32 rng_step, hi32 rng_step),
+ *           key (lo32 rng_seed, hi32 rng_seed)),  vg = vocab_offset + v
+ *     u_v = ((y >> 9) + 0.5) * 2^-23
+ * and L is a fixed fp32 logarithm made of exactly rounded operations (see sbw_sample.cu), so
+ * that `out_tokens` is reproducible bit for bit on any IEEE machine.
+ *
+ *   logits        device, read only, [B, ld] of `dtype`.
+ *   temperature   tau > 0.                 rng_seed, rng_step  select the Gumbel stream; use a
+ *                 new rng_step for every decode step.
+ *   out_tokens    device [B] int32: sampled column index (0-based within this shard).
+ *   out_max, out_sumexp, out_prob   device [B] float, each may be NULL: m, Z, p.
+ *   out_probs     device [B, V] float or NULL: the full softmax of the biased logits
+ *                 (costs a second pass; meant for tests and small batches).
+ *   workspace     device scratch, 256-byte aligned, at least
+ *                 sbw_sample_workspace_bytes(B, V) bytes; contents undefined afterwards.
+ *                 Calls that share a workspace must not overlap on the GPU.
+ * Rows whose logits are all -inf return id 0; m, Z, p of such rows, and every output of rows
+ * that contain NaN or +inf, are unspecified.
+ */
+size_t sbw_sample_workspace_bytes(int64_t B, int64_t V);
+int sbw_bias_sample(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
+                    int64_t vocab_offset, const int32_t *ctx_tokens, int ctx_width, uint64_t key,
+                    double gamma, float delta, int scheme, float temperature, uint64_t rng_seed,
+                    uint64_t rng_step, int32_t *out_tokens, float *out_max, float *out_sumexp,
+                    float *out_prob, float *out_probs, void *workspace, size_t workspace_bytes,
+                    void *stream);
+
+/*
+ * sbw_detect -- batch detection (Section 2.2 "Detection": one membership test per token, no
+ * green list is built; Eq. 5 for the score).  For sequence s with tokens t_0..t_{L-1}:
+ *     scored positions  i = W .. L-1  (the first W = ctx_width tokens only seed), T = max(L-W, 0)
+ *     Y_i = green(seed(t_{i-W..i-1}[, t_i]), v = t_i),   G = sum Y_i
+ *     z   = (G - gamma T) / sqrt(T gamma (1 - gamma))     in fp64;  T = 0 gives G = 0, z = 0.
+ *
+ *   tokens        device, int32, the N sequences back to back (total_tokens ids).
+ *   lengths       device [N] int32 (negative values count as 0).
+ *   offsets       device [N+1] int64 start of each sequence in `tokens`, or NULL: the library
+ *                 then scans `lengths` into the workspace first.
+ *   total_tokens  number of ids in `tokens`; positions at or beyond it are never read, and a
+ *                 sequence that would run past it is scored only up to it.
+ *   out_counts    device [N] int32: G.    out_T  device [N] int32 or NULL: T.
+ *   out_z         device [N] double: z.
+ *   workspace     device scratch, 256-byte aligned, at least sbw_detect_workspace_bytes(N) bytes
+ *                 (may be NULL with size 0 when `offsets` is given).
+ */
+size_t sbw_detect_workspace_bytes(int64_t N);
+int sbw_detect(const int32_t *tokens, const int32_t *lengths, const int64_t *offsets, int64_t N,
+               int64_t total_tokens, int ctx_width, uint64_t key, double gamma, int scheme,
+               int32_t *out_counts, int32_t *out_T, double *out_z, void *workspace,
+               size_t workspace_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SBW_H */

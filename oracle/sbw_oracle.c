@@ -22,6 +22,9 @@
  *      products of two 32-bit hashes taken in 64 bits.
  *  R6  Bias: green -> one IEEE round-to-nearest-even add in the logits' own precision;
  *      not green -> the element's bits are untouched.  bf16: delta is first rounded to bf16.
+ *      A delta that is zero in that precision is the paper's delta = 0 control (Section 4.5:
+ *      "non-watermarked completions"): nothing is added and every bit stays (an IEEE add of
+ *      +0 would turn -0 into +0).
  *  R7  Detection scores positions t = W .. L-1 (the first W tokens only seed), T = max(L-W,0),
  *      every position counted (no repeated-n-gram filter); T = 0 gives G = 0, z = 0.
  *  R8  The fused sampler is this library's own (the paper leaves sampling to the engine):
@@ -158,7 +161,7 @@ uint16_t sbw_oracle_f32_to_bf16(float x)
 /* R6, fp32 logits. */
 float sbw_oracle_bias_elem_f32(float l, float delta, int green)
 {
-    if (!green)
+    if (!green || delta == 0.0f)
         return l;
     return l + delta;
 }
@@ -172,6 +175,8 @@ uint16_t sbw_oracle_bias_elem_bf16(uint16_t l, float delta, int green)
     if (!green)
         return l;
     float d = sbw_oracle_bf16_to_f32(sbw_oracle_f32_to_bf16(delta));
+    if (d == 0.0f)
+        return l;
     float s = sbw_oracle_bf16_to_f32(l) + d;
     return sbw_oracle_f32_to_bf16(s);
 }

@@ -1,0 +1,218 @@
+// sbw_detect: batch detection -- one membership test per generated token (Section 2.2 of the
+// paper, "Detection"), green counts by warp ballot + popcount, z-score of Eq. 5 in fp64.
+//
+// One warp scores one sequence.  Lanes read consecutive tokens (coalesced 128-byte requests;
+// the W predecessors of a token come from the same cache lines), derive the token's seed, run
+// one Philox evaluation, and the warp adds popc(ballot(green)) to a warp-uniform counter, so no
+// per-lane reduction is needed at the end.  Each lane carries kDetectIlp independent tokens per
+// trip so that the dependent multiply/xor chain of one hash overlaps with the others.
+// Sequence starts come from a caller-supplied offsets array or from a two-kernel exclusive scan
+// of the lengths into the workspace.
+#include "sbw_common.cuh"
+#include "sbw_hash.cuh"
+
+namespace sbw {
+namespace {
+
+constexpr int kDetectThreads = 128;  // 4 sequences per block: short blocks keep the tail small
+constexpr int kDetectIlp = 2;
+constexpr int kScanThreads = 256;
+constexpr int kScanItems = 4;        // lengths per thread
+constexpr int kScanTile = kScanThreads * kScanItems;
+
+struct DetectArgs {
+    const int32_t *tokens;
+    const int32_t *lengths;
+    const int64_t *offsets;
+    int64_t N, total_tokens;
+    int W;
+    uint64_t key;
+    uint32_t thr_m1;
+    double gamma;
+    int32_t *out_counts;
+    int32_t *out_T;
+    double *out_z;
+};
+
+__device__ __forceinline__ int64_t clamp_len(int32_t l) { return l > 0 ? l : 0; }
+
+// ---- exclusive scan of the lengths: tile sums, then per-tile scan with a look-back sum ----
+__global__ void __launch_bounds__(kScanThreads)
+scan_tile_sums(const int32_t *lengths, int64_t N, int64_t *tile_sums) {
+    __shared__ int64_t warp_sums[kScanThreads / 32];
+    const int64_t base = static_cast<int64_t>(blockIdx.x) * kScanTile;
+    int64_t s = 0;
+#pragma unroll
+    for (int i = 0; i < kScanItems; ++i) {
+        const int64_t idx = base + i * kScanThreads + threadIdx.x;
+        if (idx < N) s += clamp_len(lengths[idx]);
+    }
+    for (int d = 16; d > 0; d >>= 1) s += __shfl_down_sync(0xffffffffu, s, d);
+    if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int64_t t = 0;
+        for (int w = 0; w < kScanThreads / 32; ++w) t += warp_sums[w];
+        tile_sums[blockIdx.x] = t;
+    }
+}
+
+__global__ void __launch_bounds__(kScanThreads)
+scan_offsets(const int32_t *lengths, int64_t N, const int64_t *tile_sums, int64_t *offsets) {
+    __shared__ int64_t warp_sums[kScanThreads / 32];
+    __shared__ int64_t tile_base;
+    // sum of all earlier tiles
+    int64_t s = 0;
+    for (int64_t t = threadIdx.x; t < blockIdx.x; t += kScanThreads) s += tile_sums[t];
+    for (int d = 16; d > 0; d >>= 1) s += __shfl_down_sync(0xffffffffu, s, d);
+    if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int64_t t = 0;
+        for (int w = 0; w < kScanThreads / 32; ++w) t += warp_sums[w];
+        tile_base = t;
+    }
+    __syncthreads();
+    // each thread owns kScanItems consecutive lengths
+    const int64_t first = static_cast<int64_t>(blockIdx.x) * kScanTile + threadIdx.x * kScanItems;
+    int64_t v[kScanItems];
+    int64_t mine = 0;
+#pragma unroll
+    for (int i = 0; i < kScanItems; ++i) {
+        v[i] = (first + i < N) ? clamp_len(lengths[first + i]) : 0;
+        mine += v[i];
+    }
+    // inclusive scan of `mine` over the block
+    int64_t incl = mine;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int d = 1; d < 32; d <<= 1) {
+        const int64_t up = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += up;
+    }
+    __syncthreads();
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    int64_t before = tile_base;
+    for (int w = 0; w < warp; ++w) before += warp_sums[w];
+    int64_t run = before + incl - mine;
+#pragma unroll
+    for (int i = 0; i < kScanItems; ++i) {
+        if (first + i < N) offsets[first + i] = run;
+        run += v[i];
+        if (first + i == N - 1) offsets[N] = run;
+    }
+}
+
+// ---- the detector ----
+template <int SCHEME>
+__global__ void __launch_bounds__(kDetectThreads)
+detect_kernel(const DetectArgs a) {
+    const int lane = threadIdx.x & 31;
+    const int64_t seq = static_cast<int64_t>(blockIdx.x) * (kDetectThreads / 32) + (threadIdx.x >> 5);
+    if (seq >= a.N) return;
+    const int64_t off = a.offsets[seq];
+    int64_t L = clamp_len(a.lengths[seq]);
+    if (off < 0 || off >= a.total_tokens) L = 0;
+    else if (off + L > a.total_tokens) L = a.total_tokens - off;
+    const int W = a.W;
+    const int32_t *tok = a.tokens + off;
+    const int len = static_cast<int>(L);
+
+    int count = 0;
+    for (int base = W; base < len; base += 32 * kDetectIlp) {
+        bool g[kDetectIlp];
+#pragma unroll
+        for (int u = 0; u < kDetectIlp; ++u) {
+            const int t = base + u * 32 + lane;
+            const bool valid = t < len;
+            const int ts = valid ? t : W;        // any readable position; result is discarded
+            const uint32_t v = static_cast<uint32_t>(tok[ts]);
+            uint64_t r;
+            if constexpr (SCHEME == SBW_SCHEME_CONTEXT) {
+                uint64_t sigma = 0;
+                for (int i = 1; i <= W; ++i) sigma += static_cast<uint32_t>(tok[ts - i]);
+                r = a.key * sigma;
+            } else {
+                uint32_t jmin = 0xFFFFFFFFu;
+                for (int i = 1; i <= W; ++i) jmin = min(jmin, jenkins(static_cast<uint32_t>(tok[ts - i])));
+                r = seed_selfsalt(a.key, jmin, v);
+            }
+            g[u] = valid && (philox_word0(v, r) <= a.thr_m1);
+        }
+#pragma unroll
+        for (int u = 0; u < kDetectIlp; ++u) count += __popc(__ballot_sync(0xffffffffu, g[u]));
+    }
+    if (lane == 0) {
+        const int T = len > W ? len - W : 0;
+        a.out_counts[seq] = count;
+        if (a.out_T) a.out_T[seq] = T;
+        double z = 0.0;
+        if (T > 0) {
+            // Eq. 5, every operation rounded separately
+            const double num = __dsub_rn(static_cast<double>(count), __dmul_rn(a.gamma, static_cast<double>(T)));
+            const double var = __dmul_rn(__dmul_rn(static_cast<double>(T), a.gamma), __dsub_rn(1.0, a.gamma));
+            z = __ddiv_rn(num, __dsqrt_rn(var));
+        }
+        a.out_z[seq] = z;
+    }
+}
+
+}  // namespace
+}  // namespace sbw
+
+extern "C" size_t sbw_detect_workspace_bytes(int64_t N) {
+    if (N <= 0) return 0;
+    const size_t tiles = static_cast<size_t>((N + sbw::kScanTile - 1) / sbw::kScanTile);
+    return sbw::align_up((static_cast<size_t>(N) + 1) * sizeof(int64_t), 256) +
+           sbw::align_up(tiles * sizeof(int64_t), 256);
+}
+
+extern "C" int sbw_detect(const int32_t *tokens, const int32_t *lengths, const int64_t *offsets,
+                          int64_t N, int64_t total_tokens, int ctx_width, uint64_t key, double gamma,
+                          int scheme, int32_t *out_counts, int32_t *out_T, double *out_z,
+                          void *workspace, size_t workspace_bytes, void *stream) {
+    using namespace sbw;
+    if (!valid_common(SBW_DTYPE_F32, ctx_width, gamma, scheme)) return SBW_ERR_INVALID_ARG;
+    if (N < 0 || total_tokens < 0) return SBW_ERR_INVALID_ARG;
+    if (N == 0) return SBW_OK;
+    if (N > (int64_t(1) << 31) * (kDetectThreads / 32) - 1) return SBW_ERR_UNSUPPORTED;
+    if (!lengths || !out_counts || !out_z) return SBW_ERR_INVALID_ARG;
+    if (!tokens && total_tokens > 0) return SBW_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    DetectArgs a;
+    a.tokens = tokens;
+    a.lengths = lengths;
+    a.offsets = offsets;
+    a.N = N;
+    a.total_tokens = total_tokens;
+    a.W = ctx_width;
+    a.key = key;
+    a.thr_m1 = threshold_minus_one(gamma);
+    a.gamma = gamma;
+    a.out_counts = out_counts;
+    a.out_T = out_T;
+    a.out_z = out_z;
+
+    if (!offsets) {
+        const size_t need = sbw_detect_workspace_bytes(N);
+        if (!workspace || workspace_bytes < need || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
+            return SBW_ERR_WORKSPACE;
+        int64_t *ws_offsets = static_cast<int64_t *>(workspace);
+        int64_t *tile_sums = reinterpret_cast<int64_t *>(
+            static_cast<char *>(workspace) + align_up((static_cast<size_t>(N) + 1) * sizeof(int64_t), 256));
+        const unsigned tiles = static_cast<unsigned>((N + kScanTile - 1) / kScanTile);
+        scan_tile_sums<<<tiles, kScanThreads, 0, s>>>(lengths, N, tile_sums);
+        SBW_CUDA_TRY(cudaGetLastError());
+        scan_offsets<<<tiles, kScanThreads, 0, s>>>(lengths, N, tile_sums, ws_offsets);
+        SBW_CUDA_TRY(cudaGetLastError());
+        a.offsets = ws_offsets;
+    }
+    const unsigned grid = static_cast<unsigned>((N + kDetectThreads / 32 - 1) / (kDetectThreads / 32));
+    if (scheme == SBW_SCHEME_CONTEXT)
+        detect_kernel<SBW_SCHEME_CONTEXT><<<grid, kDetectThreads, 0, s>>>(a);
+    else
+        detect_kernel<SBW_SCHEME_SELFSALT><<<grid, kDetectThreads, 0, s>>>(a);
+    SBW_CUDA_TRY(cudaGetLastError());
+    return SBW_OK;
+}

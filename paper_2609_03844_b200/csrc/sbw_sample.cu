@@ -1,0 +1,497 @@
+// sbw_bias_sample: the bias of Eq. 1 + Eq. 2 fused with temperature softmax statistics and
+// Gumbel-max sampling, in one read-only pass over the [B, V] logits.  The paper leaves sampling
+// to the serving engine; this kernel is the "absorbed into existing logit post-processing" form
+// that Section 5.1 points at.
+//
+// Work layout.  A row is cut into 16-byte slots as in the bias kernel; a row may further be split
+// into `split` column chunks so that small batches still fill the 148 SMs.  One CTA handles one
+// (row, chunk): every thread keeps an online-softmax pair (running max m, sum of
+// exp2((l' - m) c)) and its best Gumbel score, all in registers; a CTA reduces them with warp
+// shuffles (max, then sum of rescaled partial sums, then lexicographic argmax) and shared memory
+// across its warps.  When a row is split, CTAs leave their partial in the workspace and the last
+// one to arrive (an atomic ticket, nobody waits) merges the row's partials in index order.
+//
+// Numerics.  The sampled id must be reproducible bit for bit, so everything that feeds it is an
+// exactly rounded fp32 operation spelled with intrinsics: the Gumbel variate is -L(-L(u)) with L
+// the fixed logarithm below, and the score is fmaf(l', 1/tau, g).  The softmax sum only has to be
+// accurate (1e-6 relative): exponent arguments are formed as a rounded product plus its exact
+// rounding error, exp2 of the rounded part comes from the SFU (2 ulp), and the error term is
+// applied to first order.  The per-row finish (merging chunk partials, p = exp(.)/Z) is fp64.
+#include <cuda_bf16.h>
+
+#include <cfloat>
+#include <climits>
+
+#include "sbw_common.cuh"
+#include "sbw_hash.cuh"
+
+namespace sbw {
+namespace {
+
+constexpr int kSampleThreads = 256;
+constexpr int kSampleWarps = kSampleThreads / 32;
+constexpr int kTargetCtas = 1184;      // 148 SMs x 8: enough CTAs to fill the GPU twice over
+constexpr int kMinSlotsPerCta = 256;   // one slot per thread at least
+
+struct __align__(32) Partial {
+    float m;      // max of l' over the chunk
+    float z;      // sum of exp((l' - m)/tau) over the chunk
+    float s;      // best Gumbel score
+    int id;       // its column (INT_MAX: none)
+    float l;      // its biased logit
+    float pad[3];
+};
+
+struct SampleArgs {
+    const void *logits;
+    int64_t B, V, ld;
+    uint32_t nslot, slots_per_chunk;
+    int split;
+    const int32_t *ctx;
+    int W;
+    uint32_t vocab_offset;
+    uint64_t key;
+    uint32_t thr_m1;
+    float delta;          // in the logits' precision, widened
+    float inv_tau;        // 1/tau rounded once to fp32 (feeds the score)
+    float c2_hi, c2_lo;   // log2(e)/tau as an fp32 pair (feeds the softmax sum)
+    double tau;
+    uint32_t gk0, gk1, step_lo, step_hi;   // Gumbel stream
+    int32_t *out_tokens;
+    float *out_max, *out_sumexp, *out_prob;
+    Partial *partials;    // [B * split]
+    unsigned *tickets;    // [B], zero before the launch
+    double2 *rowstats;    // [B] (m, Z) for the optional probabilities pass
+};
+
+// ---------------------------------------------------------------------------------------------
+// Fixed fp32 natural logarithm for positive normal x; every step is one IEEE operation.
+//   ix = bits(x); e = (int)(ix - 0x3f3504f3) >> 23; m = bits^-1(ix - (e << 23)) in [sqrt(1/2), sqrt(2))
+//   f = m - 1; r = Horner_{C6..C0}(f); q = fma(r, f, -1/2); t = fma(f*f, q, f)
+//   L = fma(e, LN2_HI, fma(e, LN2_LO, t))
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float fixed_log(float x) {
+    const uint32_t ix = __float_as_uint(x);
+    const int e = static_cast<int>(ix - 0x3f3504f3u) >> 23;
+    const float m = __uint_as_float(ix - (static_cast<uint32_t>(e) << 23));
+    const float f = __fadd_rn(m, -1.0f);
+    float r = 0x1.645de2p-4f;
+    r = __fmaf_rn(r, f, -0x1.2432aap-3f);
+    r = __fmaf_rn(r, f, 0x1.31747p-3f);
+    r = __fmaf_rn(r, f, -0x1.53824cp-3f);
+    r = __fmaf_rn(r, f, 0x1.98d7fp-3f);
+    r = __fmaf_rn(r, f, -0x1.000382p-2f);
+    r = __fmaf_rn(r, f, 0x1.5556d8p-2f);
+    const float q = __fmaf_rn(r, f, -0.5f);
+    const float t = __fmaf_rn(__fmul_rn(f, f), q, f);
+    const float fe = __int2float_rn(e);
+    return __fmaf_rn(fe, 0x1.62e43p-1f, __fmaf_rn(fe, -0x1.05c61p-29f, t));
+}
+
+// -L(u) for the uniform built from a Philox word: u = ((y >> 9) + 1/2) 2^-23 (exact in fp32).
+__device__ __forceinline__ float neg_log_uniform(uint32_t y) {
+    const float u = __fmaf_rn(__uint2float_rn(y >> 9), 0x1p-23f, 0x1p-24f);
+    return -fixed_log(u);
+}
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// exp2(d * c) for d <= 0 with c = c_hi + c_lo: returns e = exp2(round(d c_hi)) and the residual
+// `lo` such that the true value is e * 2^lo ~ e * (1 + lo ln 2).
+__device__ __forceinline__ float exp2_split(float d, float c_hi, float c_lo, float &lo) {
+    d = fmaxf(d, -1e15f);                       // keeps -inf logits finite below
+    const float hi = __fmul_rn(d, c_hi);
+    lo = __fmaf_rn(d, c_lo, __fmaf_rn(d, c_hi, -hi));
+    return ex2_approx(hi);
+}
+__device__ __forceinline__ float exp2_scaled(float d, float c_hi, float c_lo) {
+    float lo;
+    const float e = exp2_split(d, c_hi, c_lo, lo);
+    return __fmaf_rn(e, lo * 0.693147180559945f, e);
+}
+
+struct Best {
+    float s;
+    int id;
+    float l;
+};
+__device__ __forceinline__ bool better(float s1, int id1, float s2, int id2) {
+    return s1 > s2 || (s1 == s2 && id1 < id2);
+}
+
+template <int SCHEME>
+struct RowSeedS;
+template <>
+struct RowSeedS<SBW_SCHEME_CONTEXT> {
+    RowKeys rk;
+    __device__ __forceinline__ void init(uint64_t key, const int32_t *ctx, int W) {
+        rk = make_row_keys(seed_context(key, ctx, W));
+    }
+    __device__ __forceinline__ uint32_t word0(uint32_t v, uint64_t) const { return philox_word0(v, rk); }
+};
+template <>
+struct RowSeedS<SBW_SCHEME_SELFSALT> {
+    uint32_t jmin;
+    __device__ __forceinline__ void init(uint64_t, const int32_t *ctx, int W) { jmin = jenkins_min(ctx, W); }
+    __device__ __forceinline__ uint32_t word0(uint32_t v, uint64_t key) const {
+        return philox_word0(v, seed_selfsalt(key, jmin, v));
+    }
+};
+
+// Biased logit of one element, widened to fp32 (Eq. 2 in the logits' own precision).
+template <int DTYPE>
+__device__ __forceinline__ float biased(uint32_t raw, bool green, float delta) {
+    if constexpr (DTYPE == SBW_DTYPE_F32) {
+        const float x = __uint_as_float(raw);
+        return green ? __fadd_rn(x, delta) : x;
+    } else {
+        const float x = __uint_as_float(raw << 16);
+        // fp32 sum of two bf16 values, rounded once more to bf16 = correctly rounded bf16 sum
+        return green ? __bfloat162float(__float2bfloat16_rn(__fadd_rn(x, delta))) : x;
+    }
+}
+
+// Final per-row merge of `n` partials in index order, by one warp; fp64.
+__device__ void finish_row(const SampleArgs &a, int64_t row, const Partial *parts, int n) {
+    const int lane = threadIdx.x & 31;
+    double m = -INFINITY, Z = 0.0;
+    float s = -INFINITY, l = -INFINITY;
+    int id = INT_MAX;
+    for (int i = lane; i < n; i += 32) {
+        // L2 loads: the partials were written by other SMs during this launch
+        const float4 q0 = __ldcg(reinterpret_cast<const float4 *>(parts + i));
+        const float4 q1 = __ldcg(reinterpret_cast<const float4 *>(parts + i) + 1);
+        Partial p;
+        p.m = q0.x; p.z = q0.y; p.s = q0.z; p.id = __float_as_int(q0.w); p.l = q1.x;
+        const double pm = p.m;
+        if (pm > -INFINITY) {
+            if (pm > m) {
+                Z = Z * exp((m - pm) / a.tau) + p.z;     // exp(-inf) = 0 on the first one
+                m = pm;
+            } else {
+                Z += p.z * exp((pm - m) / a.tau);
+            }
+        }
+        if (better(p.s, p.id, s, id)) { s = p.s; id = p.id; l = p.l; }
+    }
+    for (int d = 16; d > 0; d >>= 1) {
+        const double om = __shfl_down_sync(0xffffffffu, m, d);
+        const double oZ = __shfl_down_sync(0xffffffffu, Z, d);
+        const float os = __shfl_down_sync(0xffffffffu, s, d);
+        const int oid = __shfl_down_sync(0xffffffffu, id, d);
+        const float ol = __shfl_down_sync(0xffffffffu, l, d);
+        if (om > -INFINITY) {
+            if (om > m) {
+                Z = Z * exp((m - om) / a.tau) + oZ;
+                m = om;
+            } else {
+                Z += oZ * exp((om - m) / a.tau);
+            }
+        }
+        if (better(os, oid, s, id)) { s = os; id = oid; l = ol; }
+    }
+    if (lane == 0) {
+        if (id == INT_MAX) id = 0;                       // every score was -inf: lowest id
+        a.out_tokens[row] = id;
+        if (a.out_max) a.out_max[row] = static_cast<float>(m);
+        if (a.out_sumexp) a.out_sumexp[row] = static_cast<float>(Z);
+        if (a.out_prob) a.out_prob[row] = static_cast<float>(exp((static_cast<double>(l) - m) / a.tau) / Z);
+        a.rowstats[row] = make_double2(m, Z);
+    }
+}
+
+template <int DTYPE, int SCHEME, bool VECTOR>
+__global__ void __launch_bounds__(kSampleThreads)
+sample_kernel(const SampleArgs a) {
+    constexpr int VEC = VECTOR ? (DTYPE == SBW_DTYPE_F32 ? 4 : 8) : 1;
+    constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
+    constexpr int NBLK = VEC >= 4 ? VEC / 4 : 1;     // Philox blocks per aligned slot
+    __shared__ float sh_f[kSampleWarps];
+    __shared__ float sh_s[kSampleWarps];
+    __shared__ int sh_id[kSampleWarps];
+    __shared__ float sh_l[kSampleWarps];
+    __shared__ unsigned sh_ticket;
+
+    const int64_t row = blockIdx.x / a.split;
+    const int chunk = static_cast<int>(blockIdx.x - row * a.split);
+    const uint32_t j_begin = chunk * a.slots_per_chunk;
+    const uint32_t j_end = min(a.nslot, j_begin + a.slots_per_chunk);
+    const uint32_t V = static_cast<uint32_t>(a.V);
+    const uint32_t rowb = static_cast<uint32_t>(row);
+    const char *row_ptr = static_cast<const char *>(a.logits) + row * a.ld * ESIZE;
+
+    RowSeedS<SCHEME> rs;
+    rs.init(a.key, a.ctx + row * a.W, a.W);
+
+    float m_t = -INFINITY, z1 = 0.0f, z2 = 0.0f;
+    Best best = {-INFINITY, INT_MAX, -INFINITY};
+
+    for (uint32_t j = j_begin + threadIdx.x; j < j_end; j += kSampleThreads) {
+        const uint32_t cb = j * VEC;
+        const uint32_t vg = a.vocab_offset + cb;
+        float lp[VEC];
+        uint32_t y[VEC];
+        int nvalid = VEC;
+        if (VECTOR && cb + VEC <= V) {
+            const uint4 w = __ldg(reinterpret_cast<const uint4 *>(row_ptr) + j);
+            const uint32_t *e = reinterpret_cast<const uint32_t *>(&w);
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                uint32_t raw;
+                if constexpr (DTYPE == SBW_DTYPE_F32) raw = e[i];
+                else raw = (i & 1) ? (e[i >> 1] >> 16) : (e[i >> 1] & 0xffffu);
+                const bool green = rs.word0(vg + i, a.key) <= a.thr_m1;
+                lp[i] = biased<DTYPE>(raw, green, a.delta);
+            }
+        } else {
+            nvalid = static_cast<int>(min(static_cast<uint32_t>(VEC), V - cb));
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                lp[i] = -INFINITY;
+                if (i < nvalid) {
+                    uint32_t raw;
+                    if constexpr (DTYPE == SBW_DTYPE_F32) raw = reinterpret_cast<const uint32_t *>(row_ptr)[cb + i];
+                    else raw = reinterpret_cast<const uint16_t *>(row_ptr)[cb + i];
+                    const bool green = rs.word0(vg + i, a.key) <= a.thr_m1;
+                    lp[i] = biased<DTYPE>(raw, green, a.delta);
+                }
+            }
+        }
+        // Gumbel words: candidate vg+i uses word (vg+i)&3 of block (vg+i)>>2
+        if (VEC >= 4 && (vg & 3u) == 0) {
+#pragma unroll
+            for (int b = 0; b < NBLK; ++b) {
+                const uint4 r = philox4x32_10((vg >> 2) + b, rowb, a.step_lo, a.step_hi, a.gk0, a.gk1);
+                if (4 * b + 0 < VEC) y[4 * b + 0] = r.x;
+                if (4 * b + 1 < VEC) y[4 * b + 1] = r.y;
+                if (4 * b + 2 < VEC) y[4 * b + 2] = r.z;
+                if (4 * b + 3 < VEC) y[4 * b + 3] = r.w;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                const uint32_t v = vg + i;
+                const uint4 r = philox4x32_10(v >> 2, rowb, a.step_lo, a.step_hi, a.gk0, a.gk1);
+                const uint32_t k = v & 3u;
+                y[i] = k == 0 ? r.x : k == 1 ? r.y : k == 2 ? r.z : r.w;
+            }
+        }
+        // online softmax
+        float vmax = lp[0];
+#pragma unroll
+        for (int i = 1; i < VEC; ++i) vmax = fmaxf(vmax, lp[i]);
+        if (vmax > m_t) {
+            const float f = exp2_scaled(m_t - vmax, a.c2_hi, a.c2_lo);   // 0 when m_t = -inf
+            z1 *= f;
+            z2 *= f;
+            m_t = vmax;
+        }
+        if (m_t > -INFINITY) {
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                float lo;
+                const float e = exp2_split(lp[i] - m_t, a.c2_hi, a.c2_lo, lo);
+                z1 += e;
+                z2 = fmaf(e, lo, z2);
+            }
+        }
+        // Gumbel-max
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+            if (i < nvalid) {
+                const float w = neg_log_uniform(y[i]);
+                const float s = __fmaf_rn(lp[i], a.inv_tau, -fixed_log(w));
+                if (s > best.s) { best.s = s; best.id = static_cast<int>(cb + i); best.l = lp[i]; }
+            }
+        }
+    }
+
+    // ---- CTA reduction ----
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float m_w = m_t;
+    for (int d = 16; d > 0; d >>= 1) m_w = fmaxf(m_w, __shfl_xor_sync(0xffffffffu, m_w, d));
+    if (lane == 0) sh_f[warp] = m_w;
+    __syncthreads();
+    float m_cta = sh_f[0];
+#pragma unroll
+    for (int w = 1; w < kSampleWarps; ++w) m_cta = fmaxf(m_cta, sh_f[w]);
+    __syncthreads();
+    float z_t = 0.0f;
+    if (m_t > -INFINITY) z_t = (z1 + 0.693147180559945f * z2) * exp2_scaled(m_t - m_cta, a.c2_hi, a.c2_lo);
+    for (int d = 16; d > 0; d >>= 1) z_t += __shfl_down_sync(0xffffffffu, z_t, d);
+    for (int d = 16; d > 0; d >>= 1) {
+        const float os = __shfl_down_sync(0xffffffffu, best.s, d);
+        const int oid = __shfl_down_sync(0xffffffffu, best.id, d);
+        const float ol = __shfl_down_sync(0xffffffffu, best.l, d);
+        if (better(os, oid, best.s, best.id)) { best.s = os; best.id = oid; best.l = ol; }
+    }
+    if (lane == 0) { sh_f[warp] = z_t; sh_s[warp] = best.s; sh_id[warp] = best.id; sh_l[warp] = best.l; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        Partial p;
+        p.m = m_cta;
+        p.z = 0.0f;
+        p.s = sh_s[0]; p.id = sh_id[0]; p.l = sh_l[0];
+        for (int w = 0; w < kSampleWarps; ++w) {
+            p.z += sh_f[w];
+            if (w > 0 && better(sh_s[w], sh_id[w], p.s, p.id)) { p.s = sh_s[w]; p.id = sh_id[w]; p.l = sh_l[w]; }
+        }
+        p.pad[0] = p.pad[1] = p.pad[2] = 0.0f;
+        a.partials[blockIdx.x] = p;
+        unsigned ticket = 0;
+        __threadfence();                           // partial visible before the ticket is taken
+        if (a.split > 1) ticket = atomicAdd(&a.tickets[row], 1u);
+        sh_ticket = ticket;
+    }
+    __syncthreads();
+    if (a.split > 1 && sh_ticket != static_cast<unsigned>(a.split - 1)) return;
+    if (warp == 0) {
+        if (a.split > 1) __threadfence();          // the other CTAs' partials are visible now
+        finish_row(a, row, a.partials + row * a.split, a.split);
+        if (lane == 0 && a.split > 1) a.tickets[row] = 0;
+    }
+}
+
+// Optional second pass: the full softmax of the biased logits, fp64 per element.
+template <int DTYPE, int SCHEME>
+__global__ void __launch_bounds__(256)
+probs_kernel(const SampleArgs a, float *out_probs) {
+    constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
+    for (int64_t row = blockIdx.y; row < a.B; row += gridDim.y) {
+        RowSeedS<SCHEME> rs;
+        rs.init(a.key, a.ctx + row * a.W, a.W);
+        const double2 st = a.rowstats[row];
+        const char *row_ptr = static_cast<const char *>(a.logits) + row * a.ld * ESIZE;
+        for (int64_t c = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; c < a.V;
+             c += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+            uint32_t raw;
+            if constexpr (DTYPE == SBW_DTYPE_F32) raw = reinterpret_cast<const uint32_t *>(row_ptr)[c];
+            else raw = reinterpret_cast<const uint16_t *>(row_ptr)[c];
+            const uint32_t v = a.vocab_offset + static_cast<uint32_t>(c);
+            const bool green = rs.word0(v, a.key) <= a.thr_m1;
+            const double lp = biased<DTYPE>(raw, green, a.delta);
+            out_probs[row * a.V + c] = static_cast<float>(exp((lp - st.x) / a.tau) / st.y);
+        }
+    }
+}
+
+int choose_split(int64_t B, int64_t nslot) {
+    int64_t split = (kTargetCtas + B - 1) / B;
+    const int64_t max_split = nslot / kMinSlotsPerCta > 1 ? nslot / kMinSlotsPerCta : 1;
+    if (split > max_split) split = max_split;
+    if (split < 1) split = 1;
+    return static_cast<int>(split);
+}
+
+struct Workspace {
+    double2 *rowstats;
+    unsigned *tickets;
+    Partial *partials;
+    size_t bytes;
+};
+Workspace carve(void *base, int64_t B) {
+    Workspace w;
+    char *p = static_cast<char *>(base);
+    size_t off = 0;
+    w.rowstats = reinterpret_cast<double2 *>(p + off);
+    off += align_up(static_cast<size_t>(B) * sizeof(double2), 256);
+    w.tickets = reinterpret_cast<unsigned *>(p + off);
+    off += align_up(static_cast<size_t>(B) * sizeof(unsigned), 256);
+    w.partials = reinterpret_cast<Partial *>(p + off);
+    off += align_up(static_cast<size_t>(B + kTargetCtas) * sizeof(Partial), 256);
+    w.bytes = off;
+    return w;
+}
+
+template <int DTYPE, int SCHEME>
+int launch(const SampleArgs &a, bool vector, float *out_probs, cudaStream_t s) {
+    const unsigned grid = static_cast<unsigned>(a.B * a.split);
+    if (vector) sample_kernel<DTYPE, SCHEME, true><<<grid, kSampleThreads, 0, s>>>(a);
+    else sample_kernel<DTYPE, SCHEME, false><<<grid, kSampleThreads, 0, s>>>(a);
+    SBW_CUDA_TRY(cudaGetLastError());
+    if (out_probs) {
+        const unsigned gx = static_cast<unsigned>((a.V + 255) / 256 < 1024 ? (a.V + 255) / 256 : 1024);
+        const unsigned gy = static_cast<unsigned>(a.B < 4096 ? a.B : 4096);
+        probs_kernel<DTYPE, SCHEME><<<dim3(gx, gy), 256, 0, s>>>(a, out_probs);
+        SBW_CUDA_TRY(cudaGetLastError());
+    }
+    return SBW_OK;
+}
+
+}  // namespace
+}  // namespace sbw
+
+extern "C" size_t sbw_sample_workspace_bytes(int64_t B, int64_t V) {
+    if (B <= 0 || V <= 0) return 0;
+    return sbw::carve(nullptr, B).bytes;
+}
+
+extern "C" int sbw_bias_sample(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
+                               int64_t vocab_offset, const int32_t *ctx_tokens, int ctx_width,
+                               uint64_t key, double gamma, float delta, int scheme, float temperature,
+                               uint64_t rng_seed, uint64_t rng_step, int32_t *out_tokens, float *out_max,
+                               float *out_sumexp, float *out_prob, float *out_probs, void *workspace,
+                               size_t workspace_bytes, void *stream) {
+    using namespace sbw;
+    if (!valid_common(dtype, ctx_width, gamma, scheme)) return SBW_ERR_INVALID_ARG;
+    if (B < 0 || V <= 0 || ld < V || vocab_offset < 0) return SBW_ERR_INVALID_ARG;
+    if (!(temperature > 0.0f) || temperature - temperature != 0.0f) return SBW_ERR_INVALID_ARG;
+    if (!(delta == delta) || delta - delta != 0.0f) return SBW_ERR_INVALID_ARG;
+    if (V > 0x7fffffffLL) return SBW_ERR_UNSUPPORTED;
+    if (B == 0) return SBW_OK;
+    if (!logits || !ctx_tokens || !out_tokens) return SBW_ERR_INVALID_ARG;
+    const double c2 = 1.4426950408889634 / static_cast<double>(temperature);
+    const float c2_hi = static_cast<float>(c2);
+    if (!(c2_hi * 1e15f < FLT_MAX)) return SBW_ERR_INVALID_ARG;   // temperature too small
+    const Workspace ws = carve(workspace, B);
+    if (!workspace || workspace_bytes < ws.bytes || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
+        return SBW_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    const int esize = dtype == SBW_DTYPE_F32 ? 4 : 2;
+    const bool vector = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && ((ld * esize) % 16 == 0);
+    const int vec = vector ? 16 / esize : 1;
+    const int64_t nslot = (V + vec - 1) / vec;
+    if (B * static_cast<int64_t>(choose_split(B, nslot)) > 0x7fffffffLL) return SBW_ERR_UNSUPPORTED;
+
+    SampleArgs a;
+    a.logits = logits;
+    a.B = B; a.V = V; a.ld = ld;
+    a.nslot = static_cast<uint32_t>(nslot);
+    a.split = choose_split(B, nslot);
+    a.slots_per_chunk = static_cast<uint32_t>((nslot + a.split - 1) / a.split);
+    a.ctx = ctx_tokens;
+    a.W = ctx_width;
+    a.vocab_offset = static_cast<uint32_t>(vocab_offset);
+    a.key = key;
+    a.thr_m1 = threshold_minus_one(gamma);
+    a.delta = dtype == SBW_DTYPE_BF16 ? __bfloat162float(__float2bfloat16_rn(delta)) : delta;
+    a.inv_tau = 1.0f / temperature;
+    a.c2_hi = c2_hi;
+    a.c2_lo = static_cast<float>(c2 - static_cast<double>(c2_hi));
+    a.tau = static_cast<double>(temperature);
+    a.gk0 = static_cast<uint32_t>(rng_seed);
+    a.gk1 = static_cast<uint32_t>(rng_seed >> 32);
+    a.step_lo = static_cast<uint32_t>(rng_step);
+    a.step_hi = static_cast<uint32_t>(rng_step >> 32);
+    a.out_tokens = out_tokens;
+    a.out_max = out_max;
+    a.out_sumexp = out_sumexp;
+    a.out_prob = out_prob;
+    a.partials = ws.partials;
+    a.tickets = ws.tickets;
+    a.rowstats = ws.rowstats;
+
+    if (a.split > 1)
+        SBW_CUDA_TRY(cudaMemsetAsync(ws.tickets, 0, static_cast<size_t>(B) * sizeof(unsigned), s));
+    if (dtype == SBW_DTYPE_F32) {
+        return scheme == SBW_SCHEME_CONTEXT ? launch<SBW_DTYPE_F32, SBW_SCHEME_CONTEXT>(a, vector, out_probs, s)
+                                            : launch<SBW_DTYPE_F32, SBW_SCHEME_SELFSALT>(a, vector, out_probs, s);
+    }
+    return scheme == SBW_SCHEME_CONTEXT ? launch<SBW_DTYPE_BF16, SBW_SCHEME_CONTEXT>(a, vector, out_probs, s)
+                                        : launch<SBW_DTYPE_BF16, SBW_SCHEME_SELFSALT>(a, vector, out_probs, s);
+}

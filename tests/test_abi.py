@@ -1,0 +1,108 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+headers declare, and rejects bad arguments before touching the device."""
+import ctypes
+import re
+from pathlib import Path
+
+import pytest
+
+import paper_2609_03844_b200 as sbw
+from paper_2609_03844_b200 import binding
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+def _declared():
+    names = set()
+    for h in sorted((ROOT / "include").glob("*.h")):
+        text = re.sub(r"/\*.*?\*/", "", h.read_text(), flags=re.S)
+        names |= set(re.findall(r"\b(sbw_[a-z0-9_]+)\s*\(", text))
+    return names
+
+
+def test_library_loads_and_exports_every_declared_symbol():
+    L = sbw.lib()
+    declared = _declared()
+    assert {"sbw_bias_logits", "sbw_bias_sample", "sbw_detect", "sbw_version"} <= declared
+    for name in declared:
+        assert hasattr(L, name), f"{name} declared in include/ but not exported by libsbw.so"
+    assert set(binding.EXPORTS) <= declared
+    assert "sm_100a" in sbw.sbw_version()
+
+
+def test_binding_has_the_same_names():
+    for name in ("sbw_bias_logits", "sbw_bias_logits_host", "sbw_bias_sample", "sbw_detect",
+                 "sbw_sample_workspace_bytes", "sbw_detect_workspace_bytes", "sbw_version"):
+        assert callable(getattr(sbw, name))
+
+
+def test_workspace_size_queries():
+    assert sbw.sbw_sample_workspace_bytes(0, 128256) == 0
+    a = sbw.sbw_sample_workspace_bytes(1, 128256)
+    b = sbw.sbw_sample_workspace_bytes(1024, 128256)
+    assert 0 < a < b and a % 256 == 0 and b % 256 == 0
+    assert sbw.sbw_detect_workspace_bytes(0) == 0
+    assert sbw.sbw_detect_workspace_bytes(100000) >= 8 * 100001
+    assert sbw.sbw_bias_logits_host_staging_bytes(__import__("torch").bfloat16, 64, 128256, 1) >= \
+        64 * 128256 * 2 + 64 * 4
+
+
+def test_argument_validation_happens_on_the_host():
+    """Every rejected call returns before any CUDA work, so this runs without a device."""
+    L = sbw.lib()
+    fake = ctypes.c_void_p(0x1000)          # never dereferenced on the host
+    ok = dict(dtype=0, B=2, V=8, ld=8, off=0, W=1, key=1, gamma=0.25, delta=2.0, scheme=0)
+
+    def bias(**kw):
+        a = {**ok, **kw}
+        return L.sbw_bias_logits(a.get("logits", fake), a["dtype"], a["B"], a["V"], a["ld"], a["off"],
+                                 a.get("ctx", fake), a["W"], a["key"], a["gamma"], a["delta"],
+                                 a["scheme"], None)
+
+    assert bias(B=0) == binding.SBW_OK
+    assert bias(B=0, logits=None, ctx=None) == binding.SBW_OK
+    for bad in (dict(gamma=0.0), dict(gamma=1.0), dict(gamma=-0.1), dict(gamma=float("nan")),
+                dict(V=0), dict(V=-3), dict(ld=7), dict(B=-1), dict(dtype=2), dict(scheme=5),
+                dict(W=0), dict(W=9), dict(off=-1), dict(logits=None), dict(ctx=None),
+                dict(delta=float("nan")), dict(delta=float("inf"))):
+        assert bias(**bad) == binding.SBW_ERR_INVALID_ARG, bad
+    assert bias(V=1 << 31, ld=1 << 31) == binding.SBW_ERR_UNSUPPORTED
+    # delta = 0 is the paper's control: accepted, nothing to do
+    assert bias(delta=0.0) == binding.SBW_OK
+
+    def sample(**kw):
+        a = {**ok, "tau": 0.7, "ws": fake, "ws_bytes": 1 << 20, **kw}
+        return L.sbw_bias_sample(a.get("logits", fake), a["dtype"], a["B"], a["V"], a["ld"], a["off"],
+                                 a.get("ctx", fake), a["W"], a["key"], a["gamma"], a["delta"],
+                                 a["scheme"], a["tau"], 1, 2, a.get("out", fake), None, None, None,
+                                 None, a["ws"], a["ws_bytes"], None)
+
+    assert sample(B=0) == binding.SBW_OK
+    for bad in (dict(tau=0.0), dict(tau=-1.0), dict(tau=float("nan")), dict(tau=1e-30),
+                dict(gamma=1.5), dict(out=None), dict(logits=None), dict(ld=3)):
+        assert sample(**bad) == binding.SBW_ERR_INVALID_ARG, bad
+    assert sample(ws=None) == binding.SBW_ERR_WORKSPACE
+    assert sample(ws_bytes=16) == binding.SBW_ERR_WORKSPACE
+    assert sample(ws=ctypes.c_void_p(0x1008)) == binding.SBW_ERR_WORKSPACE   # not 256-aligned
+
+    def detect(**kw):
+        a = dict(N=4, total=40, W=1, gamma=0.25, scheme=0, ws=fake, ws_bytes=1 << 20, off=None)
+        a.update(kw)
+        return L.sbw_detect(a.get("tokens", fake), a.get("lengths", fake), a["off"], a["N"], a["total"],
+                            a["W"], 1, a["gamma"], a["scheme"], a.get("counts", fake), None,
+                            a.get("z", fake), a["ws"], a["ws_bytes"], None)
+
+    assert detect(N=0) == binding.SBW_OK
+    for bad in (dict(gamma=0.0), dict(N=-1), dict(total=-5), dict(W=0), dict(scheme=2),
+                dict(lengths=None), dict(counts=None), dict(z=None), dict(tokens=None)):
+        assert detect(**bad) == binding.SBW_ERR_INVALID_ARG, bad
+    assert detect(ws=None, ws_bytes=0) == binding.SBW_ERR_WORKSPACE
+    assert detect(ws_bytes=8) == binding.SBW_ERR_WORKSPACE
+    assert L.sbw_last_cuda_error() == 0
+
+
+def test_python_binding_type_checks():
+    import torch
+
+    with pytest.raises(ValueError):
+        sbw.sbw_bias_logits(torch.zeros(2, 8), torch.zeros(2, 1, dtype=torch.int32), 1, 0.25, 2.0, 0)

@@ -1,0 +1,161 @@
+"""GPU parity of sbw_bias_logits (Eq. 1 + Eq. 2) against the CPU oracle: biased logits must be
+bit-identical, element by element, on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_03844_b200 as sbw
+from paper_2609_03844_b200 import inputs
+from gpu_util import KEY, assert_same_bits, host_bits, require_gpu
+
+pytestmark = pytest.mark.gpu
+
+SCHEMES = [sbw.SCHEME_CONTEXT, sbw.SCHEME_SELFSALT]
+DTYPES = [torch.float32, torch.bfloat16]
+
+
+def _run(x_host: torch.Tensor, V, ctx_host: torch.Tensor, key, gamma, delta, scheme, off=0,
+         view=None):
+    """Runs the CUDA path on a device copy and the oracle on the host bytes; returns both."""
+    dev = require_gpu()
+    x_dev = x_host.to(dev)
+    target = x_dev if view is None else view(x_dev)
+    host_view = x_host if view is None else view(x_host)
+    sbw.sbw_bias_logits(target, ctx_host.to(dev), key, gamma, delta, scheme, V=V, vocab_offset=off)
+    torch.cuda.synchronize()
+    want = oracle.bias_logits(host_bits(host_view.contiguous()) if view is not None else host_bits(x_host),
+                              V, ctx_host.numpy(), key, gamma, delta, scheme, vocab_offset=off, threads=8)
+    got_full = host_bits(x_dev)
+    got = host_bits(target.contiguous()) if view is not None else got_full
+    return got, want, got_full
+
+
+def test_config1_fp32_context():
+    """B=1, V=32000, fp32 N(0, 3^2) from seed 0, one context token, key 0x5EED, gamma .25, delta 2."""
+    x = inputs.logits_normal(1, 32000, 3.0, torch.float32, seed=0)
+    ctx = inputs.uniform_tokens((1, 1), 32000, seed=1)
+    got, want, _ = _run(x, 32000, ctx, KEY, 0.25, 2.0, sbw.SCHEME_CONTEXT)
+    assert_same_bits(got, want)
+    changed = (got != host_bits(x)).mean()
+    assert 0.23 < changed < 0.27
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("scheme", SCHEMES)
+@pytest.mark.parametrize("W", [1, 4])
+def test_several_tiles_ragged_tail_padding_offset(dtype, scheme, W):
+    """Rows span several CTAs' shares, V is not a multiple of the vector width, ld > V."""
+    B, V, ld, off = 37, 10007, 10016, 123457
+    x = inputs.logits_normal(B, V, 4.0, dtype, seed=2, ld=ld)
+    ctx = inputs.uniform_tokens((B, W), 151936, seed=3)
+    got, want, _ = _run(x, V, ctx, KEY, 0.5, 2.0, scheme, off=off)
+    assert_same_bits(got, want)
+    assert np.array_equal(got[:, V:], host_bits(x)[:, V:])          # padding untouched
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("scheme", SCHEMES)
+def test_unaligned_rows_take_the_scalar_path(dtype, scheme):
+    """Odd row stride and a base pointer that is not 16-byte aligned (a column slice)."""
+    B, V = 9, 1001
+    x = inputs.logits_normal(B, V + 3, 4.0, dtype, seed=4)
+    ctx = inputs.uniform_tokens((B, 1), 50000, seed=5)
+    got, want, full = _run(x, V, ctx, KEY, 0.25, 1.0, scheme, view=lambda t: t[:, 1:V + 1])
+    assert_same_bits(got, want)
+    ref = host_bits(x)
+    assert np.array_equal(full[:, 0], ref[:, 0]) and np.array_equal(full[:, V + 1:], ref[:, V + 1:])
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("V", [1, 3, 7, 8, 9, 31, 33])
+def test_tiny_vocabularies_and_empty_batch(dtype, V):
+    x = inputs.logits_normal(5, V, 4.0, dtype, seed=6 + V)
+    ctx = inputs.uniform_tokens((5, 1), 1000, seed=7)
+    for scheme in SCHEMES:
+        got, want, _ = _run(x, V, ctx, KEY, 0.5, 2.0, scheme)
+        assert_same_bits(got, want)
+    dev = require_gpu()
+    empty = torch.empty((0, V), dtype=dtype, device=dev)
+    sbw.sbw_bias_logits(empty, torch.empty((0, 1), dtype=torch.int32, device=dev), KEY, 0.5, 2.0, 0, V=V)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("delta", [0.0, -1.5, 0.3, 4.0, 1e-3])
+def test_delta_values_and_special_logits(dtype, delta):
+    """-0.0, +-inf, subnormals, huge values, NaN (payload not compared); delta = 0 changes no bit."""
+    B, V = 4, 4096
+    x = inputs.logits_normal(B, V, 4.0, dtype, seed=8)
+    specials = torch.tensor([0.0, -0.0, float("inf"), float("-inf"), 1e-40, -1e-40, 3e38, -3e38,
+                             float("nan"), 1.0, -2.0, 65504.0], dtype=torch.float32).to(dtype)
+    for b in range(B):
+        x[b, b * 100:b * 100 + len(specials)] = specials
+        x[b, 2000 + b:2000 + b + 24:2] = specials
+    ctx = inputs.uniform_tokens((B, 1), 32000, seed=9)
+    for scheme in SCHEMES:
+        got, want, _ = _run(x, V, ctx, KEY, 0.5, delta, scheme)
+        assert_same_bits(got, want, allow_nan_payload=True)
+        if delta == 0.0:
+            assert got.tobytes() == host_bits(x).tobytes()
+
+
+def test_config2_shape_one_step_bf16():
+    """B=64, V=128256 bf16 N(0, 4^2), context scheme, gamma .5, delta 2 -- every element."""
+    dev = require_gpu()
+    x = inputs.logits_normal(64, 128256, 4.0, torch.bfloat16, seed=20, device=dev)
+    ctx = inputs.uniform_tokens((64, 1), 128256, seed=21, device=dev)
+    before = host_bits(x)
+    sbw.sbw_bias_logits(x, ctx, KEY, 0.5, 2.0, sbw.SCHEME_CONTEXT)
+    torch.cuda.synchronize()
+    want = oracle.bias_logits(before, 128256, ctx.cpu().numpy(), KEY, 0.5, 2.0,
+                              oracle.SCHEME_CONTEXT, threads=8)
+    assert_same_bits(host_bits(x), want)
+
+
+def test_config3_shape_one_step_fp32_selfsalt_with_zipf_spike():
+    """B=256, V=151936 fp32 N(0, 4^2) + Zipf(1.1) spike on 50 ids per row, self-salt, gamma .25,
+    delta 4 -- every element."""
+    dev = require_gpu()
+    x = inputs.logits_normal(256, 151936, 4.0, torch.float32, seed=30, device=dev)
+    inputs.add_zipf_spike_(x, 151936, seed=31)
+    ctx = inputs.uniform_tokens((256, 1), 151936, seed=32, device=dev)
+    before = host_bits(x)
+    sbw.sbw_bias_logits(x, ctx, KEY, 0.25, 4.0, sbw.SCHEME_SELFSALT)
+    torch.cuda.synchronize()
+    want = oracle.bias_logits(before, 151936, ctx.cpu().numpy(), KEY, 0.25, 4.0,
+                              oracle.SCHEME_SELFSALT, threads=8)
+    assert_same_bits(host_bits(x), want)
+
+
+def test_consecutive_steps_on_a_side_stream_and_other_keys():
+    """Several decode steps enqueued back to back on a non-default stream, 64-bit keys."""
+    dev = require_gpu()
+    stream = torch.cuda.Stream()
+    steps = []
+    with torch.cuda.stream(stream):
+        for t in range(4):
+            x = inputs.logits_normal(16, 32000, 4.0, torch.bfloat16, seed=40 + t, device=dev)
+            ctx = inputs.uniform_tokens((16, 1), 32000, seed=50 + t, device=dev)
+            steps.append((x, host_bits(x), ctx))
+        stream.synchronize()
+        for t, (x, _, ctx) in enumerate(steps):
+            sbw.sbw_bias_logits(x, ctx, 0xFEDCBA9876543211 + t, 0.25, 1.0, t % 2, stream=stream)
+    stream.synchronize()
+    for t, (x, before, ctx) in enumerate(steps):
+        want = oracle.bias_logits(before, 32000, ctx.cpu().numpy(), 0xFEDCBA9876543211 + t, 0.25,
+                                  1.0, t % 2, threads=8)
+        assert_same_bits(host_bits(x), want)
+
+
+def test_host_buffer_entry_point():
+    dev = require_gpu()
+    B, V = 8, 32000
+    x = inputs.logits_normal(B, V, 4.0, torch.bfloat16, seed=60).pin_memory()
+    ctx = inputs.uniform_tokens((B, 1), V, seed=61).pin_memory()
+    before = host_bits(x)
+    nbytes = sbw.sbw_bias_logits_host_staging_bytes(torch.bfloat16, B, V, 1)
+    staging = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    sbw.sbw_bias_logits_host(x, ctx, KEY, 0.5, 2.0, sbw.SCHEME_CONTEXT, staging)
+    torch.cuda.synchronize()
+    want = oracle.bias_logits(before, V, ctx.numpy(), KEY, 0.5, 2.0, oracle.SCHEME_CONTEXT)
+    assert_same_bits(host_bits(x), want)

@@ -38,6 +38,8 @@ def test_bf16_add_matches_torch_on_every_bit_pattern(oracle, delta):
     t = torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16)
     d = torch.tensor(delta, dtype=torch.float32).to(torch.bfloat16)
     want = (t + d).view(torch.int16).numpy().view(np.uint16)
+    if float(d) == 0.0:
+        want = bits        # the paper's delta = 0 control: no add at all, -0.0 stays -0.0
     nan = torch.isnan(t).numpy()
     assert np.array_equal(got[~nan], want[~nan])
     g32 = torch.from_numpy(got.view(np.int16).copy()).view(torch.bfloat16)
