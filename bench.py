@@ -34,9 +34,10 @@ POOL = 256                          # distinct step inputs kept resident
 #   context scheme: Philox4x32-10 word 0 = 20 32x32->64 multiplies + 20 three-input xors, and one
 #   compare = 41 integer operations; 2 bytes read + 2 bytes written (bf16).
 INT_OPS = {"context": 41, "selfsalt": 80, "detect_context": 62, "detect_selfsalt": 100}
-# Integer ceiling of one B200: 148 SMs x 4 schedulers x 32 lanes = 18944 thread-operations per
-# clock (one warp instruction per scheduler per clock) at the 1965 MHz maximum SM clock.
-SMS, LANES_PER_SM_CLK, SM_MAX_MHZ = 148, 128, 1965.0
+# INT32 ceiling of one B200: 148 SMs x 64 INT32 lanes per SM per clock (16 per scheduler; the
+# probe measures 64 ops/clk/SM for integer add, logic and 32-bit multiply-add, and 32 for the
+# 32x32->64 multiply) at the 1965 MHz maximum SM clock = 18.6 T integer operations per second.
+SMS, LANES_PER_SM_CLK, SM_MAX_MHZ = 148, 64, 1965.0
 INT_PEAK_TOPS = SMS * LANES_PER_SM_CLK * SM_MAX_MHZ * 1e6 / 1e12
 # DRAM bytes per bias launch of the headline workload from the ncu capture summarised under
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
@@ -264,7 +265,7 @@ def run_ours(args) -> None:
     hbm_gbs = 4 * elems_step / launch_s / 1e9
     roofline = {"bound": "alu", "achieved": ach_tops, "peak": INT_PEAK_TOPS, "unit": "Tint-op/s",
                 "frac": ach_tops / INT_PEAK_TOPS, "traffic": NCU_TRAFFIC_BYTES,
-                "peak_source": "derived: 148 SMs x 4 schedulers x 32 lanes x 1965 MHz",
+                "peak_source": "derived: 148 SMs x 64 INT32 lanes x 1965 MHz",
                 "kernel": "bias_kernel<bf16, context, vector>", "avg_launch_us": launch_s * 1e6,
                 "int_ops_per_elem": INT_OPS["context"],
                 "hbm": {"achieved": hbm_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -421,6 +422,46 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
     return out
 
 
+PROFILE_CASES = ("bias_bf16_context", "bias_bf16_selfsalt", "bias_fp32_context", "bias_fp32_selfsalt",
+                 "detect_context", "detect_selfsalt", "sample_bf16_context", "sample_bf16_selfsalt")
+
+
+def run_profile_case(name: str, launches: int) -> None:
+    """A few launches of one kernel on an input larger than L2 and small enough for a profiler
+    capture (a few hundred MB): 3 warm-up launches, then `launches` more.  Prints the launch count;
+    numbers printed under a profiler are never bench values."""
+    import torch
+    import paper_2609_03844_b200 as sbw
+    from paper_2609_03844_b200 import inputs
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    kind, dt, scheme_name = (name.split("_") + [""])[:3] if not name.startswith("detect") else \
+        ("detect", "", name.split("_")[1])
+    scheme = sbw.SCHEME_SELFSALT if scheme_name == "selfsalt" else sbw.SCHEME_CONTEXT
+    if kind == "detect":
+        N = 100000
+        tokens, lengths = inputs.null_token_streams(N, 64, 1024, V2, seed=500, device=dev)
+        counts = torch.empty(N, dtype=torch.int32, device=dev)
+        z = torch.empty(N, dtype=torch.float64, device=dev)
+        ws = torch.empty(sbw.sbw_detect_workspace_bytes(N), dtype=torch.uint8, device=dev)
+        fn = lambda i: sbw.sbw_detect(tokens, lengths, KEY, 0.25, scheme, counts, z, workspace=ws)  # noqa: E731
+    else:
+        B, V, dtype = (512, V2, torch.bfloat16) if dt == "bf16" else (256, 151936, torch.float32)
+        x = inputs.logits_normal(B, V, 4.0, dtype, seed=1, device=dev)
+        ctx = inputs.uniform_tokens((B, 1), V, seed=2, device=dev)
+        if kind == "bias":
+            fn = lambda i: sbw.sbw_bias_logits(x, ctx, KEY, 0.5, 2.0, scheme)  # noqa: E731
+        else:
+            ids = torch.empty(B, dtype=torch.int32, device=dev)
+            ws = torch.empty(sbw.sbw_sample_workspace_bytes(B, V), dtype=torch.uint8, device=dev)
+            fn = lambda i: sbw.sbw_bias_sample(x, ctx, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, ws)  # noqa: E731
+    for i in range(3 + launches):
+        fn(i)
+    torch.cuda.synchronize()
+    print(json.dumps({"profile_case": name, "launches": 3 + launches}))
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -429,7 +470,13 @@ def main() -> None:
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches only")
     ap.add_argument("--no-extra", action="store_true", help="skip the secondary workloads and the CPU baseline")
+    ap.add_argument("--profile-case", choices=PROFILE_CASES, default=None,
+                    help="run a few launches of one kernel on a small (> L2) input, for a profiler")
+    ap.add_argument("--profile-launches", type=int, default=3)
     args = ap.parse_args()
+    if args.profile_case:
+        run_profile_case(args.profile_case, args.profile_launches)
+        return
     if args.impl == "reference":
         if args.steps == 2048:
             args.steps, args.warmup = 32, 3
