@@ -1,0 +1,71 @@
+"""The N > 1 host logic of bench.py on CPU: two gloo ranks shard a batch with no collective on
+the data path, each scores its own sequences with the oracle, and the timing reduction takes the
+maximum over ranks."""
+import os
+import socket
+import sys
+from pathlib import Path
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = Path(__file__).resolve().parent.parent
+sys.path.insert(0, str(ROOT))
+
+
+def _free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank: int, world: int, port: int, out_dir: str):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank),
+                      WORLD_SIZE=str(world), LOCAL_RANK=str(rank))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    import oracle
+    from paper_2609_03844_b200 import inputs
+
+    assert bench.dist_env() == (rank, rank, world)
+    # max over ranks of a per-rank time
+    assert bench.max_over_ranks(10.0 + rank, world) == 10.0 + world - 1
+    # shard 11 sequences over the ranks: every rank scores its own rows, no exchange needed
+    tokens, lengths = inputs.null_token_streams(11, 5, 40, 32000, seed=3)
+    lo, hi = bench.shard_rows(11, rank, world)
+    off = np.concatenate([[0], np.cumsum(lengths.numpy())])
+    c, T, z = oracle.detect(tokens.numpy()[off[lo]:off[hi]], lengths.numpy()[lo:hi], 0x5EED, 0.25, 0)
+    np.savez(os.path.join(out_dir, f"rank{rank}.npz"), lo=lo, hi=hi, c=c, z=z)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_shard_rows_and_reduce_time(tmp_path):
+    world = 2
+    mp.spawn(_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    import oracle
+    from paper_2609_03844_b200 import inputs
+
+    tokens, lengths = inputs.null_token_streams(11, 5, 40, 32000, seed=3)
+    c_all, _, z_all = oracle.detect(tokens.numpy(), lengths.numpy(), 0x5EED, 0.25, 0)
+    covered = []
+    for r in range(world):
+        d = np.load(tmp_path / f"rank{r}.npz")
+        lo, hi = int(d["lo"]), int(d["hi"])
+        covered += list(range(lo, hi))
+        assert np.array_equal(d["c"], c_all[lo:hi]) and np.array_equal(d["z"], z_all[lo:hi])
+    assert covered == list(range(11))          # a partition: every row exactly once
+
+
+def test_shard_rows_is_a_balanced_partition():
+    import bench
+
+    for total in (0, 1, 7, 64, 100000):
+        for world in (1, 2, 3, 8):
+            parts = [bench.shard_rows(total, r, world) for r in range(world)]
+            assert parts[0][0] == 0 and parts[-1][1] == total
+            assert all(parts[i][1] == parts[i + 1][0] for i in range(world - 1))
+            sizes = [hi - lo for lo, hi in parts]
+            assert max(sizes) - min(sizes) <= 1
