@@ -47,6 +47,7 @@ extern "C" {
 #define SBW_ERR_UNSUPPORTED (-2) /* a value the ABI reserves but this build does not implement */
 #define SBW_ERR_WORKSPACE (-3)   /* workspace missing, misaligned or too small */
 #define SBW_ERR_CUDA (-4)        /* a CUDA runtime call failed; see sbw_last_cuda_error() */
+#define SBW_ERR_TOO_LARGE (-5)   /* the problem exceeds a fixed built-in capacity (see the call) */
 
 #define SBW_SCHEME_CONTEXT 0  /* seed from the preceding tokens only (SBW-1, SBW-4) */
 #define SBW_SCHEME_SELFSALT 1 /* seed from the preceding tokens and the candidate (SBW-ss-V) */
@@ -136,6 +137,35 @@ int sbw_bias_sample(const void *logits, int dtype, int64_t B, int64_t V, int64_t
                     uint64_t rng_step, int32_t *out_tokens, float *out_max, float *out_sumexp,
                     float *out_prob, float *out_probs, void *workspace, size_t workspace_bytes,
                     void *stream);
+
+/*
+ * sbw_bias_sample_noalloc -- sbw_bias_sample for callers that cannot hand over a workspace.
+ * The paper has no counterpart for this call; it exists for deployment.  Some users of this
+ * library cannot allocate device memory at all: a logits processor plugged into a serving
+ * engine that gave every free byte of the GPU to its KV-cache pool at start-up, or a component
+ * that runs inside another process under a fixed memory budget.  For them cudaMalloc either
+ * fails or stalls the whole device, so this variant needs none: the scratch that
+ * sbw_bias_sample takes as `workspace` lives in a fixed array inside the library instead
+ * (256 KiB of device memory, held by every GPU that loads the library until the process exits).
+ *
+ * Arguments and results are exactly those of sbw_bias_sample without `workspace` and
+ * `workspace_bytes`; inputs and outputs are still the caller's.  Differences:
+ *   - B may be at most SBW_NOALLOC_MAX_ROWS; a larger batch returns SBW_ERR_TOO_LARGE and
+ *     enqueues nothing (split it, or use sbw_bias_sample).
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current) before launching; make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  The library clears what has to start at zero
+ *     on every call, but two calls that overlap on the GPU (different streams, no ordering
+ *     between them) race on it and give undefined results: order them.
+ * The call itself allocates nothing: no cudaMalloc, no cudaFree, no allocating library routine.
+ */
+#define SBW_NOALLOC_MAX_ROWS 4096
+int sbw_bias_sample_noalloc(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
+                            int64_t vocab_offset, const int32_t *ctx_tokens, int ctx_width,
+                            uint64_t key, double gamma, float delta, int scheme, float temperature,
+                            uint64_t rng_seed, uint64_t rng_step, int32_t *out_tokens,
+                            float *out_max, float *out_sumexp, float *out_prob, float *out_probs,
+                            void *stream);
 
 /*
  * sbw_detect -- batch detection (Section 2.2 "Detection": one membership test per token, no

@@ -18,6 +18,8 @@ SBW_ERR_INVALID_ARG = -1
 SBW_ERR_UNSUPPORTED = -2
 SBW_ERR_WORKSPACE = -3
 SBW_ERR_CUDA = -4
+SBW_ERR_TOO_LARGE = -5
+NOALLOC_MAX_ROWS = 4096
 SCHEME_CONTEXT = 0
 SCHEME_SELFSALT = 1
 DTYPE_F32 = 0
@@ -26,7 +28,7 @@ DTYPE_BF16 = 1
 EXPORTS = ("sbw_version", "sbw_last_cuda_error", "sbw_bias_logits",
            "sbw_bias_logits_host_staging_bytes", "sbw_bias_logits_host",
            "sbw_sample_workspace_bytes", "sbw_bias_sample", "sbw_detect_workspace_bytes",
-           "sbw_detect", "sbw_int_probe")
+           "sbw_detect", "sbw_int_probe", "sbw_bias_sample_noalloc")
 
 _lib = None
 
@@ -34,7 +36,7 @@ _lib = None
 class SbwError(RuntimeError):
     def __init__(self, call: str, code: int, cuda_error: int = 0):
         names = {-1: "SBW_ERR_INVALID_ARG", -2: "SBW_ERR_UNSUPPORTED", -3: "SBW_ERR_WORKSPACE",
-                 -4: "SBW_ERR_CUDA"}
+                 -4: "SBW_ERR_CUDA", -5: "SBW_ERR_TOO_LARGE"}
         msg = f"{call} returned {names.get(code, code)}"
         if code == SBW_ERR_CUDA:
             msg += f" (cudaError_t {cuda_error})"
@@ -74,6 +76,10 @@ def lib() -> ctypes.CDLL:
         L.sbw_bias_sample.argtypes = [vp, i32, i64, i64, i64, i64, vp, i32, u64, c.c_double,
                                       c.c_float, i32, c.c_float, u64, u64, vp, vp, vp, vp, vp, vp,
                                       sz, vp]
+        L.sbw_bias_sample_noalloc.restype = i32
+        L.sbw_bias_sample_noalloc.argtypes = [vp, i32, i64, i64, i64, i64, vp, i32, u64, c.c_double,
+                                              c.c_float, i32, c.c_float, u64, u64, vp, vp, vp, vp, vp,
+                                              vp]
         L.sbw_detect_workspace_bytes.restype = sz
         L.sbw_detect_workspace_bytes.argtypes = [i64]
         L.sbw_detect.restype = i32
@@ -191,6 +197,30 @@ def sbw_bias_sample(logits: torch.Tensor, ctx_tokens: torch.Tensor, key: int, ga
                                _ptr(out_sumexp), _ptr(out_prob), _ptr(out_probs), _ptr(workspace),
                                workspace.numel() * workspace.element_size(), _stream(stream))
     _check("sbw_bias_sample", rc)
+    return out_tokens
+
+
+def sbw_bias_sample_noalloc(logits: torch.Tensor, ctx_tokens: torch.Tensor, key: int, gamma: float,
+                            delta: float, scheme: int, temperature: float, rng_seed: int,
+                            rng_step: int, out_tokens: torch.Tensor, *,
+                            out_max: torch.Tensor | None = None,
+                            out_sumexp: torch.Tensor | None = None,
+                            out_prob: torch.Tensor | None = None,
+                            out_probs: torch.Tensor | None = None, V: int | None = None,
+                            vocab_offset: int = 0, stream=None) -> torch.Tensor:
+    """sbw_bias_sample for callers that cannot allocate device memory (for instance a logits
+    processor inside a serving engine whose cache pool already owns the GPU): no workspace
+    argument, the scratch is a fixed 256 KiB array inside the library.  At most
+    ``NOALLOC_MAX_ROWS`` rows per call; calls on one device share the scratch and must not
+    overlap on the GPU; make the first call on a device outside stream capture."""
+    B, V, ld = _row_layout(logits, V)
+    W = _ctx(ctx_tokens, B)
+    rc = lib().sbw_bias_sample_noalloc(_ptr(logits), _dtype_code(logits), B, V, ld, vocab_offset,
+                                       _ptr(ctx_tokens), W, key, gamma, delta, scheme, temperature,
+                                       rng_seed, rng_step, _ptr(out_tokens), _ptr(out_max),
+                                       _ptr(out_sumexp), _ptr(out_prob), _ptr(out_probs),
+                                       _stream(stream))
+    _check("sbw_bias_sample_noalloc", rc)
     return out_tokens
 
 

@@ -21,6 +21,7 @@
 
 #include <cfloat>
 #include <climits>
+#include <mutex>
 
 #include "sbw_common.cuh"
 #include "sbw_hash.cuh"
@@ -494,4 +495,64 @@ extern "C" int sbw_bias_sample(const void *logits, int dtype, int64_t B, int64_t
     }
     return scheme == SBW_SCHEME_CONTEXT ? launch<SBW_DTYPE_BF16, SBW_SCHEME_CONTEXT>(a, vector, out_probs, s)
                                         : launch<SBW_DTYPE_BF16, SBW_SCHEME_SELFSALT>(a, vector, out_probs, s);
+}
+
+// ---------------------------------------------------------------------------------------------
+// sbw_bias_sample_noalloc: the same call for users that cannot allocate device memory (a plugin
+// inside a serving engine whose KV-cache pool owns the whole GPU, a component under a fixed
+// memory budget).  The scratch is a fixed array that is part of the library image.
+// ---------------------------------------------------------------------------------------------
+namespace sbw {
+namespace {
+
+constexpr size_t kNoallocScratchBytes = 256 * 1024;   // covers SBW_NOALLOC_MAX_ROWS rows
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoallocScratchBytes];
+
+// In host code `g_noalloc_scratch` is only a handle for the runtime, not a device address: the
+// address the kernels need comes from cudaGetSymbolAddress, asked once per device with that
+// device current, and is cached here.
+int noalloc_scratch_address(void **out) {
+    constexpr int kMaxDevices = 64;
+    static void *cached[kMaxDevices] = {nullptr};
+    static std::mutex mu;
+    int dev = 0;
+    SBW_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return SBW_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cached[dev]) {
+        void *p = nullptr;
+        SBW_CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+        cached[dev] = p;
+    }
+    *out = cached[dev];
+    return SBW_OK;
+}
+
+}  // namespace
+}  // namespace sbw
+
+extern "C" int sbw_bias_sample_noalloc(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
+                                       int64_t vocab_offset, const int32_t *ctx_tokens, int ctx_width,
+                                       uint64_t key, double gamma, float delta, int scheme,
+                                       float temperature, uint64_t rng_seed, uint64_t rng_step,
+                                       int32_t *out_tokens, float *out_max, float *out_sumexp,
+                                       float *out_prob, float *out_probs, void *stream) {
+    using namespace sbw;
+    if (B > SBW_NOALLOC_MAX_ROWS) return SBW_ERR_TOO_LARGE;
+    static_assert(sizeof(double2) * SBW_NOALLOC_MAX_ROWS + sizeof(unsigned) * SBW_NOALLOC_MAX_ROWS +
+                          sizeof(Partial) * (SBW_NOALLOC_MAX_ROWS + kTargetCtas) + 3 * 256 <=
+                      kNoallocScratchBytes,
+                  "the built-in scratch must hold the workspace of SBW_NOALLOC_MAX_ROWS rows");
+    if (B > 0 && V > 0 && sbw_sample_workspace_bytes(B, V) > kNoallocScratchBytes) return SBW_ERR_TOO_LARGE;
+    void *scratch = nullptr;
+    if (B > 0) {
+        const int rc = noalloc_scratch_address(&scratch);
+        if (rc != SBW_OK) return rc;
+    }
+    // The shared array keeps whatever the previous call left in it.  The only part that must
+    // start at zero is the per-row ticket counters, and sbw_bias_sample clears those on the
+    // stream before every launch that uses them; everything else is written before it is read.
+    return sbw_bias_sample(logits, dtype, B, V, ld, vocab_offset, ctx_tokens, ctx_width, key, gamma, delta,
+                           scheme, temperature, rng_seed, rng_step, out_tokens, out_max, out_sumexp,
+                           out_prob, out_probs, scratch, kNoallocScratchBytes, stream);
 }
