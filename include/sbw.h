@@ -71,7 +71,8 @@ int sbw_last_cuda_error(void);
  *                row are biased, columns V..ld-1 are neither read nor written.  Any alignment is
  *                accepted; rows that start on 16-byte boundaries take the vectorised path.
  *   B, V, ld     rows, vocabulary columns, row stride in elements (ld >= V > 0, B >= 0).
- *   vocab_offset global id of column 0 (>= 0; non-zero when the vocabulary is sharded).
+ *   vocab_offset global id of column 0 (>= 0; non-zero when the vocabulary is sharded);
+ *                vocab_offset + V may not exceed 2^32 (ids are 32-bit), else SBW_ERR_UNSUPPORTED.
  *   ctx_tokens   device, [B, ctx_width] int32: the ctx_width tokens preceding the one being
  *                generated, per row.  1 <= ctx_width <= SBW_MAX_CTX_WIDTH.
  *   key          64-bit secret key.      gamma  green fraction, 0 < gamma < 1.

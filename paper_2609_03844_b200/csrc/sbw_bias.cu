@@ -5,11 +5,15 @@
 // the SM count), so every SM receives the same number of slots whatever B and V are.  A block
 // walks its share row by row: per row it derives the seed material once (context scheme: the ten
 // Philox round keys; self-salt scheme: the smallest context hash), then its threads stride over
-// the row's slots.  Per slot a thread issues one 128-bit load, evaluates the 4 or 8 independent
-// hash chains in registers (that independence is the instruction-level parallelism that keeps
-// the integer pipes busy), applies the bias, and issues one 128-bit store.  No shared memory, no
-// mask tensor, no other global traffic.  Rows that do not start on 16-byte boundaries, and the
-// ragged last slot of a row, go through the same code one element at a time.
+// the row's slots.  Per trip a thread issues 128-bit loads for 8 logits, evaluates the 8 hash
+// chains round by round in registers (the interleaving is what keeps the multiply pipe busy: the
+// kernel is bound by the 32x32->64 multiplier, not by HBM), applies the bias, and stores 128 bits
+// back.  No shared memory, no mask tensor, no other global traffic.  Rows that do not start on
+// 16-byte boundaries, and the ragged last slot of a row, go through a scalar routine.
+//
+// The kernel is launched with programmatic stream serialisation: it lets the next kernel of the
+// stream begin its launch while this one drains, and itself waits for everything before it in the
+// stream before it touches memory, so stream order is preserved.
 #include <cuda_bf16.h>
 
 #include "sbw_common.cuh"
@@ -60,39 +64,88 @@ struct RowSeed<SBW_SCHEME_SELFSALT> {
     }
 };
 
-// One logit, any alignment: used for ragged tails and for rows that are not 16-byte aligned.
+// Columns [c_begin, c_end) of one row, one logit at a time, any alignment: ragged tails and rows
+// that are not 16-byte aligned.  Kept out of line so that it does not weigh on the fast path.
 template <int DTYPE, int SCHEME>
-__device__ __forceinline__ void bias_one(const BiasArgs &a, const RowSeed<SCHEME> &rs, void *row_ptr,
-                                         uint32_t col) {
-    const uint32_t v = a.vocab_offset + col;
-    const bool green = rs.word0(v, a.key) <= a.thr_m1;
-    if (!green) return;
-    if constexpr (DTYPE == SBW_DTYPE_F32) {
-        float *p = static_cast<float *>(row_ptr) + col;
-        *p = __fadd_rn(*p, a.delta);
-    } else {
-        __nv_bfloat16 *p = static_cast<__nv_bfloat16 *>(row_ptr) + col;
-        // both operands are bf16 values, so rounding their fp32 sum once more gives the
-        // correctly rounded bf16 sum
-        *p = __float2bfloat16_rn(__fadd_rn(__bfloat162float(*p), a.delta));
+__device__ __noinline__ void bias_scalar(const BiasArgs &a, const RowSeed<SCHEME> &rs, void *row_ptr,
+                                         uint32_t c_begin, uint32_t c_end, uint32_t c_step) {
+    for (uint32_t col = c_begin; col < c_end; col += c_step) {
+        const uint32_t v = a.vocab_offset + col;
+        if (rs.word0(v, a.key) > a.thr_m1) continue;
+        if constexpr (DTYPE == SBW_DTYPE_F32) {
+            float *p = static_cast<float *>(row_ptr) + col;
+            *p = __fadd_rn(*p, a.delta);
+        } else {
+            __nv_bfloat16 *p = static_cast<__nv_bfloat16 *>(row_ptr) + col;
+            // both operands are bf16 values, so rounding their fp32 sum once more gives the
+            // correctly rounded bf16 sum
+            *p = __float2bfloat16_rn(__fadd_rn(__bfloat162float(*p), a.delta));
+        }
     }
 }
 
+// Green flags of the 8 consecutive ids vg .. vg+7.
+template <int SCHEME>
+__device__ __forceinline__ void green8(const BiasArgs &a, const RowSeed<SCHEME> &rs, uint32_t vg,
+                                       bool (&g)[8]) {
+    uint32_t x[8];
+    if constexpr (SCHEME == SBW_SCHEME_CONTEXT) {
+        philox_word0_n<8>(vg, rs.rk, x);
+    } else {
+        uint32_t v[8];
+        uint64_t r[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            v[i] = vg + i;
+            r[i] = seed_selfsalt(a.key, rs.jmin, v[i]);
+        }
+        philox_word0_n<8>(v, r, x);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) g[i] = x[i] <= a.thr_m1;
+}
+template <int SCHEME>
+__device__ __forceinline__ void green4x2(const BiasArgs &a, const RowSeed<SCHEME> &rs, uint32_t vg0,
+                                         uint32_t vg1, bool (&g)[8]) {
+    uint32_t x[8];
+    if constexpr (SCHEME == SBW_SCHEME_CONTEXT) {
+        uint32_t xa[4], xb[4];
+        philox_word0_n<4>(vg0, rs.rk, xa);
+        philox_word0_n<4>(vg1, rs.rk, xb);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { x[i] = xa[i]; x[4 + i] = xb[i]; }
+    } else {
+        uint32_t v[8];
+        uint64_t r[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            v[i] = (i < 4 ? vg0 : vg1) + (i & 3);
+            r[i] = seed_selfsalt(a.key, rs.jmin, v[i]);
+        }
+        philox_word0_n<8>(v, r, x);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) g[i] = x[i] <= a.thr_m1;
+}
+
 template <int DTYPE, int SCHEME, bool VECTOR>
-__global__ void __launch_bounds__(kBiasThreads)
+__global__ void __launch_bounds__(kBiasThreads, 2)
 bias_kernel(const BiasArgs a) {
     constexpr int VEC = VECTOR ? (DTYPE == SBW_DTYPE_F32 ? 4 : 8) : 1;
     constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
+    // let the next kernel in the stream start launching; wait for the previous ones to finish
+    asm volatile("griddepcontrol.launch_dependents;");
     const int64_t s_begin = a.total / gridDim.x * blockIdx.x +
                             (a.total % gridDim.x) * blockIdx.x / gridDim.x;
     const int64_t s_end = a.total / gridDim.x * (blockIdx.x + 1) +
                           (a.total % gridDim.x) * (blockIdx.x + 1) / gridDim.x;
-    if (s_begin >= s_end) return;
     int64_t row = s_begin / a.nslot;
     uint32_t col = static_cast<uint32_t>(s_begin - row * a.nslot);
     int64_t left = s_end - s_begin;
     const uint32_t nslot = static_cast<uint32_t>(a.nslot);
     const uint32_t V = static_cast<uint32_t>(a.V);
+    const uint32_t nfull = V / VEC;       // slots of the row that are complete vectors
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     while (left > 0) {
         const uint32_t seg = static_cast<uint32_t>(min(static_cast<int64_t>(nslot - col), left));
@@ -100,41 +153,52 @@ bias_kernel(const BiasArgs a) {
         rs.init(a.key, a.ctx + row * a.W, a.W);
         char *row_ptr = static_cast<char *>(a.logits) + row * a.ld * ESIZE;
         const uint32_t j_end = col + seg;
-        for (uint32_t j = col + threadIdx.x; j < j_end; j += kBiasThreads) {
-            const uint32_t cb = j * VEC;
-            if constexpr (!VECTOR) {
-                bias_one<DTYPE, SCHEME>(a, rs, row_ptr, cb);
-            } else {
-                if (cb + VEC > V) {  // ragged last slot of the row
-                    for (uint32_t c = cb; c < V; ++c) bias_one<DTYPE, SCHEME>(a, rs, row_ptr, c);
-                    continue;
-                }
-                uint4 *p = reinterpret_cast<uint4 *>(row_ptr) + j;
-                uint4 w = *p;
-                const uint32_t vg = a.vocab_offset + cb;
-                bool g[VEC];
-#pragma unroll
-                for (int i = 0; i < VEC; ++i) g[i] = rs.word0(vg + i, a.key) <= a.thr_m1;
-                if constexpr (DTYPE == SBW_DTYPE_F32) {
-                    uint32_t *e = reinterpret_cast<uint32_t *>(&w);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float s = __fadd_rn(__uint_as_float(e[i]), a.delta);
-                        e[i] = g[i] ? __float_as_uint(s) : e[i];
-                    }
-                } else {
+        if constexpr (!VECTOR) {
+            bias_scalar<DTYPE, SCHEME>(a, rs, row_ptr, col + threadIdx.x, j_end, kBiasThreads);
+        } else {
+            const uint32_t jf_end = min(j_end, nfull);
+            uint4 *slots = reinterpret_cast<uint4 *>(row_ptr);
+            if constexpr (DTYPE == SBW_DTYPE_BF16) {
+                const uint32_t dlo = a.delta_bf16, dhi = a.delta_bf16 << 16;
+                for (uint32_t j = col + threadIdx.x; j < jf_end; j += kBiasThreads) {
+                    uint4 w = slots[j];
+                    bool g[8];
+                    green8<SCHEME>(a, rs, a.vocab_offset + j * 8, g);
                     // adding -0.0 returns the other operand unchanged, so a packed add with
                     // {delta or -0.0} per half biases exactly the green halves
                     uint32_t *e = reinterpret_cast<uint32_t *>(&w);
-                    const uint32_t dlo = a.delta_bf16, dhi = a.delta_bf16 << 16;
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const uint32_t d = (g[2 * i] ? dlo : 0x8000u) | (g[2 * i + 1] ? dhi : 0x80000000u);
                         e[i] = add_bf16x2(e[i], d);
                     }
+                    slots[j] = w;
                 }
-                *p = w;
+            } else {
+                // two slots (8 logits) per trip; the second one may fall off the end of the segment
+                for (uint32_t j = col + threadIdx.x; j < jf_end; j += 2 * kBiasThreads) {
+                    const uint32_t j2 = j + kBiasThreads;
+                    const bool two = j2 < jf_end;
+                    uint4 w0 = slots[j];
+                    uint4 w1 = two ? slots[j2] : make_uint4(0, 0, 0, 0);
+                    bool g[8];
+                    green4x2<SCHEME>(a, rs, a.vocab_offset + j * 4, a.vocab_offset + j2 * 4, g);
+                    uint32_t *e0 = reinterpret_cast<uint32_t *>(&w0);
+                    uint32_t *e1 = reinterpret_cast<uint32_t *>(&w1);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float s0 = __fadd_rn(__uint_as_float(e0[i]), a.delta);
+                        const float s1 = __fadd_rn(__uint_as_float(e1[i]), a.delta);
+                        e0[i] = g[i] ? __float_as_uint(s0) : e0[i];
+                        e1[i] = g[4 + i] ? __float_as_uint(s1) : e1[i];
+                    }
+                    slots[j] = w0;
+                    if (two) slots[j2] = w1;
+                }
             }
+            // ragged last slot of the row, if this block owns it
+            if (nfull < nslot && j_end == nslot && threadIdx.x == 0)
+                bias_scalar<DTYPE, SCHEME>(a, rs, row_ptr, nfull * VEC, V, 1);
         }
         left -= seg;
         ++row;
@@ -157,8 +221,7 @@ int launch(const BiasArgs &a, cudaStream_t stream) {
     const int64_t want = (a.total + kBiasThreads - 1) / kBiasThreads;
     const int64_t cap = static_cast<int64_t>(di.sm_count) * blocks_per_sm;
     const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
-    bias_kernel<DTYPE, SCHEME, VECTOR><<<grid, kBiasThreads, 0, stream>>>(a);
-    SBW_CUDA_TRY(cudaGetLastError());
+    SBW_CUDA_TRY(launch_pdl(bias_kernel<DTYPE, SCHEME, VECTOR>, dim3(grid), dim3(kBiasThreads), stream, a));
     return SBW_OK;
 }
 
@@ -175,6 +238,7 @@ int bias_logits_impl(void *logits, int dtype, int64_t B, int64_t V, int64_t ld, 
     if (!valid_common(dtype, ctx_width, gamma, scheme)) return SBW_ERR_INVALID_ARG;
     if (B < 0 || V <= 0 || ld < V || vocab_offset < 0) return SBW_ERR_INVALID_ARG;
     if (V > 0x7fffffffLL || B > (int64_t(1) << 40)) return SBW_ERR_UNSUPPORTED;
+    if (vocab_offset + V > (int64_t(1) << 32)) return SBW_ERR_UNSUPPORTED;   // ids are 32-bit
     if (!(delta == delta) || delta - delta != 0.0f) return SBW_ERR_INVALID_ARG;  // NaN or inf
     if (B == 0) return SBW_OK;
     if (!logits || !ctx_tokens) return SBW_ERR_INVALID_ARG;

@@ -138,6 +138,98 @@ __device__ __forceinline__ uint32_t philox_word0(uint32_t v, uint64_t r) {
     return __umulhi(kPhiloxM1, n2) ^ n1 ^ (k0 + 9u * kPhiloxW0);
 }
 
+// The same two evaluations for N candidates at once, written round by round so that the N
+// dependent multiply/xor chains are interleaved in program order: one warp then keeps the
+// multiply pipe busy by itself, whatever the occupancy.
+//
+// Context scheme, N consecutive ids vbase .. vbase+N-1 (which must not wrap past 2^32): the
+// round-0 product M0*(vbase+i) is formed as M0*vbase + M0*i with a 64-bit add, which moves N-1
+// multiplies off the multiply pipe.
+template <int N>
+__device__ __forceinline__ void philox_word0_n(uint32_t vbase, const RowKeys &rk, uint32_t (&out)[N]) {
+    uint32_t c0[N], c1[N], c2[N], c3[N];
+    const uint64_t p0 = static_cast<uint64_t>(kPhiloxM0) * vbase;
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        const uint64_t p = p0 + static_cast<uint64_t>(kPhiloxM0) * static_cast<uint32_t>(i);
+        c2[i] = static_cast<uint32_t>(p >> 32) ^ rk.k1[0];
+        c3[i] = static_cast<uint32_t>(p);
+    }
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        uint32_t h1, l1;
+        mulhilo(kPhiloxM1, c2[i], h1, l1);
+        c0[i] = h1 ^ rk.k0[1];
+        c1[i] = l1;
+        c2[i] = c3[i] ^ rk.r1_c2;
+    }
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        uint32_t h0, l0, h1, l1;
+        mulhilo(kPhiloxM0, c0[i], h0, l0);
+        mulhilo(kPhiloxM1, c2[i], h1, l1);
+        c0[i] = h1 ^ c1[i] ^ rk.k0[2];
+        c1[i] = l1;
+        c2[i] = h0 ^ rk.r2_c3k;
+        c3[i] = l0;
+    }
+#pragma unroll
+    for (int r = 3; r < 8; ++r) {
+#pragma unroll
+        for (int i = 0; i < N; ++i) philox_round(c0[i], c1[i], c2[i], c3[i], rk.k0[r], rk.k1[r]);
+    }
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        const uint32_t n1 = kPhiloxM1 * c2[i];
+        const uint32_t n2 = __umulhi(kPhiloxM0, c0[i]) ^ c3[i] ^ rk.k1[8];
+        out[i] = __umulhi(kPhiloxM1, n2) ^ n1 ^ rk.k0[9];
+    }
+}
+
+// Per-candidate seeds r[i] (self-salt scheme, detection), arbitrary ids v[i].
+template <int N>
+__device__ __forceinline__ void philox_word0_n(const uint32_t (&v)[N], const uint64_t (&r)[N],
+                                               uint32_t (&out)[N]) {
+    uint32_t c0[N], c1[N], c2[N], c3[N], k0[N], k1[N];
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        k0[i] = static_cast<uint32_t>(r[i]);
+        k1[i] = static_cast<uint32_t>(r[i] >> 32);
+        uint32_t h, l, h0, l0;
+        mulhilo(kPhiloxM0, v[i], h, l);
+        mulhilo(kPhiloxM0, k0[i], h0, l0);
+        c2[i] = h ^ k1[i];           // after round 0
+        c1[i] = l;                   // parked: lo(M0 v), consumed by round 1
+        c0[i] = h0;                  // parked: hi(M0 k0)
+        c3[i] = l0;                  // c3 after round 1
+    }
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        k0[i] += kPhiloxW0;
+        k1[i] += kPhiloxW1;
+        uint32_t h1, l1;
+        mulhilo(kPhiloxM1, c2[i], h1, l1);
+        c2[i] = c0[i] ^ c1[i] ^ k1[i];
+        c0[i] = h1 ^ k0[i];
+        c1[i] = l1;
+    }
+#pragma unroll
+    for (int rd = 2; rd < 8; ++rd) {
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+            k0[i] += kPhiloxW0;
+            k1[i] += kPhiloxW1;
+            philox_round(c0[i], c1[i], c2[i], c3[i], k0[i], k1[i]);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        const uint32_t n1 = kPhiloxM1 * c2[i];
+        const uint32_t n2 = __umulhi(kPhiloxM0, c0[i]) ^ c3[i] ^ (k1[i] + kPhiloxW1);
+        out[i] = __umulhi(kPhiloxM1, n2) ^ n1 ^ (k0[i] + 2u * kPhiloxW0);
+    }
+}
+
 // Table 12 "additive" PRF: key times the sum of the context ids.
 __device__ __forceinline__ uint64_t seed_context(uint64_t key, const int32_t *ctx, int W) {
     uint64_t sigma = 0;

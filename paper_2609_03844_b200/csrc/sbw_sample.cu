@@ -442,7 +442,7 @@ extern "C" int sbw_bias_sample(const void *logits, int dtype, int64_t B, int64_t
     if (B < 0 || V <= 0 || ld < V || vocab_offset < 0) return SBW_ERR_INVALID_ARG;
     if (!(temperature > 0.0f) || temperature - temperature != 0.0f) return SBW_ERR_INVALID_ARG;
     if (!(delta == delta) || delta - delta != 0.0f) return SBW_ERR_INVALID_ARG;
-    if (V > 0x7fffffffLL) return SBW_ERR_UNSUPPORTED;
+    if (V > 0x7fffffffLL || vocab_offset + V > (int64_t(1) << 32)) return SBW_ERR_UNSUPPORTED;
     if (B == 0) return SBW_OK;
     if (!logits || !ctx_tokens || !out_tokens) return SBW_ERR_INVALID_ARG;
     const double c2 = 1.4426950408889634 / static_cast<double>(temperature);
