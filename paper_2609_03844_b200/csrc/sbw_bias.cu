@@ -36,6 +36,7 @@ struct BiasArgs {
     uint32_t thr_m1;        // green <=> x <= thr_m1
     float delta;            // fp32 path: delta; bf16 path: delta rounded to bf16, widened
     uint32_t delta_bf16;    // bf16 bits of delta
+    Weyl weyl;              // Philox key-schedule increments (see sbw_hash.cuh)
 };
 
 __device__ __forceinline__ uint32_t add_bf16x2(uint32_t a, uint32_t b) {
@@ -53,14 +54,16 @@ struct RowSeed<SBW_SCHEME_CONTEXT> {
     __device__ __forceinline__ void init(uint64_t key, const int32_t *ctx, int W) {
         rk = make_row_keys(seed_context(key, ctx, W));
     }
-    __device__ __forceinline__ uint32_t word0(uint32_t v, uint64_t) const { return philox_word0(v, rk); }
+    __device__ __forceinline__ uint32_t word0(uint32_t v, uint64_t, const Weyl) const {
+        return philox_word0(v, rk);
+    }
 };
 template <>
 struct RowSeed<SBW_SCHEME_SELFSALT> {
     uint32_t jmin;
     __device__ __forceinline__ void init(uint64_t, const int32_t *ctx, int W) { jmin = jenkins_min(ctx, W); }
-    __device__ __forceinline__ uint32_t word0(uint32_t v, uint64_t key) const {
-        return philox_word0(v, seed_selfsalt(key, jmin, v));
+    __device__ __forceinline__ uint32_t word0(uint32_t v, uint64_t key, const Weyl w) const {
+        return philox_word0(v, seed_selfsalt(key, jmin, v), w);
     }
 };
 
@@ -71,7 +74,7 @@ __device__ __noinline__ void bias_scalar(const BiasArgs &a, const RowSeed<SCHEME
                                          uint32_t c_begin, uint32_t c_end, uint32_t c_step) {
     for (uint32_t col = c_begin; col < c_end; col += c_step) {
         const uint32_t v = a.vocab_offset + col;
-        if (rs.word0(v, a.key) > a.thr_m1) continue;
+        if (rs.word0(v, a.key, a.weyl) > a.thr_m1) continue;
         if constexpr (DTYPE == SBW_DTYPE_F32) {
             float *p = static_cast<float *>(row_ptr) + col;
             *p = __fadd_rn(*p, a.delta);
@@ -99,7 +102,7 @@ __device__ __forceinline__ void green8(const BiasArgs &a, const RowSeed<SCHEME> 
             v[i] = vg + i;
             r[i] = seed_selfsalt(a.key, rs.jmin, v[i]);
         }
-        philox_word0_n<8>(v, r, x);
+        philox_word0_n<8>(v, r, x, a.weyl);
     }
 #pragma unroll
     for (int i = 0; i < 8; ++i) g[i] = x[i] <= a.thr_m1;
@@ -122,7 +125,7 @@ __device__ __forceinline__ void green4x2(const BiasArgs &a, const RowSeed<SCHEME
             v[i] = (i < 4 ? vg0 : vg1) + (i & 3);
             r[i] = seed_selfsalt(a.key, rs.jmin, v[i]);
         }
-        philox_word0_n<8>(v, r, x);
+        philox_word0_n<8>(v, r, x, a.weyl);
     }
 #pragma unroll
     for (int i = 0; i < 8; ++i) g[i] = x[i] <= a.thr_m1;
@@ -253,6 +256,7 @@ int bias_logits_impl(void *logits, int dtype, int64_t B, int64_t V, int64_t ld, 
     a.thr_m1 = threshold_minus_one(gamma);
     a.delta = delta;
     a.delta_bf16 = 0;
+    a.weyl = make_weyl();
     const int esize = dtype == SBW_DTYPE_F32 ? 4 : 2;
     if (dtype == SBW_DTYPE_BF16) {
         const __nv_bfloat16 d = __float2bfloat16_rn(delta);

@@ -5,7 +5,8 @@
 // the W predecessors of a token come from the same cache lines), derive the token's seed, run
 // one Philox evaluation, and the warp adds popc(ballot(green)) to a warp-uniform counter, so no
 // per-lane reduction is needed at the end.  Each lane carries kDetectIlp independent tokens per
-// trip so that the dependent multiply/xor chain of one hash overlaps with the others.
+// trip, hashed round by round so that the dependent multiply/xor chains overlap; full trips run
+// without masks and only the last, ragged trip of a sequence is predicated.
 // Sequence starts come from a caller-supplied offsets array or from a two-kernel exclusive scan
 // of the lengths into the workspace.
 #include "sbw_common.cuh"
@@ -14,8 +15,17 @@
 namespace sbw {
 namespace {
 
-constexpr int kDetectThreads = 128;  // 4 sequences per block: short blocks keep the tail small
-constexpr int kDetectIlp = 2;
+#ifndef SBW_DETECT_THREADS
+#define SBW_DETECT_THREADS 128
+#endif
+#ifndef SBW_DETECT_ILP
+#define SBW_DETECT_ILP 4
+#endif
+#ifndef SBW_DETECT_MIN_BLOCKS
+#define SBW_DETECT_MIN_BLOCKS 1
+#endif
+constexpr int kDetectThreads = SBW_DETECT_THREADS;  // 4 sequences per block: short blocks keep the tail small
+constexpr int kDetectIlp = SBW_DETECT_ILP;
 constexpr int kScanThreads = 256;
 constexpr int kScanItems = 4;        // lengths per thread
 constexpr int kScanTile = kScanThreads * kScanItems;
@@ -32,6 +42,7 @@ struct DetectArgs {
     int32_t *out_counts;
     int32_t *out_T;
     double *out_z;
+    Weyl weyl;   // Philox key-schedule increments (see sbw_hash.cuh)
 };
 
 __device__ __forceinline__ int64_t clamp_len(int32_t l) { return l > 0 ? l : 0; }
@@ -104,8 +115,51 @@ scan_offsets(const int32_t *lengths, int64_t N, const int64_t *tile_sums, int64_
 }
 
 // ---- the detector ----
-template <int SCHEME>
-__global__ void __launch_bounds__(kDetectThreads)
+// Scores the kDetectIlp * 32 positions base + u*32 + lane (u = 0..kDetectIlp-1) of one sequence.
+// TAIL = false: every position is inside the sequence, no masking.  WIDTH > 0 fixes the context
+// width at compile time (loops unrolled), WIDTH = 0 reads it from the arguments.
+template <int SCHEME, int WIDTH, bool TAIL>
+__device__ __forceinline__ int score_trip(const DetectArgs &a, const int32_t *tok, int base, int len,
+                                          int lane) {
+    const int width = WIDTH > 0 ? WIDTH : a.W;
+    uint32_t v[kDetectIlp];
+    uint64_t r[kDetectIlp];
+    bool valid[kDetectIlp];
+#pragma unroll
+    for (int u = 0; u < kDetectIlp; ++u) {
+        const int t = base + u * 32 + lane;
+        valid[u] = !TAIL || t < len;
+        const int ts = valid[u] ? t : width;      // any readable position; its result is dropped
+        v[u] = static_cast<uint32_t>(tok[ts]);
+        if constexpr (SCHEME == SBW_SCHEME_CONTEXT) {
+            if constexpr (WIDTH == 1) {
+                r[u] = a.key * static_cast<uint64_t>(static_cast<uint32_t>(tok[ts - 1]));
+            } else {
+                uint64_t sigma = 0;
+#pragma unroll
+                for (int i = 1; i <= (WIDTH > 0 ? WIDTH : SBW_MAX_CTX_WIDTH); ++i)
+                    if (i <= width) sigma += static_cast<uint32_t>(tok[ts - i]);
+                r[u] = a.key * sigma;
+            }
+        } else {
+            uint32_t jmin = 0xFFFFFFFFu;
+#pragma unroll
+            for (int i = 1; i <= (WIDTH > 0 ? WIDTH : SBW_MAX_CTX_WIDTH); ++i)
+                if (i <= width) jmin = min(jmin, jenkins(static_cast<uint32_t>(tok[ts - i])));
+            r[u] = seed_selfsalt(a.key, jmin, v[u]);
+        }
+    }
+    uint32_t x[kDetectIlp];
+    philox_word0_n<kDetectIlp>(v, r, x, a.weyl);
+    int count = 0;
+#pragma unroll
+    for (int u = 0; u < kDetectIlp; ++u)
+        count += __popc(__ballot_sync(0xffffffffu, valid[u] && x[u] <= a.thr_m1));
+    return count;
+}
+
+template <int SCHEME, int WIDTH>
+__global__ void __launch_bounds__(kDetectThreads, SBW_DETECT_MIN_BLOCKS)
 detect_kernel(const DetectArgs a) {
     const int lane = threadIdx.x & 31;
     const int64_t seq = static_cast<int64_t>(blockIdx.x) * (kDetectThreads / 32) + (threadIdx.x >> 5);
@@ -114,36 +168,18 @@ detect_kernel(const DetectArgs a) {
     int64_t L = clamp_len(a.lengths[seq]);
     if (off < 0 || off >= a.total_tokens) L = 0;
     else if (off + L > a.total_tokens) L = a.total_tokens - off;
-    const int W = a.W;
+    const int width = WIDTH > 0 ? WIDTH : a.W;
     const int32_t *tok = a.tokens + off;
     const int len = static_cast<int>(L);
+    constexpr int kTrip = 32 * kDetectIlp;
 
     int count = 0;
-    for (int base = W; base < len; base += 32 * kDetectIlp) {
-        bool g[kDetectIlp];
-#pragma unroll
-        for (int u = 0; u < kDetectIlp; ++u) {
-            const int t = base + u * 32 + lane;
-            const bool valid = t < len;
-            const int ts = valid ? t : W;        // any readable position; result is discarded
-            const uint32_t v = static_cast<uint32_t>(tok[ts]);
-            uint64_t r;
-            if constexpr (SCHEME == SBW_SCHEME_CONTEXT) {
-                uint64_t sigma = 0;
-                for (int i = 1; i <= W; ++i) sigma += static_cast<uint32_t>(tok[ts - i]);
-                r = a.key * sigma;
-            } else {
-                uint32_t jmin = 0xFFFFFFFFu;
-                for (int i = 1; i <= W; ++i) jmin = min(jmin, jenkins(static_cast<uint32_t>(tok[ts - i])));
-                r = seed_selfsalt(a.key, jmin, v);
-            }
-            g[u] = valid && (philox_word0(v, r) <= a.thr_m1);
-        }
-#pragma unroll
-        for (int u = 0; u < kDetectIlp; ++u) count += __popc(__ballot_sync(0xffffffffu, g[u]));
-    }
+    int base = width;
+    for (; base + kTrip <= len; base += kTrip) count += score_trip<SCHEME, WIDTH, false>(a, tok, base, len, lane);
+    if (base < len) count += score_trip<SCHEME, WIDTH, true>(a, tok, base, len, lane);
+
     if (lane == 0) {
-        const int T = len > W ? len - W : 0;
+        const int T = len > width ? len - width : 0;
         a.out_counts[seq] = count;
         if (a.out_T) a.out_T[seq] = T;
         double z = 0.0;
@@ -155,6 +191,16 @@ detect_kernel(const DetectArgs a) {
         }
         a.out_z[seq] = z;
     }
+}
+
+template <int SCHEME>
+cudaError_t launch_detect(const DetectArgs &a, unsigned grid, cudaStream_t s) {
+    switch (a.W) {
+        case 1: detect_kernel<SCHEME, 1><<<grid, kDetectThreads, 0, s>>>(a); break;
+        case 4: detect_kernel<SCHEME, 4><<<grid, kDetectThreads, 0, s>>>(a); break;
+        default: detect_kernel<SCHEME, 0><<<grid, kDetectThreads, 0, s>>>(a); break;
+    }
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -193,6 +239,7 @@ extern "C" int sbw_detect(const int32_t *tokens, const int32_t *lengths, const i
     a.out_counts = out_counts;
     a.out_T = out_T;
     a.out_z = out_z;
+    a.weyl = make_weyl();
 
     if (!offsets) {
         const size_t need = sbw_detect_workspace_bytes(N);
@@ -209,10 +256,7 @@ extern "C" int sbw_detect(const int32_t *tokens, const int32_t *lengths, const i
         a.offsets = ws_offsets;
     }
     const unsigned grid = static_cast<unsigned>((N + kDetectThreads / 32 - 1) / (kDetectThreads / 32));
-    if (scheme == SBW_SCHEME_CONTEXT)
-        detect_kernel<SBW_SCHEME_CONTEXT><<<grid, kDetectThreads, 0, s>>>(a);
-    else
-        detect_kernel<SBW_SCHEME_SELFSALT><<<grid, kDetectThreads, 0, s>>>(a);
-    SBW_CUDA_TRY(cudaGetLastError());
+    SBW_CUDA_TRY(scheme == SBW_SCHEME_CONTEXT ? launch_detect<SBW_SCHEME_CONTEXT>(a, grid, s)
+                                              : launch_detect<SBW_SCHEME_SELFSALT>(a, grid, s));
     return SBW_OK;
 }

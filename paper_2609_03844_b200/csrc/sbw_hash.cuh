@@ -20,6 +20,14 @@ constexpr uint32_t kPhiloxM1 = 0xCD9E8D57u;
 constexpr uint32_t kPhiloxW0 = 0x9E3779B9u;
 constexpr uint32_t kPhiloxW1 = 0xBB67AE85u;
 
+// The Weyl increments of the Philox key schedule, handed to the kernels as launch arguments.
+// Adding a 32-bit literal costs two instructions on sm_100; adding a value that sits in a
+// register or in the constant bank costs one, and the per-candidate key schedule has 16 adds.
+struct Weyl {
+    uint32_t w0, w1;
+};
+inline Weyl make_weyl() { return Weyl{kPhiloxW0, kPhiloxW1}; }
+
 __device__ __forceinline__ void mulhilo(uint32_t a, uint32_t b, uint32_t &hi, uint32_t &lo) {
     const uint64_t p = static_cast<uint64_t>(a) * b;   // one IMAD.WIDE.U32
     hi = static_cast<uint32_t>(p >> 32);
@@ -57,6 +65,25 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
     for (int i = 0; i < 10; ++i)
         philox_round(c0, c1, c2, c3, k0 + static_cast<uint32_t>(i) * kPhiloxW0,
                      k1 + static_cast<uint32_t>(i) * kPhiloxW1);
+    return make_uint4(c0, c1, c2, c3);
+}
+
+// The same block under round keys prepared by the host (one key for the whole launch).
+struct BlockKeys {
+    uint32_t k0[10], k1[10];
+};
+inline BlockKeys make_block_keys(uint32_t k0, uint32_t k1) {
+    BlockKeys bk;
+    for (int i = 0; i < 10; ++i) {
+        bk.k0[i] = k0 + static_cast<uint32_t>(i) * kPhiloxW0;
+        bk.k1[i] = k1 + static_cast<uint32_t>(i) * kPhiloxW1;
+    }
+    return bk;
+}
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               const BlockKeys &bk) {
+#pragma unroll
+    for (int i = 0; i < 10; ++i) philox_round(c0, c1, c2, c3, bk.k0[i], bk.k1[i]);
     return make_uint4(c0, c1, c2, c3);
 }
 
@@ -118,24 +145,30 @@ __device__ __forceinline__ uint32_t philox_word0(uint32_t v, const RowKeys &rk) 
 
 // Word 0 of Philox4x32-10(counter (v,0,0,0), key (lo r, hi r)) for a seed that belongs to one
 // candidate only (self-salt scheme, detection).
-__device__ __forceinline__ uint32_t philox_word0(uint32_t v, uint64_t r) {
-    const uint32_t k0 = static_cast<uint32_t>(r), k1 = static_cast<uint32_t>(r >> 32);
+__device__ __forceinline__ uint32_t philox_word0(uint32_t v, uint64_t r, const Weyl w) {
+    uint32_t k0 = static_cast<uint32_t>(r), k1 = static_cast<uint32_t>(r >> 32);
     uint32_t h, l, c0, c1, c2, c3, h0, l0, h1, l1;
     mulhilo(kPhiloxM0, v, h, l);
     c2 = h ^ k1;
     mulhilo(kPhiloxM0, k0, h0, l0);
     mulhilo(kPhiloxM1, c2, h1, l1);
-    c0 = h1 ^ (k0 + kPhiloxW0);
+    k0 += w.w0;
+    k1 += w.w1;
+    c0 = h1 ^ k0;
     c1 = l1;
-    c2 = h0 ^ l ^ (k1 + kPhiloxW1);
+    c2 = h0 ^ l ^ k1;
     c3 = l0;
 #pragma unroll
-    for (int i = 2; i < 8; ++i)
-        philox_round(c0, c1, c2, c3, k0 + static_cast<uint32_t>(i) * kPhiloxW0,
-                     k1 + static_cast<uint32_t>(i) * kPhiloxW1);
+    for (int i = 2; i < 8; ++i) {
+        k0 += w.w0;
+        k1 += w.w1;
+        philox_round(c0, c1, c2, c3, k0, k1);
+    }
+    k1 += w.w1;
+    k0 += w.w0 + w.w0;
     const uint32_t n1 = kPhiloxM1 * c2;
-    const uint32_t n2 = __umulhi(kPhiloxM0, c0) ^ c3 ^ (k1 + 8u * kPhiloxW1);
-    return __umulhi(kPhiloxM1, n2) ^ n1 ^ (k0 + 9u * kPhiloxW0);
+    const uint32_t n2 = __umulhi(kPhiloxM0, c0) ^ c3 ^ k1;
+    return __umulhi(kPhiloxM1, n2) ^ n1 ^ k0;
 }
 
 // The same two evaluations for N candidates at once, written round by round so that the N
@@ -189,7 +222,7 @@ __device__ __forceinline__ void philox_word0_n(uint32_t vbase, const RowKeys &rk
 // Per-candidate seeds r[i] (self-salt scheme, detection), arbitrary ids v[i].
 template <int N>
 __device__ __forceinline__ void philox_word0_n(const uint32_t (&v)[N], const uint64_t (&r)[N],
-                                               uint32_t (&out)[N]) {
+                                               uint32_t (&out)[N], const Weyl w) {
     uint32_t c0[N], c1[N], c2[N], c3[N], k0[N], k1[N];
 #pragma unroll
     for (int i = 0; i < N; ++i) {
@@ -205,8 +238,8 @@ __device__ __forceinline__ void philox_word0_n(const uint32_t (&v)[N], const uin
     }
 #pragma unroll
     for (int i = 0; i < N; ++i) {
-        k0[i] += kPhiloxW0;
-        k1[i] += kPhiloxW1;
+        k0[i] += w.w0;
+        k1[i] += w.w1;
         uint32_t h1, l1;
         mulhilo(kPhiloxM1, c2[i], h1, l1);
         c2[i] = c0[i] ^ c1[i] ^ k1[i];
@@ -217,16 +250,16 @@ __device__ __forceinline__ void philox_word0_n(const uint32_t (&v)[N], const uin
     for (int rd = 2; rd < 8; ++rd) {
 #pragma unroll
         for (int i = 0; i < N; ++i) {
-            k0[i] += kPhiloxW0;
-            k1[i] += kPhiloxW1;
+            k0[i] += w.w0;
+            k1[i] += w.w1;
             philox_round(c0[i], c1[i], c2[i], c3[i], k0[i], k1[i]);
         }
     }
 #pragma unroll
     for (int i = 0; i < N; ++i) {
         const uint32_t n1 = kPhiloxM1 * c2[i];
-        const uint32_t n2 = __umulhi(kPhiloxM0, c0[i]) ^ c3[i] ^ (k1[i] + kPhiloxW1);
-        out[i] = __umulhi(kPhiloxM1, n2) ^ n1 ^ (k0[i] + 2u * kPhiloxW0);
+        const uint32_t n2 = __umulhi(kPhiloxM0, c0[i]) ^ c3[i] ^ (k1[i] + w.w1);
+        out[i] = __umulhi(kPhiloxM1, n2) ^ n1 ^ (k0[i] + w.w0 + w.w0);
     }
 }
 

@@ -57,7 +57,9 @@ struct SampleArgs {
     float inv_tau;        // 1/tau rounded once to fp32 (feeds the score)
     float c2_hi, c2_lo;   // log2(e)/tau as an fp32 pair (feeds the softmax sum)
     double tau;
-    uint32_t gk0, gk1, step_lo, step_hi;   // Gumbel stream
+    uint32_t step_lo, step_hi;   // Gumbel stream: counter words 2 and 3
+    BlockKeys gkeys;             // its ten round keys
+    Weyl weyl;                   // key-schedule increments of the green hash
     int32_t *out_tokens;
     float *out_max, *out_sumexp, *out_prob;
     Partial *partials;    // [B * split]
@@ -132,14 +134,16 @@ struct RowSeedS<SBW_SCHEME_CONTEXT> {
     __device__ __forceinline__ void init(uint64_t key, const int32_t *ctx, int W) {
         rk = make_row_keys(seed_context(key, ctx, W));
     }
-    __device__ __forceinline__ uint32_t word0(uint32_t v, uint64_t) const { return philox_word0(v, rk); }
+    __device__ __forceinline__ uint32_t word0(uint32_t v, uint64_t, const Weyl) const {
+        return philox_word0(v, rk);
+    }
 };
 template <>
 struct RowSeedS<SBW_SCHEME_SELFSALT> {
     uint32_t jmin;
     __device__ __forceinline__ void init(uint64_t, const int32_t *ctx, int W) { jmin = jenkins_min(ctx, W); }
-    __device__ __forceinline__ uint32_t word0(uint32_t v, uint64_t key) const {
-        return philox_word0(v, seed_selfsalt(key, jmin, v));
+    __device__ __forceinline__ uint32_t word0(uint32_t v, uint64_t key, const Weyl w) const {
+        return philox_word0(v, seed_selfsalt(key, jmin, v), w);
     }
 };
 
@@ -245,7 +249,7 @@ sample_kernel(const SampleArgs a) {
                 uint32_t raw;
                 if constexpr (DTYPE == SBW_DTYPE_F32) raw = e[i];
                 else raw = (i & 1) ? (e[i >> 1] >> 16) : (e[i >> 1] & 0xffffu);
-                const bool green = rs.word0(vg + i, a.key) <= a.thr_m1;
+                const bool green = rs.word0(vg + i, a.key, a.weyl) <= a.thr_m1;
                 lp[i] = biased<DTYPE>(raw, green, a.delta);
             }
         } else {
@@ -257,7 +261,7 @@ sample_kernel(const SampleArgs a) {
                     uint32_t raw;
                     if constexpr (DTYPE == SBW_DTYPE_F32) raw = reinterpret_cast<const uint32_t *>(row_ptr)[cb + i];
                     else raw = reinterpret_cast<const uint16_t *>(row_ptr)[cb + i];
-                    const bool green = rs.word0(vg + i, a.key) <= a.thr_m1;
+                    const bool green = rs.word0(vg + i, a.key, a.weyl) <= a.thr_m1;
                     lp[i] = biased<DTYPE>(raw, green, a.delta);
                 }
             }
@@ -266,7 +270,7 @@ sample_kernel(const SampleArgs a) {
         if (VEC >= 4 && (vg & 3u) == 0) {
 #pragma unroll
             for (int b = 0; b < NBLK; ++b) {
-                const uint4 r = philox4x32_10((vg >> 2) + b, rowb, a.step_lo, a.step_hi, a.gk0, a.gk1);
+                const uint4 r = philox4x32_10((vg >> 2) + b, rowb, a.step_lo, a.step_hi, a.gkeys);
                 if (4 * b + 0 < VEC) y[4 * b + 0] = r.x;
                 if (4 * b + 1 < VEC) y[4 * b + 1] = r.y;
                 if (4 * b + 2 < VEC) y[4 * b + 2] = r.z;
@@ -276,7 +280,7 @@ sample_kernel(const SampleArgs a) {
 #pragma unroll
             for (int i = 0; i < VEC; ++i) {
                 const uint32_t v = vg + i;
-                const uint4 r = philox4x32_10(v >> 2, rowb, a.step_lo, a.step_hi, a.gk0, a.gk1);
+                const uint4 r = philox4x32_10(v >> 2, rowb, a.step_lo, a.step_hi, a.gkeys);
                 const uint32_t k = v & 3u;
                 y[i] = k == 0 ? r.x : k == 1 ? r.y : k == 2 ? r.z : r.w;
             }
@@ -373,7 +377,7 @@ probs_kernel(const SampleArgs a, float *out_probs) {
             if constexpr (DTYPE == SBW_DTYPE_F32) raw = reinterpret_cast<const uint32_t *>(row_ptr)[c];
             else raw = reinterpret_cast<const uint16_t *>(row_ptr)[c];
             const uint32_t v = a.vocab_offset + static_cast<uint32_t>(c);
-            const bool green = rs.word0(v, a.key) <= a.thr_m1;
+            const bool green = rs.word0(v, a.key, a.weyl) <= a.thr_m1;
             const double lp = biased<DTYPE>(raw, green, a.delta);
             out_probs[row * a.V + c] = static_cast<float>(exp((lp - st.x) / a.tau) / st.y);
         }
@@ -475,8 +479,8 @@ extern "C" int sbw_bias_sample(const void *logits, int dtype, int64_t B, int64_t
     a.c2_hi = c2_hi;
     a.c2_lo = static_cast<float>(c2 - static_cast<double>(c2_hi));
     a.tau = static_cast<double>(temperature);
-    a.gk0 = static_cast<uint32_t>(rng_seed);
-    a.gk1 = static_cast<uint32_t>(rng_seed >> 32);
+    a.gkeys = make_block_keys(static_cast<uint32_t>(rng_seed), static_cast<uint32_t>(rng_seed >> 32));
+    a.weyl = make_weyl();
     a.step_lo = static_cast<uint32_t>(rng_step);
     a.step_hi = static_cast<uint32_t>(rng_step >> 32);
     a.out_tokens = out_tokens;
