@@ -3,20 +3,24 @@
 // to the serving engine; this kernel is the "absorbed into existing logit post-processing" form
 // that Section 5.1 points at.
 //
-// Work layout.  A row is cut into 16-byte slots as in the bias kernel; a row may further be split
-// into `split` column chunks so that small batches still fill the 148 SMs.  One CTA handles one
-// (row, chunk): every thread keeps an online-softmax pair (running max m, sum of
-// exp2((l' - m) c)) and its best Gumbel score, all in registers; a CTA reduces them with warp
-// shuffles (max, then sum of rescaled partial sums, then lexicographic argmax) and shared memory
-// across its warps.  When a row is split, CTAs leave their partial in the workspace and the last
-// one to arrive (an atomic ticket, nobody waits) merges the row's partials in index order.
+// Work layout.  A row is cut into 16-byte slots as in the bias kernel and, further, into `split`
+// column chunks; the B*split (row, chunk) items are spread over a persistent grid, with `split`
+// chosen so that the item count is close to a multiple of the number of resident CTAs.  For each
+// item a CTA's threads keep an online-softmax pair (running max m, sum of exp2((l' - m) c)) and
+// their best Gumbel score in registers; the CTA reduces them with warp shuffles and shared memory
+// and leaves a partial in the workspace.  The last CTA to take a row's ticket (an atomic, nobody
+// waits) merges that row's partials in index order.
 //
 // Numerics.  The sampled id must be reproducible bit for bit, so everything that feeds it is an
 // exactly rounded fp32 operation spelled with intrinsics: the Gumbel variate is -L(-L(u)) with L
-// the fixed logarithm below, and the score is fmaf(l', 1/tau, g).  The softmax sum only has to be
-// accurate (1e-6 relative): exponent arguments are formed as a rounded product plus its exact
-// rounding error, exp2 of the rounded part comes from the SFU (2 ulp), and the error term is
-// applied to first order.  The per-row finish (merging chunk partials, p = exp(.)/Z) is fp64.
+// the fixed logarithm below, and the score is fmaf(l', 1/tau, g).  Most candidates cannot win,
+// and the two logarithms are the most expensive part of a candidate, so each warp first applies
+// a conservative test on the raw Philox word (see word_floor) and evaluates the exact score only
+// for slots in which some candidate might reach the warp's best score so far; the result is the
+// same argmax as evaluating every candidate.  The softmax sum only has to be accurate (1e-6
+// relative): exponent arguments are formed as a rounded product plus its exact rounding error,
+// exp2 of the rounded part comes from the SFU (2 ulp), and the error term is applied to first
+// order.  The per-row finish (merging chunk partials, p = exp(.)/Z) is fp64.
 #include <cuda_bf16.h>
 
 #include <cfloat>
@@ -29,10 +33,14 @@
 namespace sbw {
 namespace {
 
+#ifndef SBW_SAMPLE_MIN_BLOCKS
+#define SBW_SAMPLE_MIN_BLOCKS 2
+#endif
 constexpr int kSampleThreads = 256;
 constexpr int kSampleWarps = kSampleThreads / 32;
-constexpr int kTargetCtas = 1184;      // 148 SMs x 8: enough CTAs to fill the GPU twice over
-constexpr int kMinSlotsPerCta = 256;   // one slot per thread at least
+constexpr int kMaxSplit = 64;          // chunks per row at most
+constexpr int kMinSlotsPerItem = 256;  // one slot per thread at least
+constexpr int kLegacyTargetCtas = 1184;
 
 struct __align__(32) Partial {
     float m;      // max of l' over the chunk
@@ -46,6 +54,7 @@ struct __align__(32) Partial {
 struct SampleArgs {
     const void *logits;
     int64_t B, V, ld;
+    int64_t n_items;      // B * split
     uint32_t nslot, slots_per_chunk;
     int split;
     const int32_t *ctx;
@@ -54,6 +63,7 @@ struct SampleArgs {
     uint64_t key;
     uint32_t thr_m1;
     float delta;          // in the logits' precision, widened
+    uint32_t delta_bf16;  // bf16 bits of delta
     float inv_tau;        // 1/tau rounded once to fp32 (feeds the score)
     float c2_hi, c2_lo;   // log2(e)/tau as an fp32 pair (feeds the softmax sum)
     double tau;
@@ -64,8 +74,25 @@ struct SampleArgs {
     float *out_max, *out_sumexp, *out_prob;
     Partial *partials;    // [B * split]
     unsigned *tickets;    // [B], zero before the launch
+    unsigned *bounds;     // [B], zero before the launch: best exact score per row, order-encoded
     double2 *rowstats;    // [B] (m, Z) for the optional probabilities pass
 };
+
+// Monotone map float -> unsigned (larger float, larger code); code 0 decodes to a NaN, which the
+// screen treats as "no bound yet", so a zeroed array needs no other initialisation.
+__device__ __forceinline__ unsigned encode_score(float f) {
+    const unsigned b = __float_as_uint(f);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float decode_score(unsigned c) {
+    return __uint_as_float((c & 0x80000000u) ? (c & 0x7fffffffu) : ~c);
+}
+
+__device__ __forceinline__ uint32_t add_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
 
 // ---------------------------------------------------------------------------------------------
 // Fixed fp32 natural logarithm for positive normal x; every step is one IEEE operation.
@@ -91,10 +118,10 @@ __device__ __forceinline__ float fixed_log(float x) {
     return __fmaf_rn(fe, 0x1.62e43p-1f, __fmaf_rn(fe, -0x1.05c61p-29f, t));
 }
 
-// -L(u) for the uniform built from a Philox word: u = ((y >> 9) + 1/2) 2^-23 (exact in fp32).
-__device__ __forceinline__ float neg_log_uniform(uint32_t y) {
+// Standard Gumbel variate of a Philox word: u = ((y >> 9) + 1/2) 2^-23 (exact), g = -L(-L(u)).
+__device__ __forceinline__ float gumbel_of_word(uint32_t y) {
     const float u = __fmaf_rn(__uint2float_rn(y >> 9), 0x1p-23f, 0x1p-24f);
-    return -fixed_log(u);
+    return -fixed_log(-fixed_log(u));
 }
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -117,6 +144,25 @@ __device__ __forceinline__ float exp2_scaled(float d, float c_hi, float c_lo) {
     return __fmaf_rn(e, lo * 0.693147180559945f, e);
 }
 
+// Conservative screen for the Gumbel-max.  A candidate of a slot whose largest biased logit is
+// `vmax` can reach the score `bound` only if its Gumbel variate g is at least
+// T = bound - vmax/tau.  g = -ln(-ln u) increases with u, so that requires
+// u >= exp(-exp(-T)), i.e. a Philox word of at least about 2^32 exp(-exp(-T)).  The value
+// returned here is a lower bound of that word: T is lowered by a margin that covers the error
+// of the fixed logarithm (|g - g_exact| < 4e-6) and every fp32 rounding on the way, the inner
+// exponential is rounded up and the outer one down by 1e-4 relative (SFU error 2^-22 plus the
+// rounding of their arguments), and 1024 is subtracted to cover the 9 dropped bits of the word
+// and the float-to-integer step.  Words below the returned value provably lose; everything
+// else is scored exactly.  bound = -inf (nothing scored yet) returns 0: nobody is screened out.
+__device__ __forceinline__ uint32_t word_floor(float bound, float vmax, float inv_tau) {
+    const float T = __fmaf_rn(-vmax, inv_tau, bound);
+    const float Tm = T - (1e-3f + 1e-5f * (fabsf(T) + fabsf(bound)));
+    const float E = ex2_approx(Tm * -1.4426950408889634f) * 1.0001f;      // >= exp(-Tm)
+    const float U = ex2_approx(E * -1.4426950408889634f) * 0.9999f;       // <= exp(-exp(-Tm))
+    const uint32_t k = __float2uint_rd(U * 4294967296.0f);                // NaN -> 0
+    return k > 1024u ? k - 1024u : 0u;
+}
+
 struct Best {
     float s;
     int id;
@@ -137,6 +183,10 @@ struct RowSeedS<SBW_SCHEME_CONTEXT> {
     __device__ __forceinline__ uint32_t word0(uint32_t v, uint64_t, const Weyl) const {
         return philox_word0(v, rk);
     }
+    template <int N>
+    __device__ __forceinline__ void word0_n(uint32_t vg, uint64_t, const Weyl, uint32_t (&x)[N]) const {
+        philox_word0_n<N>(vg, rk, x);
+    }
 };
 template <>
 struct RowSeedS<SBW_SCHEME_SELFSALT> {
@@ -144,6 +194,17 @@ struct RowSeedS<SBW_SCHEME_SELFSALT> {
     __device__ __forceinline__ void init(uint64_t, const int32_t *ctx, int W) { jmin = jenkins_min(ctx, W); }
     __device__ __forceinline__ uint32_t word0(uint32_t v, uint64_t key, const Weyl w) const {
         return philox_word0(v, seed_selfsalt(key, jmin, v), w);
+    }
+    template <int N>
+    __device__ __forceinline__ void word0_n(uint32_t vg, uint64_t key, const Weyl w, uint32_t (&x)[N]) const {
+        uint32_t v[N];
+        uint64_t r[N];
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+            v[i] = vg + i;
+            r[i] = seed_selfsalt(key, jmin, v[i]);
+        }
+        philox_word0_n<N>(v, r, x, w);
     }
 };
 
@@ -209,155 +270,206 @@ __device__ void finish_row(const SampleArgs &a, int64_t row, const Partial *part
     }
 }
 
+// Biased logits lp[0..VEC) of slot j (columns cb .. cb+VEC-1); columns at or beyond V give -inf.
+template <int DTYPE, int SCHEME, bool VECTOR, int VEC>
+__device__ __forceinline__ void load_biased(const SampleArgs &a, const RowSeedS<SCHEME> &rs, const char *row_ptr,
+                                            uint32_t j, uint32_t cb, uint32_t V, float (&lp)[VEC]) {
+    const uint32_t vg = a.vocab_offset + cb;
+    if (VECTOR && cb + VEC <= V) {
+        const uint4 w = __ldg(reinterpret_cast<const uint4 *>(row_ptr) + j);
+        const uint32_t *e = reinterpret_cast<const uint32_t *>(&w);
+        uint32_t x[VEC];
+        rs.template word0_n<VEC>(vg, a.key, a.weyl, x);
+        if constexpr (DTYPE == SBW_DTYPE_F32) {
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                const float v = __uint_as_float(e[i]);
+                lp[i] = x[i] <= a.thr_m1 ? __fadd_rn(v, a.delta) : v;
+            }
+        } else {
+            // one packed bf16 add per pair with {delta or -0.0} per half, then widen
+            const uint32_t dlo = a.delta_bf16, dhi = a.delta_bf16 << 16;
+#pragma unroll
+            for (int i = 0; i < VEC / 2; ++i) {
+                const uint32_t d = (x[2 * i] <= a.thr_m1 ? dlo : 0x8000u) |
+                                   (x[2 * i + 1] <= a.thr_m1 ? dhi : 0x80000000u);
+                const uint32_t b = add_bf16x2(e[i], d);
+                lp[2 * i] = __uint_as_float(b << 16);
+                lp[2 * i + 1] = __uint_as_float(b & 0xffff0000u);
+            }
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+            lp[i] = -INFINITY;
+            if (cb + i < V) {
+                uint32_t raw;
+                if constexpr (DTYPE == SBW_DTYPE_F32) raw = reinterpret_cast<const uint32_t *>(row_ptr)[cb + i];
+                else raw = reinterpret_cast<const uint16_t *>(row_ptr)[cb + i];
+                lp[i] = biased<DTYPE>(raw, rs.word0(vg + i, a.key, a.weyl) <= a.thr_m1, a.delta);
+            }
+        }
+    }
+}
+
+// Philox words of the Gumbel stream for the VEC candidates starting at global id vg:
+// candidate v uses word v & 3 of block v >> 2.
+template <int VEC>
+__device__ __forceinline__ void gumbel_words(const SampleArgs &a, uint32_t vg, uint32_t rowb, uint32_t (&y)[VEC]) {
+    if (VEC >= 4 && (vg & 3u) == 0) {
+#pragma unroll
+        for (int b = 0; b < (VEC >= 4 ? VEC / 4 : 1); ++b) {
+            const uint4 r = philox4x32_10((vg >> 2) + b, rowb, a.step_lo, a.step_hi, a.gkeys);
+            if (4 * b + 0 < VEC) y[4 * b + 0] = r.x;
+            if (4 * b + 1 < VEC) y[4 * b + 1] = r.y;
+            if (4 * b + 2 < VEC) y[4 * b + 2] = r.z;
+            if (4 * b + 3 < VEC) y[4 * b + 3] = r.w;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+            const uint32_t v = vg + i;
+            const uint4 r = philox4x32_10(v >> 2, rowb, a.step_lo, a.step_hi, a.gkeys);
+            const uint32_t k = v & 3u;
+            y[i] = k == 0 ? r.x : k == 1 ? r.y : k == 2 ? r.z : r.w;
+        }
+    }
+}
+
 template <int DTYPE, int SCHEME, bool VECTOR>
-__global__ void __launch_bounds__(kSampleThreads)
+__global__ void __launch_bounds__(kSampleThreads, SBW_SAMPLE_MIN_BLOCKS)
 sample_kernel(const SampleArgs a) {
     constexpr int VEC = VECTOR ? (DTYPE == SBW_DTYPE_F32 ? 4 : 8) : 1;
     constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
-    constexpr int NBLK = VEC >= 4 ? VEC / 4 : 1;     // Philox blocks per aligned slot
     __shared__ float sh_f[kSampleWarps];
     __shared__ float sh_s[kSampleWarps];
     __shared__ int sh_id[kSampleWarps];
     __shared__ float sh_l[kSampleWarps];
     __shared__ unsigned sh_ticket;
-
-    const int64_t row = blockIdx.x / a.split;
-    const int chunk = static_cast<int>(blockIdx.x - row * a.split);
-    const uint32_t j_begin = chunk * a.slots_per_chunk;
-    const uint32_t j_end = min(a.nslot, j_begin + a.slots_per_chunk);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t V = static_cast<uint32_t>(a.V);
-    const uint32_t rowb = static_cast<uint32_t>(row);
-    const char *row_ptr = static_cast<const char *>(a.logits) + row * a.ld * ESIZE;
 
-    RowSeedS<SCHEME> rs;
-    rs.init(a.key, a.ctx + row * a.W, a.W);
+    for (int64_t item = blockIdx.x; item < a.n_items; item += gridDim.x) {
+        const int64_t row = item / a.split;
+        const int chunk = static_cast<int>(item - row * a.split);
+        const uint32_t j_begin = chunk * a.slots_per_chunk;
+        const uint32_t j_end = min(a.nslot, j_begin + a.slots_per_chunk);
+        const uint32_t rowb = static_cast<uint32_t>(row);
+        const char *row_ptr = static_cast<const char *>(a.logits) + row * a.ld * ESIZE;
 
-    float m_t = -INFINITY, z1 = 0.0f, z2 = 0.0f;
-    Best best = {-INFINITY, INT_MAX, -INFINITY};
+        RowSeedS<SCHEME> rs;
+        rs.init(a.key, a.ctx + row * a.W, a.W);
 
-    for (uint32_t j = j_begin + threadIdx.x; j < j_end; j += kSampleThreads) {
-        const uint32_t cb = j * VEC;
-        const uint32_t vg = a.vocab_offset + cb;
-        float lp[VEC];
-        uint32_t y[VEC];
-        int nvalid = VEC;
-        if (VECTOR && cb + VEC <= V) {
-            const uint4 w = __ldg(reinterpret_cast<const uint4 *>(row_ptr) + j);
-            const uint32_t *e = reinterpret_cast<const uint32_t *>(&w);
+        float m_t = -INFINITY, z1 = 0.0f, z2 = 0.0f;
+        Best best = {-INFINITY, INT_MAX, -INFINITY};
+        // best exact score seen so far: by this warp, and (through the workspace) by every warp
+        // that works on the same row -- a lower bound of the row's final best score
+        float bound = -INFINITY;
+
+        // warp-uniform trip count: lanes past the end of the chunk carry an empty slot
+        for (uint32_t jb = j_begin + warp * 32; jb < j_end; jb += kSampleThreads) {
+            const unsigned shared_bound = __ldcg(a.bounds + row);
+            const uint32_t j = jb + lane;
+            const bool live = j < j_end;
+            const uint32_t cb = j * VEC;
+            float lp[VEC];
+            uint32_t y[VEC];
+            if (live) {
+                load_biased<DTYPE, SCHEME, VECTOR, VEC>(a, rs, row_ptr, j, cb, V, lp);
+                gumbel_words<VEC>(a, a.vocab_offset + cb, rowb, y);
+            } else {
 #pragma unroll
-            for (int i = 0; i < VEC; ++i) {
-                uint32_t raw;
-                if constexpr (DTYPE == SBW_DTYPE_F32) raw = e[i];
-                else raw = (i & 1) ? (e[i >> 1] >> 16) : (e[i >> 1] & 0xffffu);
-                const bool green = rs.word0(vg + i, a.key, a.weyl) <= a.thr_m1;
-                lp[i] = biased<DTYPE>(raw, green, a.delta);
+                for (int i = 0; i < VEC; ++i) { lp[i] = -INFINITY; y[i] = 0u; }
             }
-        } else {
-            nvalid = static_cast<int>(min(static_cast<uint32_t>(VEC), V - cb));
+            // online softmax
+            float vmax = lp[0];
 #pragma unroll
-            for (int i = 0; i < VEC; ++i) {
-                lp[i] = -INFINITY;
-                if (i < nvalid) {
-                    uint32_t raw;
-                    if constexpr (DTYPE == SBW_DTYPE_F32) raw = reinterpret_cast<const uint32_t *>(row_ptr)[cb + i];
-                    else raw = reinterpret_cast<const uint16_t *>(row_ptr)[cb + i];
-                    const bool green = rs.word0(vg + i, a.key, a.weyl) <= a.thr_m1;
-                    lp[i] = biased<DTYPE>(raw, green, a.delta);
+            for (int i = 1; i < VEC; ++i) vmax = fmaxf(vmax, lp[i]);
+            if (vmax > m_t) {
+                const float f = exp2_scaled(m_t - vmax, a.c2_hi, a.c2_lo);   // 0 when m_t = -inf
+                z1 *= f;
+                z2 *= f;
+                m_t = vmax;
+            }
+            if (m_t > -INFINITY) {
+#pragma unroll
+                for (int i = 0; i < VEC; ++i) {
+                    float lo;
+                    const float e = exp2_split(lp[i] - m_t, a.c2_hi, a.c2_lo, lo);
+                    z1 += e;
+                    z2 = fmaf(e, lo, z2);
+                }
+            }
+            // Gumbel-max: screen on the raw words, score exactly only where somebody might win
+            bound = fmaxf(bound, decode_score(shared_bound));     // fmaxf drops the NaN of "none yet"
+            const uint32_t floor_word = word_floor(bound, vmax, a.inv_tau);
+            bool maybe = false;
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) maybe |= y[i] >= floor_word;
+            maybe &= live;
+            if (__any_sync(0xffffffffu, maybe)) {
+                if (live) {
+#pragma unroll
+                    for (int i = 0; i < VEC; ++i) {
+                        if (cb + i < V) {
+                            const float s = __fmaf_rn(lp[i], a.inv_tau, gumbel_of_word(y[i]));
+                            if (s > best.s) { best.s = s; best.id = static_cast<int>(cb + i); best.l = lp[i]; }
+                        }
+                    }
+                }
+                float b = best.s;
+                for (int d = 16; d > 0; d >>= 1) b = fmaxf(b, __shfl_xor_sync(0xffffffffu, b, d));
+                if (b > bound) {
+                    bound = b;
+                    if (lane == 0) atomicMax(a.bounds + row, encode_score(b));
                 }
             }
         }
-        // Gumbel words: candidate vg+i uses word (vg+i)&3 of block (vg+i)>>2
-        if (VEC >= 4 && (vg & 3u) == 0) {
-#pragma unroll
-            for (int b = 0; b < NBLK; ++b) {
-                const uint4 r = philox4x32_10((vg >> 2) + b, rowb, a.step_lo, a.step_hi, a.gkeys);
-                if (4 * b + 0 < VEC) y[4 * b + 0] = r.x;
-                if (4 * b + 1 < VEC) y[4 * b + 1] = r.y;
-                if (4 * b + 2 < VEC) y[4 * b + 2] = r.z;
-                if (4 * b + 3 < VEC) y[4 * b + 3] = r.w;
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < VEC; ++i) {
-                const uint32_t v = vg + i;
-                const uint4 r = philox4x32_10(v >> 2, rowb, a.step_lo, a.step_hi, a.gkeys);
-                const uint32_t k = v & 3u;
-                y[i] = k == 0 ? r.x : k == 1 ? r.y : k == 2 ? r.z : r.w;
-            }
-        }
-        // online softmax
-        float vmax = lp[0];
-#pragma unroll
-        for (int i = 1; i < VEC; ++i) vmax = fmaxf(vmax, lp[i]);
-        if (vmax > m_t) {
-            const float f = exp2_scaled(m_t - vmax, a.c2_hi, a.c2_lo);   // 0 when m_t = -inf
-            z1 *= f;
-            z2 *= f;
-            m_t = vmax;
-        }
-        if (m_t > -INFINITY) {
-#pragma unroll
-            for (int i = 0; i < VEC; ++i) {
-                float lo;
-                const float e = exp2_split(lp[i] - m_t, a.c2_hi, a.c2_lo, lo);
-                z1 += e;
-                z2 = fmaf(e, lo, z2);
-            }
-        }
-        // Gumbel-max
-#pragma unroll
-        for (int i = 0; i < VEC; ++i) {
-            if (i < nvalid) {
-                const float w = neg_log_uniform(y[i]);
-                const float s = __fmaf_rn(lp[i], a.inv_tau, -fixed_log(w));
-                if (s > best.s) { best.s = s; best.id = static_cast<int>(cb + i); best.l = lp[i]; }
-            }
-        }
-    }
 
-    // ---- CTA reduction ----
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float m_w = m_t;
-    for (int d = 16; d > 0; d >>= 1) m_w = fmaxf(m_w, __shfl_xor_sync(0xffffffffu, m_w, d));
-    if (lane == 0) sh_f[warp] = m_w;
-    __syncthreads();
-    float m_cta = sh_f[0];
+        // ---- CTA reduction ----
+        float m_w = m_t;
+        for (int d = 16; d > 0; d >>= 1) m_w = fmaxf(m_w, __shfl_xor_sync(0xffffffffu, m_w, d));
+        if (lane == 0) sh_f[warp] = m_w;
+        __syncthreads();
+        float m_cta = sh_f[0];
 #pragma unroll
-    for (int w = 1; w < kSampleWarps; ++w) m_cta = fmaxf(m_cta, sh_f[w]);
-    __syncthreads();
-    float z_t = 0.0f;
-    if (m_t > -INFINITY) z_t = (z1 + 0.693147180559945f * z2) * exp2_scaled(m_t - m_cta, a.c2_hi, a.c2_lo);
-    for (int d = 16; d > 0; d >>= 1) z_t += __shfl_down_sync(0xffffffffu, z_t, d);
-    for (int d = 16; d > 0; d >>= 1) {
-        const float os = __shfl_down_sync(0xffffffffu, best.s, d);
-        const int oid = __shfl_down_sync(0xffffffffu, best.id, d);
-        const float ol = __shfl_down_sync(0xffffffffu, best.l, d);
-        if (better(os, oid, best.s, best.id)) { best.s = os; best.id = oid; best.l = ol; }
-    }
-    if (lane == 0) { sh_f[warp] = z_t; sh_s[warp] = best.s; sh_id[warp] = best.id; sh_l[warp] = best.l; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        Partial p;
-        p.m = m_cta;
-        p.z = 0.0f;
-        p.s = sh_s[0]; p.id = sh_id[0]; p.l = sh_l[0];
-        for (int w = 0; w < kSampleWarps; ++w) {
-            p.z += sh_f[w];
-            if (w > 0 && better(sh_s[w], sh_id[w], p.s, p.id)) { p.s = sh_s[w]; p.id = sh_id[w]; p.l = sh_l[w]; }
+        for (int w = 1; w < kSampleWarps; ++w) m_cta = fmaxf(m_cta, sh_f[w]);
+        __syncthreads();
+        float z_t = 0.0f;
+        if (m_t > -INFINITY) z_t = (z1 + 0.693147180559945f * z2) * exp2_scaled(m_t - m_cta, a.c2_hi, a.c2_lo);
+        for (int d = 16; d > 0; d >>= 1) z_t += __shfl_down_sync(0xffffffffu, z_t, d);
+        for (int d = 16; d > 0; d >>= 1) {
+            const float os = __shfl_down_sync(0xffffffffu, best.s, d);
+            const int oid = __shfl_down_sync(0xffffffffu, best.id, d);
+            const float ol = __shfl_down_sync(0xffffffffu, best.l, d);
+            if (better(os, oid, best.s, best.id)) { best.s = os; best.id = oid; best.l = ol; }
         }
-        p.pad[0] = p.pad[1] = p.pad[2] = 0.0f;
-        a.partials[blockIdx.x] = p;
-        unsigned ticket = 0;
-        __threadfence();                           // partial visible before the ticket is taken
-        if (a.split > 1) ticket = atomicAdd(&a.tickets[row], 1u);
-        sh_ticket = ticket;
-    }
-    __syncthreads();
-    if (a.split > 1 && sh_ticket != static_cast<unsigned>(a.split - 1)) return;
-    if (warp == 0) {
-        if (a.split > 1) __threadfence();          // the other CTAs' partials are visible now
-        finish_row(a, row, a.partials + row * a.split, a.split);
-        if (lane == 0 && a.split > 1) a.tickets[row] = 0;
+        if (lane == 0) { sh_f[warp] = z_t; sh_s[warp] = best.s; sh_id[warp] = best.id; sh_l[warp] = best.l; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            Partial p;
+            p.m = m_cta;
+            p.z = 0.0f;
+            p.s = sh_s[0]; p.id = sh_id[0]; p.l = sh_l[0];
+            for (int w = 0; w < kSampleWarps; ++w) {
+                p.z += sh_f[w];
+                if (w > 0 && better(sh_s[w], sh_id[w], p.s, p.id)) { p.s = sh_s[w]; p.id = sh_id[w]; p.l = sh_l[w]; }
+            }
+            p.pad[0] = p.pad[1] = p.pad[2] = 0.0f;
+            a.partials[item] = p;
+            unsigned ticket = 0;
+            __threadfence();                           // partial visible before the ticket is taken
+            if (a.split > 1) ticket = atomicAdd(&a.tickets[row], 1u);
+            sh_ticket = ticket;
+        }
+        __syncthreads();
+        const bool last = a.split == 1 || sh_ticket == static_cast<unsigned>(a.split - 1);
+        if (last && warp == 0) {
+            if (a.split > 1) __threadfence();          // the other CTAs' partials are visible now
+            finish_row(a, row, a.partials + row * a.split, a.split);
+            if (lane == 0 && a.split > 1) a.tickets[row] = 0;
+        }
+        __syncthreads();                               // shared scratch is reused by the next item
     }
 }
 
@@ -384,19 +496,12 @@ probs_kernel(const SampleArgs a, float *out_probs) {
     }
 }
 
-int choose_split(int64_t B, int64_t nslot) {
-    int64_t split = (kTargetCtas + B - 1) / B;
-    const int64_t max_split = nslot / kMinSlotsPerCta > 1 ? nslot / kMinSlotsPerCta : 1;
-    if (split > max_split) split = max_split;
-    if (split < 1) split = 1;
-    return static_cast<int>(split);
-}
-
 struct Workspace {
     double2 *rowstats;
     unsigned *tickets;
+    unsigned *bounds;
     Partial *partials;
-    size_t bytes;
+    size_t fixed_bytes;   // everything but the partials
 };
 Workspace carve(void *base, int64_t B) {
     Workspace w;
@@ -404,20 +509,71 @@ Workspace carve(void *base, int64_t B) {
     size_t off = 0;
     w.rowstats = reinterpret_cast<double2 *>(p + off);
     off += align_up(static_cast<size_t>(B) * sizeof(double2), 256);
-    w.tickets = reinterpret_cast<unsigned *>(p + off);
-    off += align_up(static_cast<size_t>(B) * sizeof(unsigned), 256);
+    w.tickets = reinterpret_cast<unsigned *>(p + off);                 // tickets and bounds are
+    w.bounds = w.tickets + B;                                           // cleared by one memset
+    off += align_up(2 * static_cast<size_t>(B) * sizeof(unsigned), 256);
     w.partials = reinterpret_cast<Partial *>(p + off);
-    off += align_up(static_cast<size_t>(B + kTargetCtas) * sizeof(Partial), 256);
-    w.bytes = off;
+    w.fixed_bytes = off;
     return w;
+}
+// Bytes every call needs (one partial per row) and bytes that let the library split rows freely.
+size_t workspace_min_bytes(int64_t B) {
+    return carve(nullptr, B).fixed_bytes + align_up(static_cast<size_t>(B) * sizeof(Partial), 256);
+}
+size_t workspace_full_bytes(int64_t B) {
+    // B * split partials with split <= kMaxSplit, but never more than B + kLegacyTargetCtas rows
+    // worth when B is large (items beyond a few waves of CTAs bring nothing)
+    const int64_t parts = B * kMaxSplit < 4 * (B + kLegacyTargetCtas) ? B * kMaxSplit : 4 * (B + kLegacyTargetCtas);
+    return carve(nullptr, B).fixed_bytes + align_up(static_cast<size_t>(parts) * sizeof(Partial), 256);
+}
+
+// Chunks per row: the smallest split whose item count B*split fills whole waves of `ctas`
+// resident CTAs to 95 %, else the fullest one; bounded by the row length and by the workspace.
+int choose_split(int64_t B, int64_t nslot, int64_t ctas, int64_t max_parts) {
+    int64_t max_split = nslot / kMinSlotsPerItem;
+    if (max_split > kMaxSplit) max_split = kMaxSplit;
+    if (max_split > max_parts / B) max_split = max_parts / B;
+    if (max_split < 1) max_split = 1;
+    int best = 1;
+    double best_eff = 0.0;
+    for (int64_t s = 1; s <= max_split; ++s) {
+        const int64_t items = B * s;
+        const int64_t waves = (items + ctas - 1) / ctas;
+        const double eff = static_cast<double>(items) / static_cast<double>(waves * ctas);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = static_cast<int>(s); }
+        if (eff >= 0.95) return static_cast<int>(s);
+    }
+    return best;
+}
+
+template <int DTYPE, int SCHEME, bool VECTOR>
+int launch_one(SampleArgs &a, int64_t nslot, size_t partial_bytes, cudaStream_t s) {
+    DeviceInfo di;
+    const int rc = current_device_info(&di);
+    if (rc != SBW_OK) return rc;
+    static int blocks_per_sm = 0;
+    if (blocks_per_sm == 0) {
+        int n = 0;
+        SBW_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, sample_kernel<DTYPE, SCHEME, VECTOR>,
+                                                                   kSampleThreads, 0));
+        blocks_per_sm = n > 0 ? n : 1;
+    }
+    const int64_t ctas = static_cast<int64_t>(di.sm_count) * blocks_per_sm;
+    a.split = choose_split(a.B, nslot, ctas, static_cast<int64_t>(partial_bytes / sizeof(Partial)));
+    a.n_items = a.B * a.split;
+    a.slots_per_chunk = static_cast<uint32_t>((nslot + a.split - 1) / a.split);
+    SBW_CUDA_TRY(cudaMemsetAsync(a.tickets, 0, 2 * static_cast<size_t>(a.B) * sizeof(unsigned), s));
+    const unsigned grid = static_cast<unsigned>(a.n_items < ctas ? a.n_items : ctas);
+    sample_kernel<DTYPE, SCHEME, VECTOR><<<grid, kSampleThreads, 0, s>>>(a);
+    SBW_CUDA_TRY(cudaGetLastError());
+    return SBW_OK;
 }
 
 template <int DTYPE, int SCHEME>
-int launch(const SampleArgs &a, bool vector, float *out_probs, cudaStream_t s) {
-    const unsigned grid = static_cast<unsigned>(a.B * a.split);
-    if (vector) sample_kernel<DTYPE, SCHEME, true><<<grid, kSampleThreads, 0, s>>>(a);
-    else sample_kernel<DTYPE, SCHEME, false><<<grid, kSampleThreads, 0, s>>>(a);
-    SBW_CUDA_TRY(cudaGetLastError());
+int launch(SampleArgs &a, bool vector, int64_t nslot, size_t partial_bytes, float *out_probs, cudaStream_t s) {
+    const int rc = vector ? launch_one<DTYPE, SCHEME, true>(a, nslot, partial_bytes, s)
+                          : launch_one<DTYPE, SCHEME, false>(a, nslot, partial_bytes, s);
+    if (rc != SBW_OK) return rc;
     if (out_probs) {
         const unsigned gx = static_cast<unsigned>((a.V + 255) / 256 < 1024 ? (a.V + 255) / 256 : 1024);
         const unsigned gy = static_cast<unsigned>(a.B < 4096 ? a.B : 4096);
@@ -427,12 +583,84 @@ int launch(const SampleArgs &a, bool vector, float *out_probs, cudaStream_t s) {
     return SBW_OK;
 }
 
+// Shared by the two entry points: `workspace_bytes` must cover workspace_min_bytes(B); more
+// lets rows be split into more chunks.
+int bias_sample_impl(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld, int64_t vocab_offset,
+                     const int32_t *ctx_tokens, int ctx_width, uint64_t key, double gamma, float delta,
+                     int scheme, float temperature, uint64_t rng_seed, uint64_t rng_step, int32_t *out_tokens,
+                     float *out_max, float *out_sumexp, float *out_prob, float *out_probs, void *workspace,
+                     size_t workspace_bytes, bool need_full_workspace, cudaStream_t s) {
+    if (!valid_common(dtype, ctx_width, gamma, scheme)) return SBW_ERR_INVALID_ARG;
+    if (B < 0 || V <= 0 || ld < V || vocab_offset < 0) return SBW_ERR_INVALID_ARG;
+    if (!(temperature > 0.0f) || temperature - temperature != 0.0f) return SBW_ERR_INVALID_ARG;
+    if (!(delta == delta) || delta - delta != 0.0f) return SBW_ERR_INVALID_ARG;
+    if (V > 0x7fffffffLL || vocab_offset + V > (int64_t(1) << 32)) return SBW_ERR_UNSUPPORTED;
+    if (B > 0x7fffffffLL / kMaxSplit) return SBW_ERR_UNSUPPORTED;
+    if (B == 0) return SBW_OK;
+    if (!logits || !ctx_tokens || !out_tokens) return SBW_ERR_INVALID_ARG;
+    const double c2 = 1.4426950408889634 / static_cast<double>(temperature);
+    const float c2_hi = static_cast<float>(c2);
+    if (!(c2_hi * 1e15f < FLT_MAX)) return SBW_ERR_INVALID_ARG;   // temperature too small
+    const size_t need = need_full_workspace ? workspace_full_bytes(B) : workspace_min_bytes(B);
+    if (!workspace || workspace_bytes < need || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
+        return SBW_ERR_WORKSPACE;
+    const Workspace ws = carve(workspace, B);
+
+    const int esize = dtype == SBW_DTYPE_F32 ? 4 : 2;
+    const bool vector = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && ((ld * esize) % 16 == 0);
+    const int vec = vector ? 16 / esize : 1;
+    const int64_t nslot = (V + vec - 1) / vec;
+
+    SampleArgs a;
+    a.logits = logits;
+    a.B = B; a.V = V; a.ld = ld;
+    a.nslot = static_cast<uint32_t>(nslot);
+    a.ctx = ctx_tokens;
+    a.W = ctx_width;
+    a.vocab_offset = static_cast<uint32_t>(vocab_offset);
+    a.key = key;
+    a.thr_m1 = threshold_minus_one(gamma);
+    a.delta = delta;
+    a.delta_bf16 = 0;
+    if (dtype == SBW_DTYPE_BF16) {
+        const __nv_bfloat16 d = __float2bfloat16_rn(delta);
+        a.delta_bf16 = static_cast<uint32_t>(__bfloat16_as_ushort(d));
+        a.delta = __bfloat162float(d);
+    }
+    a.inv_tau = 1.0f / temperature;
+    a.c2_hi = c2_hi;
+    a.c2_lo = static_cast<float>(c2 - static_cast<double>(c2_hi));
+    a.tau = static_cast<double>(temperature);
+    a.step_lo = static_cast<uint32_t>(rng_step);
+    a.step_hi = static_cast<uint32_t>(rng_step >> 32);
+    a.gkeys = make_block_keys(static_cast<uint32_t>(rng_seed), static_cast<uint32_t>(rng_seed >> 32));
+    a.weyl = make_weyl();
+    a.out_tokens = out_tokens;
+    a.out_max = out_max;
+    a.out_sumexp = out_sumexp;
+    a.out_prob = out_prob;
+    a.partials = ws.partials;
+    a.tickets = ws.tickets;
+    a.bounds = ws.bounds;
+    a.rowstats = ws.rowstats;
+    const size_t partial_bytes = workspace_bytes - ws.fixed_bytes;
+
+    if (dtype == SBW_DTYPE_F32) {
+        return scheme == SBW_SCHEME_CONTEXT
+                   ? launch<SBW_DTYPE_F32, SBW_SCHEME_CONTEXT>(a, vector, nslot, partial_bytes, out_probs, s)
+                   : launch<SBW_DTYPE_F32, SBW_SCHEME_SELFSALT>(a, vector, nslot, partial_bytes, out_probs, s);
+    }
+    return scheme == SBW_SCHEME_CONTEXT
+               ? launch<SBW_DTYPE_BF16, SBW_SCHEME_CONTEXT>(a, vector, nslot, partial_bytes, out_probs, s)
+               : launch<SBW_DTYPE_BF16, SBW_SCHEME_SELFSALT>(a, vector, nslot, partial_bytes, out_probs, s);
+}
+
 }  // namespace
 }  // namespace sbw
 
 extern "C" size_t sbw_sample_workspace_bytes(int64_t B, int64_t V) {
     if (B <= 0 || V <= 0) return 0;
-    return sbw::carve(nullptr, B).bytes;
+    return sbw::workspace_full_bytes(B);
 }
 
 extern "C" int sbw_bias_sample(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
@@ -441,64 +669,10 @@ extern "C" int sbw_bias_sample(const void *logits, int dtype, int64_t B, int64_t
                                uint64_t rng_seed, uint64_t rng_step, int32_t *out_tokens, float *out_max,
                                float *out_sumexp, float *out_prob, float *out_probs, void *workspace,
                                size_t workspace_bytes, void *stream) {
-    using namespace sbw;
-    if (!valid_common(dtype, ctx_width, gamma, scheme)) return SBW_ERR_INVALID_ARG;
-    if (B < 0 || V <= 0 || ld < V || vocab_offset < 0) return SBW_ERR_INVALID_ARG;
-    if (!(temperature > 0.0f) || temperature - temperature != 0.0f) return SBW_ERR_INVALID_ARG;
-    if (!(delta == delta) || delta - delta != 0.0f) return SBW_ERR_INVALID_ARG;
-    if (V > 0x7fffffffLL || vocab_offset + V > (int64_t(1) << 32)) return SBW_ERR_UNSUPPORTED;
-    if (B == 0) return SBW_OK;
-    if (!logits || !ctx_tokens || !out_tokens) return SBW_ERR_INVALID_ARG;
-    const double c2 = 1.4426950408889634 / static_cast<double>(temperature);
-    const float c2_hi = static_cast<float>(c2);
-    if (!(c2_hi * 1e15f < FLT_MAX)) return SBW_ERR_INVALID_ARG;   // temperature too small
-    const Workspace ws = carve(workspace, B);
-    if (!workspace || workspace_bytes < ws.bytes || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
-        return SBW_ERR_WORKSPACE;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-
-    const int esize = dtype == SBW_DTYPE_F32 ? 4 : 2;
-    const bool vector = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && ((ld * esize) % 16 == 0);
-    const int vec = vector ? 16 / esize : 1;
-    const int64_t nslot = (V + vec - 1) / vec;
-    if (B * static_cast<int64_t>(choose_split(B, nslot)) > 0x7fffffffLL) return SBW_ERR_UNSUPPORTED;
-
-    SampleArgs a;
-    a.logits = logits;
-    a.B = B; a.V = V; a.ld = ld;
-    a.nslot = static_cast<uint32_t>(nslot);
-    a.split = choose_split(B, nslot);
-    a.slots_per_chunk = static_cast<uint32_t>((nslot + a.split - 1) / a.split);
-    a.ctx = ctx_tokens;
-    a.W = ctx_width;
-    a.vocab_offset = static_cast<uint32_t>(vocab_offset);
-    a.key = key;
-    a.thr_m1 = threshold_minus_one(gamma);
-    a.delta = dtype == SBW_DTYPE_BF16 ? __bfloat162float(__float2bfloat16_rn(delta)) : delta;
-    a.inv_tau = 1.0f / temperature;
-    a.c2_hi = c2_hi;
-    a.c2_lo = static_cast<float>(c2 - static_cast<double>(c2_hi));
-    a.tau = static_cast<double>(temperature);
-    a.gkeys = make_block_keys(static_cast<uint32_t>(rng_seed), static_cast<uint32_t>(rng_seed >> 32));
-    a.weyl = make_weyl();
-    a.step_lo = static_cast<uint32_t>(rng_step);
-    a.step_hi = static_cast<uint32_t>(rng_step >> 32);
-    a.out_tokens = out_tokens;
-    a.out_max = out_max;
-    a.out_sumexp = out_sumexp;
-    a.out_prob = out_prob;
-    a.partials = ws.partials;
-    a.tickets = ws.tickets;
-    a.rowstats = ws.rowstats;
-
-    if (a.split > 1)
-        SBW_CUDA_TRY(cudaMemsetAsync(ws.tickets, 0, static_cast<size_t>(B) * sizeof(unsigned), s));
-    if (dtype == SBW_DTYPE_F32) {
-        return scheme == SBW_SCHEME_CONTEXT ? launch<SBW_DTYPE_F32, SBW_SCHEME_CONTEXT>(a, vector, out_probs, s)
-                                            : launch<SBW_DTYPE_F32, SBW_SCHEME_SELFSALT>(a, vector, out_probs, s);
-    }
-    return scheme == SBW_SCHEME_CONTEXT ? launch<SBW_DTYPE_BF16, SBW_SCHEME_CONTEXT>(a, vector, out_probs, s)
-                                        : launch<SBW_DTYPE_BF16, SBW_SCHEME_SELFSALT>(a, vector, out_probs, s);
+    return sbw::bias_sample_impl(logits, dtype, B, V, ld, vocab_offset, ctx_tokens, ctx_width, key, gamma,
+                                 delta, scheme, temperature, rng_seed, rng_step, out_tokens, out_max,
+                                 out_sumexp, out_prob, out_probs, workspace, workspace_bytes, true,
+                                 static_cast<cudaStream_t>(stream));
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -543,20 +717,22 @@ extern "C" int sbw_bias_sample_noalloc(const void *logits, int dtype, int64_t B,
                                        float *out_prob, float *out_probs, void *stream) {
     using namespace sbw;
     if (B > SBW_NOALLOC_MAX_ROWS) return SBW_ERR_TOO_LARGE;
-    static_assert(sizeof(double2) * SBW_NOALLOC_MAX_ROWS + sizeof(unsigned) * SBW_NOALLOC_MAX_ROWS +
-                          sizeof(Partial) * (SBW_NOALLOC_MAX_ROWS + kTargetCtas) + 3 * 256 <=
+    static_assert(sizeof(double2) * SBW_NOALLOC_MAX_ROWS + 2 * sizeof(unsigned) * SBW_NOALLOC_MAX_ROWS +
+                          sizeof(Partial) * SBW_NOALLOC_MAX_ROWS + 3 * 256 <=
                       kNoallocScratchBytes,
                   "the built-in scratch must hold the workspace of SBW_NOALLOC_MAX_ROWS rows");
-    if (B > 0 && V > 0 && sbw_sample_workspace_bytes(B, V) > kNoallocScratchBytes) return SBW_ERR_TOO_LARGE;
+    if (B > 0 && workspace_min_bytes(B) > kNoallocScratchBytes) return SBW_ERR_TOO_LARGE;
     void *scratch = nullptr;
     if (B > 0) {
         const int rc = noalloc_scratch_address(&scratch);
         if (rc != SBW_OK) return rc;
     }
     // The shared array keeps whatever the previous call left in it.  The only part that must
-    // start at zero is the per-row ticket counters, and sbw_bias_sample clears those on the
+    // start at zero is the per-row ticket counters, and the launch code clears those on the
     // stream before every launch that uses them; everything else is written before it is read.
-    return sbw_bias_sample(logits, dtype, B, V, ld, vocab_offset, ctx_tokens, ctx_width, key, gamma, delta,
-                           scheme, temperature, rng_seed, rng_step, out_tokens, out_max, out_sumexp,
-                           out_prob, out_probs, scratch, kNoallocScratchBytes, stream);
+    // Rows are split into as many chunks as the fixed array has room for.
+    return bias_sample_impl(logits, dtype, B, V, ld, vocab_offset, ctx_tokens, ctx_width, key, gamma, delta,
+                            scheme, temperature, rng_seed, rng_step, out_tokens, out_max, out_sumexp,
+                            out_prob, out_probs, scratch, kNoallocScratchBytes, false,
+                            static_cast<cudaStream_t>(stream));
 }
