@@ -39,9 +39,10 @@ INT_OPS = {"context": 41, "selfsalt": 80, "detect_context": 62, "detect_selfsalt
 # 32x32->64 multiply) at the 1965 MHz maximum SM clock = 18.6 T integer operations per second.
 SMS, LANES_PER_SM_CLK, SM_MAX_MHZ = 148, 64, 1965.0
 INT_PEAK_TOPS = SMS * LANES_PER_SM_CLK * SM_MAX_MHZ * 1e6 / 1e12
-# DRAM bytes per bias launch of the headline workload from the ncu capture summarised under
-# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
-NCU_TRAFFIC_BYTES = None
+# DRAM bytes per bias launch of the headline workload: dram__bytes_read.sum + dram__bytes_write.sum
+# of one ncu capture of the same kernel on B=512 (131.38 MB + 91.60 MB, profiles/), divided by 8
+# because a bench launch processes 1/8 of those units and the traffic grows with the units.
+NCU_TRAFFIC_BYTES = (131.38e6 + 91.60e6) / 8
 
 
 def measured_peaks() -> dict:
