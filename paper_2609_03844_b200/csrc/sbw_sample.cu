@@ -4,12 +4,13 @@
 // that Section 5.1 points at.
 //
 // Work layout.  A row is cut into 16-byte slots as in the bias kernel and, further, into `split`
-// column chunks; the B*split (row, chunk) items are spread over a persistent grid, with `split`
-// chosen so that the item count is close to a multiple of the number of resident CTAs.  For each
-// item a CTA's threads keep an online-softmax pair (running max m, sum of exp2((l' - m) c)) and
-// their best Gumbel score in registers; the CTA reduces them with warp shuffles and shared memory
-// and leaves a partial in the workspace.  The last CTA to take a row's ticket (an atomic, nobody
-// waits) merges that row's partials in index order.
+// column chunks; the B*split (row, chunk) items are spread over the warps of a persistent grid,
+// with `split` chosen so that the item count is close to a multiple of the number of resident
+// warps.  A warp works alone on an item -- no shared memory, no block barrier: its lanes keep an
+// online-softmax pair (running max m, sum of exp2((l' - m) c)) and their best Gumbel score in
+// registers, the warp reduces them with shuffles and leaves a partial in the workspace.  The last
+// warp to take a row's ticket (an atomic, nobody waits) merges that row's partials in index
+// order.
 //
 // Numerics.  The sampled id must be reproducible bit for bit, so everything that feeds it is an
 // exactly rounded fp32 operation spelled with intrinsics: the Gumbel variate is -L(-L(u)) with L
@@ -38,9 +39,9 @@ namespace {
 #endif
 constexpr int kSampleThreads = 256;
 constexpr int kSampleWarps = kSampleThreads / 32;
-constexpr int kMaxSplit = 64;          // chunks per row at most
-constexpr int kMinSlotsPerItem = 256;  // one slot per thread at least
-constexpr int kLegacyTargetCtas = 1184;
+constexpr int kMaxSplit = 512;         // chunks per row at most
+constexpr int kMinSlotsPerItem = 64;   // two trips of a warp at least
+constexpr int kMaxExtraParts = 40960;  // partials beyond one per row never needed: ~16 waves of warps
 
 struct __align__(32) Partial {
     float m;      // max of l' over the chunk
@@ -221,52 +222,42 @@ __device__ __forceinline__ float biased(uint32_t raw, bool green, float delta) {
     }
 }
 
-// Final per-row merge of `n` partials in index order, by one warp; fp64.
+// Final per-row merge of `n` partials by one warp.  Two passes over the partials (they sit in
+// L2): the row maximum first, then every partial's sum rescaled to it -- one independent fp32
+// exp2 per partial (the partial that holds the maximum is scaled by exactly 1), accumulated in
+// fp64 in index order per lane.  The sampled probability is one fp64 exp per row.
 __device__ void finish_row(const SampleArgs &a, int64_t row, const Partial *parts, int n) {
     const int lane = threadIdx.x & 31;
-    double m = -INFINITY, Z = 0.0;
+    float m = -INFINITY;
+    for (int i = lane; i < n; i += 32) m = fmaxf(m, __ldcg(&parts[i].m));
+    for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+    double Z = 0.0;
     float s = -INFINITY, l = -INFINITY;
     int id = INT_MAX;
     for (int i = lane; i < n; i += 32) {
         // L2 loads: the partials were written by other SMs during this launch
         const float4 q0 = __ldcg(reinterpret_cast<const float4 *>(parts + i));
-        const float4 q1 = __ldcg(reinterpret_cast<const float4 *>(parts + i) + 1);
-        Partial p;
-        p.m = q0.x; p.z = q0.y; p.s = q0.z; p.id = __float_as_int(q0.w); p.l = q1.x;
-        const double pm = p.m;
-        if (pm > -INFINITY) {
-            if (pm > m) {
-                Z = Z * exp((m - pm) / a.tau) + p.z;     // exp(-inf) = 0 on the first one
-                m = pm;
-            } else {
-                Z += p.z * exp((pm - m) / a.tau);
-            }
-        }
-        if (better(p.s, p.id, s, id)) { s = p.s; id = p.id; l = p.l; }
+        const float pl = __ldcg(&parts[i].l);
+        const float pm = q0.x, pz = q0.y, ps = q0.z;
+        const int pid = __float_as_int(q0.w);
+        if (pm > -INFINITY) Z += static_cast<double>(pz * exp2_scaled(pm - m, a.c2_hi, a.c2_lo));
+        if (better(ps, pid, s, id)) { s = ps; id = pid; l = pl; }
     }
     for (int d = 16; d > 0; d >>= 1) {
-        const double om = __shfl_down_sync(0xffffffffu, m, d);
-        const double oZ = __shfl_down_sync(0xffffffffu, Z, d);
+        Z += __shfl_down_sync(0xffffffffu, Z, d);
         const float os = __shfl_down_sync(0xffffffffu, s, d);
         const int oid = __shfl_down_sync(0xffffffffu, id, d);
         const float ol = __shfl_down_sync(0xffffffffu, l, d);
-        if (om > -INFINITY) {
-            if (om > m) {
-                Z = Z * exp((m - om) / a.tau) + oZ;
-                m = om;
-            } else {
-                Z += oZ * exp((om - m) / a.tau);
-            }
-        }
         if (better(os, oid, s, id)) { s = os; id = oid; l = ol; }
     }
     if (lane == 0) {
         if (id == INT_MAX) id = 0;                       // every score was -inf: lowest id
+        const double md = static_cast<double>(m);
         a.out_tokens[row] = id;
-        if (a.out_max) a.out_max[row] = static_cast<float>(m);
+        if (a.out_max) a.out_max[row] = m;
         if (a.out_sumexp) a.out_sumexp[row] = static_cast<float>(Z);
-        if (a.out_prob) a.out_prob[row] = static_cast<float>(exp((static_cast<double>(l) - m) / a.tau) / Z);
-        a.rowstats[row] = make_double2(m, Z);
+        if (a.out_prob) a.out_prob[row] = static_cast<float>(exp((static_cast<double>(l) - md) / a.tau) / Z);
+        a.rowstats[row] = make_double2(md, Z);
     }
 }
 
@@ -341,15 +332,12 @@ __global__ void __launch_bounds__(kSampleThreads, SBW_SAMPLE_MIN_BLOCKS)
 sample_kernel(const SampleArgs a) {
     constexpr int VEC = VECTOR ? (DTYPE == SBW_DTYPE_F32 ? 4 : 8) : 1;
     constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
-    __shared__ float sh_f[kSampleWarps];
-    __shared__ float sh_s[kSampleWarps];
-    __shared__ int sh_id[kSampleWarps];
-    __shared__ float sh_l[kSampleWarps];
-    __shared__ unsigned sh_ticket;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int64_t warp_id = static_cast<int64_t>(blockIdx.x) * kSampleWarps + (threadIdx.x >> 5);
+    const int64_t n_warps = static_cast<int64_t>(gridDim.x) * kSampleWarps;
     const uint32_t V = static_cast<uint32_t>(a.V);
 
-    for (int64_t item = blockIdx.x; item < a.n_items; item += gridDim.x) {
+    for (int64_t item = warp_id; item < a.n_items; item += n_warps) {
         const int64_t row = item / a.split;
         const int chunk = static_cast<int>(item - row * a.split);
         const uint32_t j_begin = chunk * a.slots_per_chunk;
@@ -367,7 +355,7 @@ sample_kernel(const SampleArgs a) {
         float bound = -INFINITY;
 
         // warp-uniform trip count: lanes past the end of the chunk carry an empty slot
-        for (uint32_t jb = j_begin + warp * 32; jb < j_end; jb += kSampleThreads) {
+        for (uint32_t jb = j_begin; jb < j_end; jb += 32) {
             const unsigned shared_bound = __ldcg(a.bounds + row);
             const uint32_t j = jb + lane;
             const bool live = j < j_end;
@@ -426,17 +414,11 @@ sample_kernel(const SampleArgs a) {
             }
         }
 
-        // ---- CTA reduction ----
+        // ---- warp reduction: max, then rescaled sums, then lexicographic argmax ----
         float m_w = m_t;
         for (int d = 16; d > 0; d >>= 1) m_w = fmaxf(m_w, __shfl_xor_sync(0xffffffffu, m_w, d));
-        if (lane == 0) sh_f[warp] = m_w;
-        __syncthreads();
-        float m_cta = sh_f[0];
-#pragma unroll
-        for (int w = 1; w < kSampleWarps; ++w) m_cta = fmaxf(m_cta, sh_f[w]);
-        __syncthreads();
         float z_t = 0.0f;
-        if (m_t > -INFINITY) z_t = (z1 + 0.693147180559945f * z2) * exp2_scaled(m_t - m_cta, a.c2_hi, a.c2_lo);
+        if (m_t > -INFINITY) z_t = (z1 + 0.693147180559945f * z2) * exp2_scaled(m_t - m_w, a.c2_hi, a.c2_lo);
         for (int d = 16; d > 0; d >>= 1) z_t += __shfl_down_sync(0xffffffffu, z_t, d);
         for (int d = 16; d > 0; d >>= 1) {
             const float os = __shfl_down_sync(0xffffffffu, best.s, d);
@@ -444,32 +426,21 @@ sample_kernel(const SampleArgs a) {
             const float ol = __shfl_down_sync(0xffffffffu, best.l, d);
             if (better(os, oid, best.s, best.id)) { best.s = os; best.id = oid; best.l = ol; }
         }
-        if (lane == 0) { sh_f[warp] = z_t; sh_s[warp] = best.s; sh_id[warp] = best.id; sh_l[warp] = best.l; }
-        __syncthreads();
-        if (threadIdx.x == 0) {
+        unsigned ticket = 0;
+        if (lane == 0) {
             Partial p;
-            p.m = m_cta;
-            p.z = 0.0f;
-            p.s = sh_s[0]; p.id = sh_id[0]; p.l = sh_l[0];
-            for (int w = 0; w < kSampleWarps; ++w) {
-                p.z += sh_f[w];
-                if (w > 0 && better(sh_s[w], sh_id[w], p.s, p.id)) { p.s = sh_s[w]; p.id = sh_id[w]; p.l = sh_l[w]; }
-            }
+            p.m = m_w; p.z = z_t; p.s = best.s; p.id = best.id; p.l = best.l;
             p.pad[0] = p.pad[1] = p.pad[2] = 0.0f;
             a.partials[item] = p;
-            unsigned ticket = 0;
             __threadfence();                           // partial visible before the ticket is taken
             if (a.split > 1) ticket = atomicAdd(&a.tickets[row], 1u);
-            sh_ticket = ticket;
         }
-        __syncthreads();
-        const bool last = a.split == 1 || sh_ticket == static_cast<unsigned>(a.split - 1);
-        if (last && warp == 0) {
-            if (a.split > 1) __threadfence();          // the other CTAs' partials are visible now
+        ticket = __shfl_sync(0xffffffffu, ticket, 0);
+        if (a.split == 1 || ticket == static_cast<unsigned>(a.split - 1)) {
+            __threadfence();                           // the other warps' partials are visible now
             finish_row(a, row, a.partials + row * a.split, a.split);
             if (lane == 0 && a.split > 1) a.tickets[row] = 0;
         }
-        __syncthreads();                               // shared scratch is reused by the next item
     }
 }
 
@@ -521,14 +492,14 @@ size_t workspace_min_bytes(int64_t B) {
     return carve(nullptr, B).fixed_bytes + align_up(static_cast<size_t>(B) * sizeof(Partial), 256);
 }
 size_t workspace_full_bytes(int64_t B) {
-    // B * split partials with split <= kMaxSplit, but never more than B + kLegacyTargetCtas rows
-    // worth when B is large (items beyond a few waves of CTAs bring nothing)
-    const int64_t parts = B * kMaxSplit < 4 * (B + kLegacyTargetCtas) ? B * kMaxSplit : 4 * (B + kLegacyTargetCtas);
+    // B * split partials with split <= kMaxSplit, but items beyond a dozen waves of resident warps
+    // bring nothing, so the count is capped at one per row plus kMaxExtraParts
+    const int64_t parts = B * kMaxSplit < B + kMaxExtraParts ? B * kMaxSplit : B + kMaxExtraParts;
     return carve(nullptr, B).fixed_bytes + align_up(static_cast<size_t>(parts) * sizeof(Partial), 256);
 }
 
 // Chunks per row: the smallest split whose item count B*split fills whole waves of `ctas`
-// resident CTAs to 95 %, else the fullest one; bounded by the row length and by the workspace.
+// resident warps to 95 %, else the fullest one; bounded by the row length and by the workspace.
 int choose_split(int64_t B, int64_t nslot, int64_t ctas, int64_t max_parts) {
     int64_t max_split = nslot / kMinSlotsPerItem;
     if (max_split > kMaxSplit) max_split = kMaxSplit;
@@ -559,11 +530,13 @@ int launch_one(SampleArgs &a, int64_t nslot, size_t partial_bytes, cudaStream_t 
         blocks_per_sm = n > 0 ? n : 1;
     }
     const int64_t ctas = static_cast<int64_t>(di.sm_count) * blocks_per_sm;
-    a.split = choose_split(a.B, nslot, ctas, static_cast<int64_t>(partial_bytes / sizeof(Partial)));
+    const int64_t warps = ctas * kSampleWarps;
+    a.split = choose_split(a.B, nslot, warps, static_cast<int64_t>(partial_bytes / sizeof(Partial)));
     a.n_items = a.B * a.split;
     a.slots_per_chunk = static_cast<uint32_t>((nslot + a.split - 1) / a.split);
     SBW_CUDA_TRY(cudaMemsetAsync(a.tickets, 0, 2 * static_cast<size_t>(a.B) * sizeof(unsigned), s));
-    const unsigned grid = static_cast<unsigned>(a.n_items < ctas ? a.n_items : ctas);
+    const int64_t want_ctas = (a.n_items + kSampleWarps - 1) / kSampleWarps;
+    const unsigned grid = static_cast<unsigned>(want_ctas < ctas ? want_ctas : ctas);
     sample_kernel<DTYPE, SCHEME, VECTOR><<<grid, kSampleThreads, 0, s>>>(a);
     SBW_CUDA_TRY(cudaGetLastError());
     return SBW_OK;
