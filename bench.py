@@ -160,7 +160,7 @@ def run_reference(args) -> None:
             "n_gpus": 0, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": workload_config(),
+            "config": {**workload_config(), "l2": f"{n_in} host-resident step inputs visited in turn (CPU run)"},
             "cpu_baseline": {"value": value, "unit": "Gelem/s", "cores": cores, "kind": "oracle",
                              "sample": f"{args.steps} full decode steps of the headline workload"},
             "e2e": {"value": value, "unit": "Gelem/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -323,6 +323,7 @@ def run_ours(args) -> None:
         del logits, ctxs
         torch.cuda.empty_cache()
         line["extra"] = run_extra(sbw, inputs, dev, peaks)
+        line["detect_tokens_per_s"] = line["extra"]["detect_context_N100000"]["tokens_per_s"]
         line["cpu_baseline"] = cpu_baseline()
     if rank == 0:
         print(json.dumps(line))
@@ -426,6 +427,28 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
             s = _time_calls(lambda i: sbw.sbw_bias_sample(x, c, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, wsb), 20)
             out[f"sample_bf16_{name}_B{B}"] = {"gelem_s": B * V2 / s / 1e9, "ms": s * 1e3,
                                                "l2_resident": B * V2 * 2 < 100e6}
+    # the paper's isolated-benchmark protocol (Appendix B: fresh (B, 151936) logits, 20 warm-up + 200
+    # timed calls, CUDA events, synchronise between calls, p50/p99) on its two full-vocabulary schemes
+    # with context width 4 (SBW-4, SBW-ss-V); fp32 logits (the paper does not state its dtype)
+    sweep = {}
+    for B in (1, 16, 64, 256, 512):
+        x = inputs.logits_normal(B, 151936, 4.0, torch.float32, seed=800 + B, device=dev)
+        c = inputs.uniform_tokens((B, 4), 151936, seed=900 + B, device=dev)
+        for name, scheme in (("sbw4", sbw.SCHEME_CONTEXT), ("sbw_ss_v", sbw.SCHEME_SELFSALT)):
+            times = []
+            for i in range(220):
+                e0 = torch.cuda.Event(enable_timing=True)
+                e1 = torch.cuda.Event(enable_timing=True)
+                e0.record()
+                sbw.sbw_bias_logits(x, c, KEY, 0.25, 2.0, scheme)
+                e1.record()
+                torch.cuda.synchronize()
+                if i >= 20:
+                    times.append(e0.elapsed_time(e1))
+            times.sort()
+            sweep[f"{name}_B{B}"] = {"p50_ms": times[len(times) // 2], "p99_ms": times[int(len(times) * 0.99)],
+                                     "l2_resident": B * 151936 * 4 < 100e6}
+    out["paper_protocol_latency_fp32_V151936_W4"] = sweep
     # integer-throughput probe
     probes = {}
     for kind in ("mulwide", "lop3", "iadd3", "imad", "philox", "ffma"):
