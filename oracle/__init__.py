@@ -74,6 +74,9 @@ def lib() -> ctypes.CDLL:
         L.sbw_oracle_bias_logits.restype = None
         L.sbw_oracle_bias_logits.argtypes = [vp, i32, i64, i64, i64, i64, vp, i32, u64, c.c_double,
                                              c.c_float, i32, i32]
+        L.sbw_oracle_bias_logits_topk.restype = None
+        L.sbw_oracle_bias_logits_topk.argtypes = [vp, i32, i64, i64, i64, i64, vp, i32, u64, c.c_double,
+                                                  c.c_float, i32, i64, vp]
         L.sbw_oracle_detect.restype = None
         L.sbw_oracle_detect.argtypes = [vp, vp, i64, i32, u64, c.c_double, i32, vp, vp, vp, i32]
         L.sbw_oracle_zscore.restype = c.c_double
@@ -156,6 +159,20 @@ def bias_logits(logits: np.ndarray, V, ctx_tokens, key, gamma, delta, scheme,
     lib().sbw_oracle_bias_logits(_ptr(out), dtype, B, V, ld, vocab_offset, _ptr(ctx), W, key,
                                  gamma, delta, scheme, threads)
     return out
+
+
+def bias_logits_topk(logits: np.ndarray, V, ctx_tokens, key, gamma, delta, scheme, top_k,
+                     vocab_offset=0):
+    """Top-k restricted bias (SBW-ss) on a copy of ``logits``; returns (biased, chosen columns)."""
+    assert logits.ndim == 2 and logits.dtype in (np.float32, np.uint16)
+    out = np.ascontiguousarray(logits).copy()
+    B, ld = out.shape
+    ctx, W = _ctx(ctx_tokens, B)
+    dtype = DTYPE_F32 if out.dtype == np.float32 else DTYPE_BF16
+    sel = np.zeros((B, min(top_k, V)), dtype=np.int32)
+    lib().sbw_oracle_bias_logits_topk(_ptr(out), dtype, B, V, ld, vocab_offset, _ptr(ctx), W, key,
+                                      gamma, delta, scheme, top_k, _ptr(sel))
+    return out, sel
 
 
 def detect(tokens, lengths, key, gamma, scheme, ctx_width=1, threads=1):

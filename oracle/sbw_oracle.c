@@ -27,6 +27,9 @@
  *      +0 would turn -0 into +0).
  *  R7  Detection scores positions t = W .. L-1 (the first W tokens only seed), T = max(L-W,0),
  *      every position counted (no repeated-n-gram filter); T = 0 gives G = 0, z = 0.
+ *  R9  SBW-ss (Table 1: self-salt, candidates "top-40"): per row only the k largest logits are
+ *      tested and biased; "largest" is the total order on order-encoded bit patterns with ties
+ *      to the lowest column (the paper inherits KGW's top-k and states no tie rule).
  *  R8  The fused sampler is this library's own (the paper leaves sampling to the engine):
  *      bias first, then temperature; Gumbel-max with a Philox stream of its own and a
  *      fully specified fp32 logarithm so that sampled ids are reproducible bit for bit.
@@ -209,6 +212,70 @@ void sbw_oracle_bias_logits(void *logits, int dtype, int64_t B, int64_t V, int64
     for (int64_t b = 0; b < B; ++b)
         bias_row(logits, dtype, b, V, ld, vocab_offset, ctx_tokens + b * ctx_width, ctx_width,
                  key, thr, delta, scheme);
+}
+
+/* ------------------------------------------------------------------ top-k (SBW-ss) - */
+/* Order-preserving code of a logit's bit pattern: larger float, larger code; every pattern
+ * (both zeros, infinities, NaNs) gets its own code, so the order is total. */
+static uint32_t order_code(uint32_t bits32)
+{
+    return (bits32 & 0x80000000u) ? ~bits32 : (bits32 | 0x80000000u);
+}
+
+typedef struct {
+    uint32_t code;
+    int64_t col;
+} ranked_t;
+
+static int ranked_cmp(const void *pa, const void *pb)
+{
+    const ranked_t *a = (const ranked_t *)pa, *b = (const ranked_t *)pb;
+    if (a->code != b->code)
+        return a->code > b->code ? -1 : 1;        /* larger logit first */
+    return a->col < b->col ? -1 : (a->col > b->col ? 1 : 0);   /* ties: lowest column first */
+}
+
+void sbw_oracle_bias_logits_topk(void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
+                                 int64_t vocab_offset, const int32_t *ctx_tokens, int ctx_width,
+                                 uint64_t key, double gamma, float delta, int scheme, int64_t top_k,
+                                 int32_t *sel)
+{
+    uint64_t thr = sbw_oracle_threshold(gamma);
+    int64_t k = top_k < V ? top_k : V;
+    ranked_t *order = (ranked_t *)malloc((size_t)V * sizeof(ranked_t));
+    if (!order)
+        return;
+    for (int64_t b = 0; b < B; ++b) {
+        const int32_t *ctx = ctx_tokens + b * ctx_width;
+        for (int64_t j = 0; j < V; ++j) {
+            uint32_t bits;
+            if (dtype == SBW_O_DTYPE_BF16) {
+                bits = (uint32_t)((const uint16_t *)logits)[b * ld + j] << 16;
+            } else {
+                float f = ((const float *)logits)[b * ld + j];
+                memcpy(&bits, &f, sizeof bits);
+            }
+            order[j].code = order_code(bits);
+            order[j].col = j;
+        }
+        qsort(order, (size_t)V, sizeof(ranked_t), ranked_cmp);
+        for (int64_t i = 0; i < k; ++i) {
+            int64_t j = order[i].col;
+            if (sel)
+                sel[b * k + i] = (int32_t)j;
+            uint32_t v = (uint32_t)(vocab_offset + j);
+            uint64_t r = seed_for(scheme, key, ctx, ctx_width, v);
+            int g = sbw_oracle_green(r, v, thr);
+            if (dtype == SBW_O_DTYPE_BF16) {
+                uint16_t *p = (uint16_t *)logits + b * ld + j;
+                *p = sbw_oracle_bias_elem_bf16(*p, delta, g);
+            } else {
+                float *p = (float *)logits + b * ld + j;
+                *p = sbw_oracle_bias_elem_f32(*p, delta, g);
+            }
+        }
+    }
+    free(order);
 }
 
 /* ------------------------------------------------------------------ Eq. 5 ---------- */

@@ -16,6 +16,7 @@
  *   seeds, green       pinned: big-integer restatement, Binomial(V,gamma)   (test_oracle_hash,
  *                      green-list statistics of Appendix H                   test_oracle_stats)
  *   bias add           pinned: numpy float32 / torch bfloat16 adds           (test_oracle_bias)
+ *   top-k restriction  pinned: torch.topk, brute force on ties, k >= V case  (test_oracle_topk)
  *   detect             pinned: brute force, closed forms, null law of Eq. 5  (test_oracle_detect)
  *   log / gumbel /     pinned: fp64 log, chi-square of sampled ids against    (test_oracle_sample)
  *   sample             softmax, scipy softmax / logsumexp, closed form
@@ -71,6 +72,17 @@ uint16_t sbw_oracle_bias_elem_bf16(uint16_t l, float delta, int green);
 void sbw_oracle_bias_logits(void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
                             int64_t vocab_offset, const int32_t *ctx_tokens, int ctx_width,
                             uint64_t key, double gamma, float delta, int scheme, int threads);
+
+/* Top-k candidate restriction (the paper's SBW-ss scheme, Table 1: self-salt on the top-40
+ * candidates only, as KGW's selfhash does).  Per row the k candidates are the k largest logits in
+ * the total order "bit pattern order-encoded descending, then column ascending" (so ties go to the
+ * lowest ids and every bit pattern, NaN included, has a place); only they are tested and biased.
+ * k >= V biases like sbw_oracle_bias_logits.  sel (nullable) receives the chosen columns, [B, min(k,V)],
+ * in rank order. */
+void sbw_oracle_bias_logits_topk(void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
+                                 int64_t vocab_offset, const int32_t *ctx_tokens, int ctx_width,
+                                 uint64_t key, double gamma, float delta, int scheme, int64_t top_k,
+                                 int32_t *sel);
 
 /* Eq. 5 and the O(1)-per-token membership test of Section 2.2.
  * tokens: concatenation of N sequences; lengths[N].  Writes counts[N], T[N] (nullable), z[N]. */
