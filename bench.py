@@ -397,6 +397,12 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
         n = B3 * V3
         out[f"bias_fp32_{name}_B256_V151936"] = {"gelem_s": n / s / 1e9, "ms": s * 1e3,
                                                  **place(INT_OPS[name] * n, 8 * n, s)}
+    # the paper's SBW-ss: self-salt on the top-40 candidates of each row only (same shape)
+    s = _time_calls(lambda i: sbw.sbw_bias_logits_topk(p3[i % 4], c3[i % 4], KEY, 0.25, 4.0, sbw.SCHEME_SELFSALT, 40), 128)
+    out["bias_top40_fp32_selfsalt_B256_V151936"] = {
+        "gelem_s": B3 * V3 / s / 1e9, "ms": s * 1e3, "bound": "hbm",
+        "achieved_gbs": 4 * B3 * V3 / s / 1e9, "frac": 4 * B3 * V3 / s / 1e9 / hbm,
+        "note": "one read of the row from HBM (4 B/logit), second read from L2, 40 columns written"}
     del p3, c3
     # config 2 shape under the self-salt scheme
     p2 = [inputs.logits_normal(B2, V2, 4.0, torch.bfloat16, seed=400 + i, device=dev) for i in range(16)]

@@ -85,6 +85,20 @@ int sbw_bias_logits(void *logits, int dtype, int64_t B, int64_t V, int64_t ld, i
                     float delta, int scheme, void *stream);
 
 /*
+ * sbw_bias_logits_topk -- the paper's SBW-ss scheme (Table 1: Bernoulli list, self-salt, candidates
+ * "top-40"; Section 5.2 describes the top-k restriction it inherits from KGW): per row only the
+ * top_k largest logits are tested (Eq. 1) and biased (Eq. 2); every other element of the row
+ * keeps its bits.  "Largest" is the total order on order-encoded bit patterns -- +NaN > +inf >
+ * ... > +0 > -0 > ... > -inf > -NaN -- with ties to the lowest column (the paper states no tie
+ * rule).  Arguments as for sbw_bias_logits; top_k >= 1; top_k >= V is the full-vocabulary call.
+ * Needs no workspace.  Fast for ordinary rows and top_k <= 256; rows of mostly equal values or
+ * larger top_k take a slow, exact fallback (top_k block reductions per row).
+ */
+int sbw_bias_logits_topk(void *logits, int dtype, int64_t B, int64_t V, int64_t ld, int64_t vocab_offset,
+                         const int32_t *ctx_tokens, int ctx_width, uint64_t key, double gamma,
+                         float delta, int scheme, int64_t top_k, void *stream);
+
+/*
  * sbw_bias_logits_host -- the same step for callers whose logits live in HOST memory: copies
  * B*ld elements and the context tokens to the device staging buffer, runs sbw_bias_logits on
  * it, and copies the logits back, all enqueued on `stream` (the copies are asynchronous only if

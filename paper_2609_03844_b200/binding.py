@@ -28,7 +28,7 @@ DTYPE_BF16 = 1
 EXPORTS = ("sbw_version", "sbw_last_cuda_error", "sbw_bias_logits",
            "sbw_bias_logits_host_staging_bytes", "sbw_bias_logits_host",
            "sbw_sample_workspace_bytes", "sbw_bias_sample", "sbw_detect_workspace_bytes",
-           "sbw_detect", "sbw_int_probe", "sbw_bias_sample_noalloc")
+           "sbw_detect", "sbw_int_probe", "sbw_bias_sample_noalloc", "sbw_bias_logits_topk")
 
 _lib = None
 
@@ -65,6 +65,9 @@ def lib() -> ctypes.CDLL:
         L.sbw_bias_logits.restype = i32
         L.sbw_bias_logits.argtypes = [vp, i32, i64, i64, i64, i64, vp, i32, u64, c.c_double,
                                       c.c_float, i32, vp]
+        L.sbw_bias_logits_topk.restype = i32
+        L.sbw_bias_logits_topk.argtypes = [vp, i32, i64, i64, i64, i64, vp, i32, u64, c.c_double,
+                                           c.c_float, i32, i64, vp]
         L.sbw_bias_logits_host_staging_bytes.restype = sz
         L.sbw_bias_logits_host_staging_bytes.argtypes = [i32, i64, i64, i32]
         L.sbw_bias_logits_host.restype = i32
@@ -147,6 +150,21 @@ def sbw_bias_logits(logits: torch.Tensor, ctx_tokens: torch.Tensor, key: int, ga
     rc = lib().sbw_bias_logits(_ptr(logits), _dtype_code(logits), B, V, ld, vocab_offset,
                                _ptr(ctx_tokens), W, key, gamma, delta, scheme, _stream(stream))
     _check("sbw_bias_logits", rc)
+    return logits
+
+
+def sbw_bias_logits_topk(logits: torch.Tensor, ctx_tokens: torch.Tensor, key: int, gamma: float,
+                         delta: float, scheme: int, top_k: int = 40, *, V: int | None = None,
+                         vocab_offset: int = 0, stream=None) -> torch.Tensor:
+    """In-place bias of the ``top_k`` largest logits of every row only (the paper's SBW-ss)."""
+    if not logits.is_cuda or not ctx_tokens.is_cuda:
+        raise ValueError("sbw_bias_logits_topk takes CUDA tensors")
+    B, V, ld = _row_layout(logits, V)
+    W = _ctx(ctx_tokens, B)
+    rc = lib().sbw_bias_logits_topk(_ptr(logits), _dtype_code(logits), B, V, ld, vocab_offset,
+                                    _ptr(ctx_tokens), W, key, gamma, delta, scheme, top_k,
+                                    _stream(stream))
+    _check("sbw_bias_logits_topk", rc)
     return logits
 
 

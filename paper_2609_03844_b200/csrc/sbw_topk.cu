@@ -1,0 +1,268 @@
+// sbw_bias_logits_topk: the paper's SBW-ss scheme (Table 1: Bernoulli list, self-salt seeding,
+// candidates "top-40") -- per row only the k largest logits are tested and biased, as KGW's
+// selfhash does; everything else in the row is left alone.
+//
+// One CTA per row.  "Largest" is the total order on order-encoded bit patterns with ties to the
+// lowest column, expressed as one 64-bit composite (code << 32 | ~column).
+//   1. A pass over a prefix of the row (32 columns per thread): every thread keeps the largest code
+//      it has seen; groups of four threads give 256 maxima of disjoint column sets.  Their k-th
+//      largest value L is a lower bound of the row's k-th largest logit (k distinct columns reach
+//      it), and it is known after a fifth of the row.
+//   2. One pass over the whole row: columns with code >= L -- a few hundred for ordinary logits --
+//      go into a shared-memory candidate list.  The common path is one compare per logit.
+//   3. Candidates are ranked by counting larger composites; ranks below k are hashed and biased.
+// If the list overflows (rows of equal values, k > 256) the CTA falls back to k rounds of "largest
+// composite below the previous one", a block reduction each, and one pass that biases every
+// column at or above the k-th composite: slow, but it needs no assumption about the data.
+#include <cuda_bf16.h>
+
+#include "sbw_common.cuh"
+#include "sbw_hash.cuh"
+
+namespace sbw {
+
+int bias_logits_impl(void *logits, int dtype, int64_t B, int64_t V, int64_t ld, int64_t vocab_offset,
+                     const int32_t *ctx_tokens, int ctx_width, uint64_t key, double gamma, float delta,
+                     int scheme, cudaStream_t stream);
+
+namespace {
+
+#ifndef SBW_TOPK_CTAS_PER_SM
+#define SBW_TOPK_CTAS_PER_SM 1
+#endif
+constexpr int kTopkThreads = 1024;
+constexpr int kTopkWarps = kTopkThreads / 32;
+constexpr int kGroups = kTopkThreads / 4;   // maxima of disjoint column sets used for the lower bound
+constexpr int kCap = 2048;                  // candidate list entries
+constexpr int kPrefixPerThread = 32;        // columns per thread in the pass that finds the bound
+
+struct TopkArgs {
+    void *logits;
+    int64_t B, V, ld;
+    const int32_t *ctx;
+    int W;
+    uint32_t vocab_offset;
+    uint64_t key;
+    uint32_t thr_m1;
+    float delta;       // in the logits' precision, widened
+    Weyl weyl;
+    int k;
+    bool vector;       // rows start on 16-byte boundaries
+};
+
+__device__ __forceinline__ uint32_t order_code(uint32_t bits) {
+    return (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+}
+__device__ __forceinline__ uint64_t composite(uint32_t code, uint32_t col) {
+    return (static_cast<uint64_t>(code) << 32) | (0xFFFFFFFFu - col);
+}
+
+// Calls f(column, code) for the columns of one row that this thread owns.
+template <int DTYPE, typename F>
+__device__ __forceinline__ void for_each_code(const char *row_ptr, uint32_t V, bool vector, F f) {
+    // V here is the number of leading columns to visit (the whole row or a prefix of it)
+    constexpr int VEC = DTYPE == SBW_DTYPE_F32 ? 4 : 8;
+    uint32_t done = 0;
+    if (vector) {
+        const uint32_t nfull = V / VEC;
+        constexpr int kInFlight = 8;   // independent 128-bit loads per thread before the first use
+        for (uint32_t j0 = threadIdx.x; j0 < nfull; j0 += kInFlight * kTopkThreads) {
+            uint4 w[kInFlight];
+#pragma unroll
+            for (int u = 0; u < kInFlight; ++u) {
+                const uint32_t j = j0 + u * kTopkThreads;
+                // plain loads: the row is written later by this kernel
+                w[u] = j < nfull ? reinterpret_cast<const uint4 *>(row_ptr)[j] : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int u = 0; u < kInFlight; ++u) {
+                const uint32_t j = j0 + u * kTopkThreads;
+                if (j >= nfull) break;
+                const uint32_t *e = reinterpret_cast<const uint32_t *>(&w[u]);
+#pragma unroll
+                for (int i = 0; i < VEC; ++i) {
+                    uint32_t bits;
+                    if constexpr (DTYPE == SBW_DTYPE_F32) bits = e[i];
+                    else bits = (i & 1) ? (e[i >> 1] & 0xffff0000u) : (e[i >> 1] << 16);
+                    f(j * VEC + i, order_code(bits));
+                }
+            }
+        }
+        done = nfull * VEC;
+    }
+    for (uint32_t c = done + threadIdx.x; c < V; c += kTopkThreads) {
+        uint32_t bits;
+        if constexpr (DTYPE == SBW_DTYPE_F32) bits = reinterpret_cast<const uint32_t *>(row_ptr)[c];
+        else bits = static_cast<uint32_t>(reinterpret_cast<const uint16_t *>(row_ptr)[c]) << 16;
+        f(c, order_code(bits));
+    }
+}
+
+// Eq. 1 + Eq. 2 on one chosen column.
+template <int DTYPE, int SCHEME>
+__device__ __noinline__ void bias_column(const TopkArgs &a, int64_t row, char *row_ptr, uint32_t col) {
+    const int32_t *ctx = a.ctx + row * a.W;
+    const uint32_t v = a.vocab_offset + col;
+    uint64_t r;
+    if constexpr (SCHEME == SBW_SCHEME_CONTEXT) r = seed_context(a.key, ctx, a.W);
+    else r = seed_selfsalt(a.key, jenkins_min(ctx, a.W), v);
+    if (philox_word0(v, r, a.weyl) > a.thr_m1) return;
+    if constexpr (DTYPE == SBW_DTYPE_F32) {
+        float *p = reinterpret_cast<float *>(row_ptr) + col;
+        *p = __fadd_rn(*p, a.delta);
+    } else {
+        __nv_bfloat16 *p = reinterpret_cast<__nv_bfloat16 *>(row_ptr) + col;
+        *p = __float2bfloat16_rn(__fadd_rn(__bfloat162float(*p), a.delta));
+    }
+}
+
+__device__ __forceinline__ uint64_t block_max_u64(uint64_t x, uint64_t *sh_red, uint64_t *sh_out) {
+    for (int d = 16; d > 0; d >>= 1) {
+        const uint64_t o = __shfl_xor_sync(0xffffffffu, x, d);
+        x = o > x ? o : x;
+    }
+    if ((threadIdx.x & 31) == 0) sh_red[threadIdx.x >> 5] = x;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint64_t m = sh_red[0];
+        for (int w = 1; w < kTopkWarps; ++w) m = sh_red[w] > m ? sh_red[w] : m;
+        *sh_out = m;
+    }
+    __syncthreads();
+    return *sh_out;
+}
+
+template <int DTYPE, int SCHEME>
+__global__ void __launch_bounds__(kTopkThreads)
+topk_kernel(const TopkArgs a) {
+    constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
+    __shared__ uint32_t sh_max[kGroups];
+    __shared__ uint64_t sh_cand[kCap];
+    __shared__ uint64_t sh_red[kTopkWarps];
+    __shared__ uint64_t sh_best;
+    __shared__ uint32_t sh_floor;
+    __shared__ unsigned sh_count;
+    const uint32_t V = static_cast<uint32_t>(a.V);
+    const uint32_t k = static_cast<uint32_t>(a.k);
+
+    for (int64_t row = blockIdx.x; row < a.B; row += gridDim.x) {
+        char *row_ptr = static_cast<char *>(a.logits) + row * a.ld * ESIZE;
+
+        // 1. lower bound of the k-th largest code from a prefix of the row
+        const uint32_t prefix = min(V, static_cast<uint32_t>(kPrefixPerThread * kTopkThreads));
+        uint32_t mx = 0;
+        for_each_code<DTYPE>(row_ptr, prefix, a.vector, [&](uint32_t, uint32_t code) { mx = max(mx, code); });
+        mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        if ((threadIdx.x & 3) == 0) sh_max[threadIdx.x >> 2] = mx;
+        if (threadIdx.x == 0) {
+            sh_floor = 0;            // k > kGroups: no bound, everything is a candidate
+            sh_count = 0;
+        }
+        __syncthreads();
+        if (k <= kGroups && threadIdx.x < kGroups) {
+            const uint32_t mine = sh_max[threadIdx.x];
+            uint32_t rank = 0;
+            for (int u = 0; u < kGroups; ++u) {
+                const uint32_t o = sh_max[u];
+                rank += (o > mine || (o == mine && u < static_cast<int>(threadIdx.x))) ? 1u : 0u;
+            }
+            if (rank == k - 1) sh_floor = mine;
+        }
+        __syncthreads();
+        const uint32_t floor_code = sh_floor;
+
+        // 2. candidates: every column of the row that reaches the bound
+        for_each_code<DTYPE>(row_ptr, V, a.vector, [&](uint32_t col, uint32_t code) {
+            if (code >= floor_code) {
+                const unsigned pos = atomicAdd(&sh_count, 1u);
+                if (pos < kCap) sh_cand[pos] = composite(code, col);
+            }
+        });
+        __syncthreads();
+        const unsigned n = sh_count;
+
+        if (n <= kCap) {
+            // 3. rank by counting, bias ranks below k
+            for (unsigned e = threadIdx.x; e < n; e += kTopkThreads) {
+                const uint64_t mine = sh_cand[e];
+                uint32_t rank = 0;
+                for (unsigned u = 0; u < n; ++u) rank += sh_cand[u] > mine ? 1u : 0u;
+                if (rank < k) bias_column<DTYPE, SCHEME>(a, row, row_ptr, 0xFFFFFFFFu - static_cast<uint32_t>(mine));
+            }
+        } else {
+            // fallback: k rounds of "largest composite below the previous one" find the composite
+            // of the k-th ranked column without touching the row; one more pass then biases every
+            // column at or above it (each column is judged on its own original value).  A real
+            // composite is never 0 (its low word is 2^32 - 1 - column >= 2^31), so 0 means "none".
+            uint64_t prev = 0;
+            const uint32_t rounds = k < V ? k : V;
+            for (uint32_t r = 0; r < rounds; ++r) {
+                uint64_t best = 0;
+                for_each_code<DTYPE>(row_ptr, V, a.vector, [&](uint32_t col, uint32_t code) {
+                    const uint64_t c = composite(code, col);
+                    if ((r == 0 || c < prev) && c > best) best = c;
+                });
+                prev = block_max_u64(best, sh_red, &sh_best);
+            }
+            const uint64_t kth = prev;
+            for_each_code<DTYPE>(row_ptr, V, a.vector, [&](uint32_t col, uint32_t code) {
+                if (composite(code, col) >= kth) bias_column<DTYPE, SCHEME>(a, row, row_ptr, col);
+            });
+        }
+        __syncthreads();             // shared scratch is reused by the next row
+    }
+}
+
+template <int DTYPE, int SCHEME>
+int launch(const TopkArgs &a, cudaStream_t s) {
+    DeviceInfo di;
+    const int rc = current_device_info(&di);
+    if (rc != SBW_OK) return rc;
+    const int64_t cap = static_cast<int64_t>(di.sm_count) * SBW_TOPK_CTAS_PER_SM;
+    const unsigned grid = static_cast<unsigned>(a.B < cap ? a.B : cap);
+    topk_kernel<DTYPE, SCHEME><<<grid, kTopkThreads, 0, s>>>(a);
+    SBW_CUDA_TRY(cudaGetLastError());
+    return SBW_OK;
+}
+
+}  // namespace
+}  // namespace sbw
+
+extern "C" int sbw_bias_logits_topk(void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
+                                    int64_t vocab_offset, const int32_t *ctx_tokens, int ctx_width,
+                                    uint64_t key, double gamma, float delta, int scheme, int64_t top_k,
+                                    void *stream) {
+    using namespace sbw;
+    if (!valid_common(dtype, ctx_width, gamma, scheme)) return SBW_ERR_INVALID_ARG;
+    if (B < 0 || V <= 0 || ld < V || vocab_offset < 0 || top_k < 1) return SBW_ERR_INVALID_ARG;
+    if (V > 0x7fffffffLL || vocab_offset + V > (int64_t(1) << 32)) return SBW_ERR_UNSUPPORTED;
+    if (!(delta == delta) || delta - delta != 0.0f) return SBW_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (top_k >= V)   // every column is a candidate: the full-vocabulary kernel
+        return bias_logits_impl(logits, dtype, B, V, ld, vocab_offset, ctx_tokens, ctx_width, key, gamma,
+                                delta, scheme, s);
+    if (B == 0) return SBW_OK;
+    if (!logits || !ctx_tokens) return SBW_ERR_INVALID_ARG;
+
+    TopkArgs a;
+    a.logits = logits;
+    a.B = B; a.V = V; a.ld = ld;
+    a.ctx = ctx_tokens;
+    a.W = ctx_width;
+    a.vocab_offset = static_cast<uint32_t>(vocab_offset);
+    a.key = key;
+    a.thr_m1 = threshold_minus_one(gamma);
+    a.delta = dtype == SBW_DTYPE_BF16 ? __bfloat162float(__float2bfloat16_rn(delta)) : delta;
+    a.weyl = make_weyl();
+    a.k = static_cast<int>(top_k);
+    const int esize = dtype == SBW_DTYPE_F32 ? 4 : 2;
+    a.vector = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && ((ld * esize) % 16 == 0);
+    if (a.delta == 0.0f) return SBW_OK;   // the paper's delta = 0 control: no bit changes
+
+    if (dtype == SBW_DTYPE_F32)
+        return scheme == SBW_SCHEME_CONTEXT ? launch<SBW_DTYPE_F32, SBW_SCHEME_CONTEXT>(a, s)
+                                            : launch<SBW_DTYPE_F32, SBW_SCHEME_SELFSALT>(a, s);
+    return scheme == SBW_SCHEME_CONTEXT ? launch<SBW_DTYPE_BF16, SBW_SCHEME_CONTEXT>(a, s)
+                                        : launch<SBW_DTYPE_BF16, SBW_SCHEME_SELFSALT>(a, s);
+}

@@ -1,0 +1,92 @@
+"""GPU parity of sbw_bias_logits_topk (the paper's SBW-ss: only the top-k candidates of a row are
+tested and biased) against the CPU oracle: every bit of the row."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_03844_b200 as sbw
+from paper_2609_03844_b200 import inputs
+from gpu_util import KEY, assert_same_bits, host_bits, require_gpu
+
+pytestmark = pytest.mark.gpu
+SCHEMES = [sbw.SCHEME_CONTEXT, sbw.SCHEME_SELFSALT]
+
+
+def _check(x, V, ctx, key, gamma, delta, scheme, k, off=0, view=None):
+    dev = require_gpu()
+    x_dev = x.to(dev)
+    target = x_dev if view is None else view(x_dev)
+    src = x if view is None else view(x).contiguous()
+    sbw.sbw_bias_logits_topk(target, ctx.to(dev), key, gamma, delta, scheme, k, V=V, vocab_offset=off)
+    torch.cuda.synchronize()
+    want, sel = oracle.bias_logits_topk(host_bits(src), V, ctx.numpy(), key, gamma, delta, scheme, k,
+                                        vocab_offset=off)
+    got = host_bits(target.contiguous()) if view is not None else host_bits(x_dev)
+    assert_same_bits(got, want)
+    return got, sel
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("scheme", SCHEMES)
+def test_top40_on_full_vocabulary_rows(dtype, scheme):
+    """V=151936 (fp32) / 128256 (bf16, many tied values near the top), context width 4, k = 40."""
+    V = 151936 if dtype == torch.float32 else 128256
+    x = inputs.logits_normal(48, V, 4.0, dtype, seed=70)
+    inputs.add_zipf_spike_(x, V, seed=71)
+    ctx = inputs.uniform_tokens((48, 4), V, seed=72)
+    got, sel = _check(x, V, ctx, KEY, 0.25, 2.0, scheme, 40)
+    changed = (got != host_bits(x)).sum(axis=1)
+    assert np.all(changed <= 40) and 100 < changed.sum() < 48 * 25      # about gamma * 40 per row
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("k", [1, 7, 40, 128, 129, 300])
+def test_various_k_ragged_rows_offset_and_unaligned(dtype, k):
+    B, V = 5, 10007
+    x = inputs.logits_normal(B, V + 9, 4.0, dtype, seed=73)
+    ctx = inputs.uniform_tokens((B, 1), 50000, seed=74)
+    _check(x, V, ctx, KEY, 0.5, 2.0, sbw.SCHEME_SELFSALT, k, off=1234)                       # padded rows
+    _check(x, V, ctx, KEY, 0.5, -1.5, sbw.SCHEME_SELFSALT, k, view=lambda t: t[:, 1:V + 1])  # unaligned
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_degenerate_rows_take_the_exact_fallback(dtype):
+    """Constant rows, two-valued rows, masked rows (-inf), zeros of both signs, NaNs: ties decide."""
+    V = 3000
+    x = inputs.logits_normal(8, V, 4.0, dtype, seed=75)
+    x[0, :] = 1.25
+    x[1, :] = float("-inf")
+    x[1, 17] = 0.5
+    x[2, ::2] = 3.0
+    x[2, 1::2] = -3.0
+    x[3, :] = 0.0
+    x[3, 5::7] = -0.0
+    x[4, 100:2900] = float("-inf")
+    x[5, 10] = float("nan")
+    x[5, 20] = float("inf")
+    x[6, :50] = 9.0
+    ctx = inputs.uniform_tokens((8, 1), V, seed=76)
+    for k in (1, 40, 200):
+        for delta in (2.0, -2.0):
+            _check(x, V, ctx, KEY, 0.5, delta, sbw.SCHEME_SELFSALT, k)
+
+
+def test_k_at_least_v_is_the_full_vocabulary_scheme_and_small_vocabularies():
+    dev = require_gpu()
+    for V in (1, 3, 8, 33):
+        x = inputs.logits_normal(4, V, 4.0, torch.float32, seed=77 + V)
+        ctx = inputs.uniform_tokens((4, 1), 1000, seed=78)
+        for k in (1, 2, V, V + 10):
+            _check(x, V, ctx, KEY, 0.5, 1.0, sbw.SCHEME_SELFSALT, k)
+    x = inputs.logits_normal(3, 4096, 4.0, torch.bfloat16, seed=79)
+    ctx = inputs.uniform_tokens((3, 1), 4096, seed=80)
+    a = x.to(dev)
+    b = x.to(dev)
+    sbw.sbw_bias_logits_topk(a, ctx.to(dev), KEY, 0.25, 2.0, 1, 5000)
+    sbw.sbw_bias_logits(b, ctx.to(dev), KEY, 0.25, 2.0, 1)
+    torch.cuda.synchronize()
+    assert host_bits(a).tobytes() == host_bits(b).tobytes()
+    L = sbw.lib()
+    assert L.sbw_bias_logits_topk(a.data_ptr(), 1, 3, 4096, 4096, 0, ctx.to(dev).data_ptr(), 1, KEY, 0.25, 2.0, 1,
+                                  0, None) == -1
