@@ -159,3 +159,46 @@ def test_host_buffer_entry_point():
     torch.cuda.synchronize()
     want = oracle.bias_logits(before, V, ctx.numpy(), KEY, 0.5, 2.0, oracle.SCHEME_CONTEXT)
     assert_same_bits(host_bits(x), want)
+
+
+def test_cuda_graph_replay_and_dependent_steps_keep_stream_order():
+    """The launch configuration the benchmark times: decode steps captured in one CUDA graph and
+    replayed.  The kernels use programmatic dependent launch, so this also checks that a step
+    which depends on the previous one (same buffer, biased twice; context tokens produced by a
+    kernel that runs just before) still sees its predecessor's writes."""
+    dev = require_gpu()
+    B, V, steps = 64, 128256, 6
+    xs = [inputs.logits_normal(B, V, 4.0, torch.bfloat16, seed=1200 + t, device=dev) for t in range(steps)]
+    ctxs = [inputs.uniform_tokens((B, 1), V, seed=1300 + t, device=dev) for t in range(steps)]
+    before = [host_bits(x) for x in xs]
+    same = inputs.logits_normal(B, V, 4.0, torch.float32, seed=1400, device=dev)
+    same_before = host_bits(same)
+    ctx_src = inputs.uniform_tokens((B, 1), V, seed=1401, device=dev)
+    ctx_dst = torch.zeros_like(ctx_src)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for t in range(2):                       # warm-up outside capture (first-call set-up)
+            sbw.sbw_bias_logits(torch.zeros((2, 64), dtype=torch.bfloat16, device=dev),
+                                torch.zeros((2, 1), dtype=torch.int32, device=dev), KEY, 0.5, 2.0, t)
+            sbw.sbw_bias_logits(torch.zeros((2, 64), dtype=torch.float32, device=dev),
+                                torch.zeros((2, 1), dtype=torch.int32, device=dev), KEY, 0.5, 2.0, t)
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for t in range(steps):
+                sbw.sbw_bias_logits(xs[t], ctxs[t], KEY, 0.5, 2.0, sbw.SCHEME_CONTEXT, stream=side)
+            ctx_dst.copy_(ctx_src + 0)           # a torch kernel writes the context tokens ...
+            for rep in range(3):                 # ... that three dependent in-place steps read
+                sbw.sbw_bias_logits(same, ctx_dst, KEY, 0.25, 1.5, rep % 2, stream=side)
+        graph.replay()
+    side.synchronize()
+    torch.cuda.synchronize()
+    for t in range(steps):
+        want = oracle.bias_logits(before[t], V, ctxs[t].cpu().numpy(), KEY, 0.5, 2.0, oracle.SCHEME_CONTEXT,
+                                  threads=8)
+        assert_same_bits(host_bits(xs[t]), want)
+    want = same_before
+    for rep in range(3):
+        want = oracle.bias_logits(want, V, ctx_src.cpu().numpy(), KEY, 0.25, 1.5, rep % 2, threads=8)
+    assert_same_bits(host_bits(same), want)
