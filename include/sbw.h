@@ -154,6 +154,34 @@ int sbw_bias_sample(const void *logits, int dtype, int64_t B, int64_t V, int64_t
                     void *stream);
 
 /*
+ * sbw_bias_sample_shard / sbw_sample_combine -- fused sampling of rows whose vocabulary is split
+ * over S shards (tensor-parallel language-model heads).  The paper states that every device can
+ * derive identical green lists from the shared key (Limitations) and leaves it unvalidated; with
+ * these two calls no shard reads another shard's logits and 32 bytes per row and shard are all
+ * that has to be exchanged.
+ *
+ * sbw_bias_sample_shard is sbw_bias_sample on one shard: `logits` holds columns vocab_offset ..
+ * vocab_offset+V-1 of rows row_offset .. row_offset+B-1 (row_offset enters the Gumbel counter, so
+ * a shard of the rows draws the same variates as the whole batch would; sbw_bias_sample uses 0).
+ *   out_shard   device, 16-byte aligned, [B, 8] float: per row (m, Z, best score s, GLOBAL id of
+ *               the best candidate as int bits, its biased logit, 0, 0, 0) of this shard.
+ *   out_tokens  device [B] int32: the shard-local column of that candidate (required).
+ * sbw_sample_combine merges S such summaries laid out [S, B, 8] (shard-major, e.g. the result of
+ * an all-gather): m = max m_r, Z = sum Z_r exp((m_r - m)/tau) in fp64, id = the global id with
+ * the largest s (ties -> lowest global id), p = exp((l_id - m)/tau)/Z.  out_max / out_sumexp /
+ * out_prob may be NULL.  The combined id, m, and (to 1e-6 relative) Z and p equal what
+ * sbw_bias_sample returns on the unsplit rows.
+ */
+int sbw_bias_sample_shard(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
+                          int64_t vocab_offset, int64_t row_offset, const int32_t *ctx_tokens,
+                          int ctx_width, uint64_t key, double gamma, float delta, int scheme,
+                          float temperature, uint64_t rng_seed, uint64_t rng_step, float *out_shard,
+                          int32_t *out_tokens, void *workspace, size_t workspace_bytes, void *stream);
+int sbw_sample_combine(const float *shards, int64_t S, int64_t B, float temperature,
+                       int32_t *out_tokens, float *out_max, float *out_sumexp, float *out_prob,
+                       void *stream);
+
+/*
  * sbw_bias_sample_noalloc -- sbw_bias_sample for callers that cannot hand over a workspace.
  * The paper has no counterpart for this call; it exists for deployment.  Some users of this
  * library cannot allocate device memory at all: a logits processor plugged into a serving

@@ -28,7 +28,8 @@ DTYPE_BF16 = 1
 EXPORTS = ("sbw_version", "sbw_last_cuda_error", "sbw_bias_logits",
            "sbw_bias_logits_host_staging_bytes", "sbw_bias_logits_host",
            "sbw_sample_workspace_bytes", "sbw_bias_sample", "sbw_detect_workspace_bytes",
-           "sbw_detect", "sbw_int_probe", "sbw_bias_sample_noalloc", "sbw_bias_logits_topk")
+           "sbw_detect", "sbw_int_probe", "sbw_bias_sample_noalloc", "sbw_bias_logits_topk",
+           "sbw_bias_sample_shard", "sbw_sample_combine")
 
 _lib = None
 
@@ -83,6 +84,11 @@ def lib() -> ctypes.CDLL:
         L.sbw_bias_sample_noalloc.argtypes = [vp, i32, i64, i64, i64, i64, vp, i32, u64, c.c_double,
                                               c.c_float, i32, c.c_float, u64, u64, vp, vp, vp, vp, vp,
                                               vp]
+        L.sbw_bias_sample_shard.restype = i32
+        L.sbw_bias_sample_shard.argtypes = [vp, i32, i64, i64, i64, i64, i64, vp, i32, u64, c.c_double,
+                                            c.c_float, i32, c.c_float, u64, u64, vp, vp, vp, sz, vp]
+        L.sbw_sample_combine.restype = i32
+        L.sbw_sample_combine.argtypes = [vp, i64, i64, c.c_float, vp, vp, vp, vp, vp]
         L.sbw_detect_workspace_bytes.restype = sz
         L.sbw_detect_workspace_bytes.argtypes = [i64]
         L.sbw_detect.restype = i32
@@ -239,6 +245,37 @@ def sbw_bias_sample_noalloc(logits: torch.Tensor, ctx_tokens: torch.Tensor, key:
                                        _ptr(out_sumexp), _ptr(out_prob), _ptr(out_probs),
                                        _stream(stream))
     _check("sbw_bias_sample_noalloc", rc)
+    return out_tokens
+
+
+def sbw_bias_sample_shard(logits: torch.Tensor, ctx_tokens: torch.Tensor, key: int, gamma: float,
+                          delta: float, scheme: int, temperature: float, rng_seed: int, rng_step: int,
+                          out_shard: torch.Tensor, out_tokens: torch.Tensor, workspace: torch.Tensor, *,
+                          vocab_offset: int, row_offset: int = 0, V: int | None = None,
+                          stream=None) -> torch.Tensor:
+    """Fused sampling on one vocabulary shard; fills ``out_shard`` ([B, 8] float32) and returns it."""
+    B, V, ld = _row_layout(logits, V)
+    W = _ctx(ctx_tokens, B)
+    if out_shard.dtype != torch.float32 or out_shard.numel() != B * 8 or not out_shard.is_contiguous():
+        raise TypeError("out_shard must be a contiguous float32 tensor of B * 8 values")
+    rc = lib().sbw_bias_sample_shard(_ptr(logits), _dtype_code(logits), B, V, ld, vocab_offset, row_offset,
+                                     _ptr(ctx_tokens), W, key, gamma, delta, scheme, temperature, rng_seed,
+                                     rng_step, _ptr(out_shard), _ptr(out_tokens), _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _stream(stream))
+    _check("sbw_bias_sample_shard", rc)
+    return out_shard
+
+
+def sbw_sample_combine(shards: torch.Tensor, temperature: float, out_tokens: torch.Tensor, *,
+                       out_max: torch.Tensor | None = None, out_sumexp: torch.Tensor | None = None,
+                       out_prob: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """Merges per-shard summaries ``[S, B, 8]`` into global token ids (and optional statistics)."""
+    if shards.dim() != 3 or shards.shape[2] != 8 or shards.dtype != torch.float32 or not shards.is_contiguous():
+        raise TypeError("shards must be a contiguous float32 tensor of shape [S, B, 8]")
+    S, B = shards.shape[0], shards.shape[1]
+    rc = lib().sbw_sample_combine(_ptr(shards), S, B, temperature, _ptr(out_tokens), _ptr(out_max),
+                                  _ptr(out_sumexp), _ptr(out_prob), _stream(stream))
+    _check("sbw_sample_combine", rc)
     return out_tokens
 
 

@@ -73,6 +73,8 @@ struct SampleArgs {
     Weyl weyl;                   // key-schedule increments of the green hash
     int32_t *out_tokens;
     float *out_max, *out_sumexp, *out_prob;
+    float *out_shard;     // [B, 8] or NULL: (m, Z, best score, global id bits, its biased logit, 0, 0, 0)
+    uint32_t row_offset;  // global index of row 0 (enters the Gumbel counter)
     Partial *partials;    // [B * split]
     unsigned *tickets;    // [B], zero before the launch
     unsigned *bounds;     // [B], zero before the launch: best exact score per row, order-encoded
@@ -258,6 +260,11 @@ __device__ void finish_row(const SampleArgs &a, int64_t row, const Partial *part
         if (a.out_sumexp) a.out_sumexp[row] = static_cast<float>(Z);
         if (a.out_prob) a.out_prob[row] = static_cast<float>(exp((static_cast<double>(l) - md) / a.tau) / Z);
         a.rowstats[row] = make_double2(md, Z);
+        if (a.out_shard) {
+            float4 *o = reinterpret_cast<float4 *>(a.out_shard + row * 8);
+            o[0] = make_float4(m, static_cast<float>(Z), s, __int_as_float(static_cast<int>(a.vocab_offset) + id));
+            o[1] = make_float4(l, 0.0f, 0.0f, 0.0f);
+        }
     }
 }
 
@@ -342,7 +349,7 @@ sample_kernel(const SampleArgs a) {
         const int chunk = static_cast<int>(item - row * a.split);
         const uint32_t j_begin = chunk * a.slots_per_chunk;
         const uint32_t j_end = min(a.nslot, j_begin + a.slots_per_chunk);
-        const uint32_t rowb = static_cast<uint32_t>(row);
+        const uint32_t rowb = a.row_offset + static_cast<uint32_t>(row);
         const char *row_ptr = static_cast<const char *>(a.logits) + row * a.ld * ESIZE;
 
         RowSeedS<SCHEME> rs;
@@ -562,7 +569,8 @@ int bias_sample_impl(const void *logits, int dtype, int64_t B, int64_t V, int64_
                      const int32_t *ctx_tokens, int ctx_width, uint64_t key, double gamma, float delta,
                      int scheme, float temperature, uint64_t rng_seed, uint64_t rng_step, int32_t *out_tokens,
                      float *out_max, float *out_sumexp, float *out_prob, float *out_probs, void *workspace,
-                     size_t workspace_bytes, bool need_full_workspace, cudaStream_t s) {
+                     size_t workspace_bytes, bool need_full_workspace, cudaStream_t s,
+                     float *out_shard = nullptr, int64_t row_offset = 0) {
     if (!valid_common(dtype, ctx_width, gamma, scheme)) return SBW_ERR_INVALID_ARG;
     if (B < 0 || V <= 0 || ld < V || vocab_offset < 0) return SBW_ERR_INVALID_ARG;
     if (!(temperature > 0.0f) || temperature - temperature != 0.0f) return SBW_ERR_INVALID_ARG;
@@ -571,6 +579,8 @@ int bias_sample_impl(const void *logits, int dtype, int64_t B, int64_t V, int64_
     if (B > 0x7fffffffLL / kMaxSplit) return SBW_ERR_UNSUPPORTED;
     if (B == 0) return SBW_OK;
     if (!logits || !ctx_tokens || !out_tokens) return SBW_ERR_INVALID_ARG;
+    if (row_offset < 0 || row_offset + B > (int64_t(1) << 32)) return SBW_ERR_INVALID_ARG;
+    if (out_shard && reinterpret_cast<uintptr_t>(out_shard) % 16 != 0) return SBW_ERR_INVALID_ARG;
     const double c2 = 1.4426950408889634 / static_cast<double>(temperature);
     const float c2_hi = static_cast<float>(c2);
     if (!(c2_hi * 1e15f < FLT_MAX)) return SBW_ERR_INVALID_ARG;   // temperature too small
@@ -612,6 +622,8 @@ int bias_sample_impl(const void *logits, int dtype, int64_t B, int64_t V, int64_
     a.out_max = out_max;
     a.out_sumexp = out_sumexp;
     a.out_prob = out_prob;
+    a.out_shard = out_shard;
+    a.row_offset = static_cast<uint32_t>(row_offset);
     a.partials = ws.partials;
     a.tickets = ws.tickets;
     a.bounds = ws.bounds;
@@ -708,4 +720,67 @@ extern "C" int sbw_bias_sample_noalloc(const void *logits, int dtype, int64_t B,
                             scheme, temperature, rng_seed, rng_step, out_tokens, out_max, out_sumexp,
                             out_prob, out_probs, scratch, kNoallocScratchBytes, false,
                             static_cast<cudaStream_t>(stream));
+}
+
+// ---------------------------------------------------------------------------------------------
+// Vocabulary-sharded sampling.  The paper notes that each device can derive identical green
+// lists from the shared key (Limitations) without validating it; here a row whose vocabulary is
+// split over S shards is sampled by S independent sbw_bias_sample_shard calls -- no shard reads
+// another's logits -- and one tiny combine over the S per-row summaries, which is the only data
+// that has to cross devices (32 bytes per row and shard).
+// ---------------------------------------------------------------------------------------------
+namespace sbw {
+namespace {
+
+__global__ void combine_kernel(const float *shards, int64_t S, int64_t B, double tau, int32_t *out_tokens,
+                               float *out_max, float *out_sumexp, float *out_prob) {
+    const int64_t row = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (row >= B) return;
+    // pass 1: row maximum and winner (ties -> lowest global id); pass 2: rescaled sum
+    float m = -INFINITY, s = -INFINITY, l = -INFINITY;
+    int id = INT_MAX;
+    for (int64_t r = 0; r < S; ++r) {
+        const float4 q = *reinterpret_cast<const float4 *>(shards + (r * B + row) * 8);
+        m = fmaxf(m, q.x);
+        const int qid = __float_as_int(q.w);
+        if (better(q.z, qid, s, id)) { s = q.z; id = qid; l = shards[(r * B + row) * 8 + 4]; }
+    }
+    double Z = 0.0;
+    for (int64_t r = 0; r < S; ++r) {
+        const float4 q = *reinterpret_cast<const float4 *>(shards + (r * B + row) * 8);
+        if (q.x > -INFINITY) Z += static_cast<double>(q.y) * exp((static_cast<double>(q.x) - m) / tau);
+    }
+    out_tokens[row] = id;
+    if (out_max) out_max[row] = m;
+    if (out_sumexp) out_sumexp[row] = static_cast<float>(Z);
+    if (out_prob) out_prob[row] = static_cast<float>(exp((static_cast<double>(l) - m) / tau) / Z);
+}
+
+}  // namespace
+}  // namespace sbw
+
+extern "C" int sbw_bias_sample_shard(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
+                                     int64_t vocab_offset, int64_t row_offset, const int32_t *ctx_tokens,
+                                     int ctx_width, uint64_t key, double gamma, float delta, int scheme,
+                                     float temperature, uint64_t rng_seed, uint64_t rng_step,
+                                     float *out_shard, int32_t *out_tokens, void *workspace,
+                                     size_t workspace_bytes, void *stream) {
+    if (B > 0 && !out_shard) return SBW_ERR_INVALID_ARG;
+    return sbw::bias_sample_impl(logits, dtype, B, V, ld, vocab_offset, ctx_tokens, ctx_width, key, gamma,
+                                 delta, scheme, temperature, rng_seed, rng_step, out_tokens, nullptr, nullptr,
+                                 nullptr, nullptr, workspace, workspace_bytes, true,
+                                 static_cast<cudaStream_t>(stream), out_shard, row_offset);
+}
+
+extern "C" int sbw_sample_combine(const float *shards, int64_t S, int64_t B, float temperature,
+                                  int32_t *out_tokens, float *out_max, float *out_sumexp, float *out_prob,
+                                  void *stream) {
+    if (S < 1 || B < 0 || !(temperature > 0.0f) || temperature - temperature != 0.0f) return SBW_ERR_INVALID_ARG;
+    if (B == 0) return SBW_OK;
+    if (!shards || !out_tokens || reinterpret_cast<uintptr_t>(shards) % 16 != 0) return SBW_ERR_INVALID_ARG;
+    const unsigned grid = static_cast<unsigned>((B + 127) / 128);
+    sbw::combine_kernel<<<grid, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        shards, S, B, static_cast<double>(temperature), out_tokens, out_max, out_sumexp, out_prob);
+    SBW_CUDA_TRY(cudaGetLastError());
+    return SBW_OK;
 }

@@ -1,0 +1,55 @@
+"""Vocabulary-sharded fused sampling across ranks: each rank samples on its own columns, the
+per-row summaries (32 bytes per row) are all-gathered, and every rank combines them.
+
+The paper observes that each device can derive identical green lists from the shared key and
+leaves the multi-device case unvalidated; this module is that case.  The only collective is one
+all-gather of a ``[B, 8]`` float32 tensor (NCCL on GPUs; any torch.distributed backend works).
+"""
+from __future__ import annotations
+
+import torch
+import torch.distributed as dist
+
+from . import binding
+
+
+def shard_columns(V: int, rank: int, world: int, align: int = 8) -> tuple[int, int]:
+    """Columns [lo, hi) of a vocabulary of V ids owned by ``rank``: contiguous, balanced, and cut
+    at multiples of ``align`` so that every shard's rows can stay 16-byte aligned."""
+    units = (V + align - 1) // align
+    base, rem = divmod(units, world)
+    lo_u = rank * base + min(rank, rem)
+    hi_u = lo_u + base + (1 if rank < rem else 0)
+    return min(lo_u * align, V), min(hi_u * align, V)
+
+
+def gather_summaries(local: torch.Tensor, group=None) -> torch.Tensor:
+    """All-gather of the per-rank ``[B, 8]`` summaries into ``[world, B, 8]`` (rank-major)."""
+    world = dist.get_world_size(group) if dist.is_initialized() else 1
+    if world == 1:
+        return local.reshape(1, *local.shape).contiguous()
+    out = torch.empty((world, *local.shape), dtype=local.dtype, device=local.device)
+    dist.all_gather([out[r] for r in range(world)], local.contiguous(), group=group)
+    return out
+
+
+def sharded_bias_sample(logits_shard: torch.Tensor, ctx_tokens: torch.Tensor, key: int, gamma: float,
+                        delta: float, scheme: int, temperature: float, rng_seed: int, rng_step: int,
+                        vocab_offset: int, workspace: torch.Tensor, group=None, row_offset: int = 0):
+    """Samples one token per row from logits whose columns are spread over the ranks of ``group``.
+    ``logits_shard`` holds this rank's columns, ``vocab_offset`` the global id of its column 0.
+    Returns (global token ids [B] int32, m [B], Z [B], p [B]) -- identical on every rank."""
+    B = logits_shard.shape[0]
+    dev = logits_shard.device
+    summary = torch.empty((B, 8), dtype=torch.float32, device=dev)
+    local_ids = torch.empty(B, dtype=torch.int32, device=dev)
+    binding.sbw_bias_sample_shard(logits_shard, ctx_tokens, key, gamma, delta, scheme, temperature, rng_seed,
+                                  rng_step, summary, local_ids, workspace, vocab_offset=vocab_offset,
+                                  row_offset=row_offset)
+    shards = gather_summaries(summary, group)
+    tokens = torch.empty(B, dtype=torch.int32, device=dev)
+    m = torch.empty(B, dtype=torch.float32, device=dev)
+    Z = torch.empty(B, dtype=torch.float32, device=dev)
+    p = torch.empty(B, dtype=torch.float32, device=dev)
+    binding.sbw_sample_combine(shards, temperature, tokens, out_max=m, out_sumexp=Z, out_prob=p)
+    return tokens, m, Z, p

@@ -69,3 +69,69 @@ def test_shard_rows_is_a_balanced_partition():
             assert all(parts[i][1] == parts[i + 1][0] for i in range(world - 1))
             sizes = [hi - lo for lo, hi in parts]
             assert max(sizes) - min(sizes) <= 1
+
+
+def _shard_worker(rank: int, world: int, port: int, out_dir: str):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank),
+                      WORLD_SIZE=str(world), LOCAL_RANK=str(rank))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import oracle
+    from paper_2609_03844_b200 import inputs, sharded
+
+    B, V, tau = 3, 4000, 0.7
+    x = inputs.logits_normal(B, V, 4.0, torch.float32, seed=5)
+    ctx = inputs.uniform_tokens((B, 1), V, seed=6).numpy()
+    lo, hi = sharded.shard_columns(V, rank, world)
+    part = np.ascontiguousarray(x.numpy()[:, lo:hi])
+    # this rank's summary, from the oracle on its own columns only (global ids via vocab_offset)
+    o = oracle.bias_sample(part, hi - lo, ctx, 0x5EED, 0.25, 2.0, 1, tau, 9, 4, vocab_offset=lo)
+    biased = oracle.bias_logits(part, hi - lo, ctx, 0x5EED, 0.25, 2.0, 1, vocab_offset=lo)
+    summ = np.zeros((B, 8), dtype=np.float32)
+    summ[:, 0] = o["max"]
+    summ[:, 1] = o["sumexp"]
+    summ[:, 2] = o["score"]
+    summ[:, 3] = (o["tokens"] + lo).astype(np.int32).view(np.float32)
+    summ[:, 4] = biased[np.arange(B), o["tokens"]]
+    gathered = sharded.gather_summaries(torch.from_numpy(summ))
+    assert gathered.shape == (world, B, 8)
+    assert torch.equal(gathered[rank], torch.from_numpy(summ))           # rank-major layout
+    np.save(os.path.join(out_dir, f"gathered{rank}.npy"), gathered.numpy())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_exchange_shard_summaries(tmp_path):
+    """Vocabulary-sharded sampling, host side: each rank summarises its own columns, one all-gather,
+    and the combination rule (largest score, ties to the lowest global id; rescaled sums) gives
+    what the oracle returns on the whole rows."""
+    world = 2
+    mp.spawn(_shard_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    import oracle
+    from paper_2609_03844_b200 import inputs
+
+    g0 = np.load(tmp_path / "gathered0.npy")
+    g1 = np.load(tmp_path / "gathered1.npy")
+    assert np.array_equal(g0.view(np.uint32), g1.view(np.uint32))         # every rank holds the same table
+    B, V, tau = 3, 4000, 0.7
+    x = inputs.logits_normal(B, V, 4.0, torch.float32, seed=5).numpy()
+    ctx = inputs.uniform_tokens((B, 1), V, seed=6).numpy()
+    want = oracle.bias_sample(x, V, ctx, 0x5EED, 0.25, 2.0, 1, tau, 9, 4)
+    tau32 = float(np.float32(tau))
+    for b in range(B):
+        ids = g0[:, b, 3].view(np.int32)
+        order = sorted(range(world), key=lambda r: (-g0[r, b, 2], ids[r]))
+        assert ids[order[0]] == want["tokens"][b]
+        m = g0[:, b, 0].max()
+        Z = sum(float(g0[r, b, 1]) * np.exp((float(g0[r, b, 0]) - float(m)) / tau32) for r in range(world))
+        assert m == want["max"][b] and abs(Z / want["sumexp"][b] - 1) < 1e-6
+
+
+def test_shard_columns_partition_is_aligned_and_complete():
+    from paper_2609_03844_b200 import sharded
+
+    for V in (1, 7, 8, 128256, 151936, 32001):
+        for world in (1, 2, 3, 8):
+            parts = [sharded.shard_columns(V, r, world) for r in range(world)]
+            assert parts[0][0] == 0 and parts[-1][1] == V
+            assert all(parts[i][1] == parts[i + 1][0] for i in range(world - 1))
+            assert all(lo % 8 == 0 or lo == V for lo, _ in parts)
