@@ -128,7 +128,7 @@ __device__ __forceinline__ int score_trip(const DetectArgs &a, const int32_t *to
 #pragma unroll
     for (int u = 0; u < kDetectIlp; ++u) {
         const int t = base + u * 32 + lane;
-        valid[u] = !TAIL || t < len;
+        valid[u] = !TAIL || static_cast<unsigned>(t) < static_cast<unsigned>(len);
         const int ts = valid[u] ? t : width;      // any readable position; its result is dropped
         v[u] = static_cast<uint32_t>(tok[ts]);
         if constexpr (SCHEME == SBW_SCHEME_CONTEXT) {
@@ -175,7 +175,8 @@ detect_kernel(const DetectArgs a) {
 
     int count = 0;
     int base = width;
-    for (; base + kTrip <= len; base += kTrip) count += score_trip<SCHEME, WIDTH, false>(a, tok, base, len, lane);
+    // written as a difference so that lengths near 2^31 cannot overflow the trip counter
+    for (; len - base >= kTrip; base += kTrip) count += score_trip<SCHEME, WIDTH, false>(a, tok, base, len, lane);
     if (base < len) count += score_trip<SCHEME, WIDTH, true>(a, tok, base, len, lane);
 
     if (lane == 0) {
