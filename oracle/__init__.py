@@ -79,6 +79,10 @@ def lib() -> ctypes.CDLL:
                                                   c.c_float, i32, i64, vp]
         L.sbw_oracle_detect.restype = None
         L.sbw_oracle_detect.argtypes = [vp, vp, i64, i32, u64, c.c_double, i32, vp, vp, vp, i32]
+        L.sbw_oracle_detect_bits.restype = None
+        L.sbw_oracle_detect_bits.argtypes = [vp, vp, i64, i32, u64, c.c_double, i32, vp]
+        L.sbw_oracle_window_z.restype = None
+        L.sbw_oracle_window_z.argtypes = [vp, vp, i64, i32, i64, c.c_double, vp, vp, vp]
         L.sbw_oracle_zscore.restype = c.c_double
         L.sbw_oracle_zscore.argtypes = [i64, i64, c.c_double]
         L.sbw_oracle_log.restype = c.c_float
@@ -185,6 +189,28 @@ def detect(tokens, lengths, key, gamma, scheme, ctx_width=1, threads=1):
     lib().sbw_oracle_detect(_ptr(tok), _ptr(lens), N, ctx_width, key, gamma, scheme, _ptr(counts),
                             _ptr(T), _ptr(z), threads)
     return counts, T, z
+
+
+def detect_bits(tokens, lengths, key, gamma, scheme, ctx_width=1) -> np.ndarray:
+    """Y_t for every token of the flat array (0 for the unscored first ctx_width tokens)."""
+    tok = np.ascontiguousarray(np.asarray(tokens, dtype=np.int32))
+    lens = np.ascontiguousarray(np.asarray(lengths, dtype=np.int32))
+    green = np.zeros(tok.shape[0], dtype=np.uint8)
+    lib().sbw_oracle_detect_bits(_ptr(tok), _ptr(lens), lens.shape[0], ctx_width, key, gamma, scheme,
+                                 _ptr(green))
+    return green
+
+
+def window_z(green, lengths, window, gamma, ctx_width=1):
+    """Best window of ``window`` scored positions per sequence: (count, start, z)."""
+    g = np.ascontiguousarray(np.asarray(green, dtype=np.uint8))
+    lens = np.ascontiguousarray(np.asarray(lengths, dtype=np.int32))
+    N = lens.shape[0]
+    bc = np.zeros(N, dtype=np.int32)
+    bs = np.zeros(N, dtype=np.int32)
+    bz = np.zeros(N, dtype=np.float64)
+    lib().sbw_oracle_window_z(_ptr(g), _ptr(lens), N, ctx_width, window, gamma, _ptr(bc), _ptr(bs), _ptr(bz))
+    return bc, bs, bz
 
 
 def zscore(G: int, T: int, gamma: float) -> float:

@@ -320,6 +320,53 @@ void sbw_oracle_detect(const int32_t *tokens, const int32_t *lengths, int64_t N,
     free(offsets);
 }
 
+void sbw_oracle_detect_bits(const int32_t *tokens, const int32_t *lengths, int64_t N, int ctx_width,
+                            uint64_t key, double gamma, int scheme, uint8_t *green)
+{
+    uint64_t thr = sbw_oracle_threshold(gamma);
+    int64_t off = 0;
+    for (int64_t s = 0; s < N; ++s) {
+        int64_t L = lengths[s] > 0 ? lengths[s] : 0;
+        const int32_t *tok = tokens + off;
+        for (int64_t t = 0; t < L; ++t) {
+            int g = 0;
+            if (t >= ctx_width) {
+                uint32_t v = (uint32_t)tok[t];
+                g = sbw_oracle_green(seed_for(scheme, key, tok + (t - ctx_width), ctx_width, v), v, thr);
+            }
+            green[off + t] = (uint8_t)g;
+        }
+        off += L;
+    }
+}
+
+void sbw_oracle_window_z(const uint8_t *green, const int32_t *lengths, int64_t N, int ctx_width,
+                         int64_t window, double gamma, int32_t *best_count, int32_t *best_start,
+                         double *best_z)
+{
+    int64_t off = 0;
+    for (int64_t s = 0; s < N; ++s) {
+        int64_t L = lengths[s] > 0 ? lengths[s] : 0;
+        int64_t T = L > ctx_width ? L - ctx_width : 0;
+        const uint8_t *y = green + off + (L > ctx_width ? ctx_width : L);   /* scored positions */
+        int64_t w = window < T ? window : T;
+        int64_t bc = 0, bs = 0;
+        for (int64_t start = 0; start + w <= T && w > 0; ++start) {
+            int64_t c = 0;
+            for (int64_t i = 0; i < w; ++i)
+                c += y[start + i];
+            if (c > bc) {               /* strict: ties keep the earliest start */
+                bc = c;
+                bs = start;
+            }
+        }
+        best_count[s] = (int32_t)bc;
+        best_start[s] = (int32_t)bs;
+        best_z[s] = sbw_oracle_zscore(bc, w, gamma);
+        off += L;
+    }
+}
+
 /* ------------------------------------------------------------------ R8: sampler ---- */
 /*
  * Specified fp32 natural logarithm for positive normal x (every step one IEEE operation):

@@ -89,6 +89,17 @@ void sbw_oracle_bias_logits_topk(void *logits, int dtype, int64_t B, int64_t V, 
 void sbw_oracle_detect(const int32_t *tokens, const int32_t *lengths, int64_t N, int ctx_width,
                        uint64_t key, double gamma, int scheme, int32_t *counts, int32_t *T,
                        double *z, int threads);
+/* The per-token indicators Y_t of Section 3 themselves: green[offset_s + t] for every token of the
+ * flat array (0 for the first W tokens of a sequence, which are not scored). */
+void sbw_oracle_detect_bits(const int32_t *tokens, const int32_t *lengths, int64_t N, int ctx_width,
+                            uint64_t key, double gamma, int scheme, uint8_t *green);
+/* Windowed detection for partly watermarked or truncated text (the paper's robustness study cuts
+ * and edits text, Appendix G): over the T scored positions of a sequence, the window of `window`
+ * consecutive positions (the whole sequence if T < window) with the most green tokens, ties to
+ * the earliest start; Eq. 5 on that window.  T = 0 gives count 0, start 0, z 0. */
+void sbw_oracle_window_z(const uint8_t *green, const int32_t *lengths, int64_t N, int ctx_width,
+                         int64_t window, double gamma, int32_t *best_count, int32_t *best_start,
+                         double *best_z);
 /* Eq. 5 alone. */
 double sbw_oracle_zscore(int64_t G, int64_t T, double gamma);
 
