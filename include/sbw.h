@@ -234,6 +234,34 @@ int sbw_detect(const int32_t *tokens, const int32_t *lengths, const int64_t *off
                int32_t *out_counts, int32_t *out_T, double *out_z, void *workspace,
                size_t workspace_bytes, void *stream);
 
+/*
+ * sbw_detect_bits -- sbw_detect that also keeps the per-token indicators Y_i of Section 3 (the
+ * paper's robustness study, Appendix G, scores cut and edited text; partly watermarked text needs
+ * more than one count per sequence).  Arguments and results as for sbw_detect, plus
+ *   out_bits   device, uint32[sbw_detect_bits_words(N, total_tokens)].  The bits of sequence s
+ *              start at word (offset_s >> 5) + 2 s; scored position i (token W + i) is bit i & 31
+ *              of word i >> 5 of that region; ceil(T / 32) words per sequence are written, unused
+ *              high bits of the last one are 0, other words are left as they were.
+ * When `offsets` is NULL the scanned int64[N + 1] offsets are left at the start of `workspace`,
+ * where sbw_window_z can read them.
+ *
+ * sbw_window_z -- windowed detection on those bits: per sequence, the window of `window`
+ * consecutive scored positions (all T of them if T < window) with the most green tokens, ties to
+ * the earliest start, and Eq. 5 on that window.  T = 0 gives count 0, start 0, z 0.
+ *   bits, lengths, offsets (required, device), total_tokens, ctx_width  as used by sbw_detect_bits.
+ *   prefix_scratch  device, uint32[sbw_detect_bits_words(N, total_tokens)], contents undefined after.
+ *   out_count, out_start  device [N] int32;  out_z  device [N] double.
+ */
+size_t sbw_detect_bits_words(int64_t N, int64_t total_tokens);
+int sbw_detect_bits(const int32_t *tokens, const int32_t *lengths, const int64_t *offsets, int64_t N,
+                    int64_t total_tokens, int ctx_width, uint64_t key, double gamma, int scheme,
+                    int32_t *out_counts, int32_t *out_T, double *out_z, uint32_t *out_bits,
+                    void *workspace, size_t workspace_bytes, void *stream);
+int sbw_window_z(const uint32_t *bits, const int32_t *lengths, const int64_t *offsets, int64_t N,
+                 int64_t total_tokens, int ctx_width, int64_t window, double gamma,
+                 uint32_t *prefix_scratch, int32_t *out_count, int32_t *out_start, double *out_z,
+                 void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -29,7 +29,8 @@ EXPORTS = ("sbw_version", "sbw_last_cuda_error", "sbw_bias_logits",
            "sbw_bias_logits_host_staging_bytes", "sbw_bias_logits_host",
            "sbw_sample_workspace_bytes", "sbw_bias_sample", "sbw_detect_workspace_bytes",
            "sbw_detect", "sbw_int_probe", "sbw_bias_sample_noalloc", "sbw_bias_logits_topk",
-           "sbw_bias_sample_shard", "sbw_sample_combine")
+           "sbw_bias_sample_shard", "sbw_sample_combine", "sbw_detect_bits_words", "sbw_detect_bits",
+           "sbw_window_z")
 
 _lib = None
 
@@ -94,6 +95,13 @@ def lib() -> ctypes.CDLL:
         L.sbw_detect.restype = i32
         L.sbw_detect.argtypes = [vp, vp, vp, i64, i64, i32, u64, c.c_double, i32, vp, vp, vp, vp,
                                  sz, vp]
+        L.sbw_detect_bits_words.restype = sz
+        L.sbw_detect_bits_words.argtypes = [i64, i64]
+        L.sbw_detect_bits.restype = i32
+        L.sbw_detect_bits.argtypes = [vp, vp, vp, i64, i64, i32, u64, c.c_double, i32, vp, vp, vp, vp, vp,
+                                      sz, vp]
+        L.sbw_window_z.restype = i32
+        L.sbw_window_z.argtypes = [vp, vp, vp, i64, i64, i32, i64, c.c_double, vp, vp, vp, vp, vp]
         L.sbw_int_probe.restype = i32
         L.sbw_int_probe.argtypes = [i32, i32, i32, i32, vp, vp, vp]
         _lib = L
@@ -302,6 +310,40 @@ def sbw_detect(tokens: torch.Tensor, lengths: torch.Tensor, key: int, gamma: flo
                           _ptr(workspace), ws_bytes, _stream(stream))
     _check("sbw_detect", rc)
     return out_counts, out_z
+
+
+def sbw_detect_bits_words(N: int, total_tokens: int) -> int:
+    return int(lib().sbw_detect_bits_words(N, total_tokens))
+
+
+def sbw_detect_bits(tokens: torch.Tensor, lengths: torch.Tensor, key: int, gamma: float, scheme: int,
+                    out_counts: torch.Tensor, out_z: torch.Tensor, out_bits: torch.Tensor, *,
+                    out_T: torch.Tensor | None = None, offsets: torch.Tensor | None = None,
+                    workspace: torch.Tensor | None = None, ctx_width: int = 1, stream=None):
+    """sbw_detect that also stores the per-token green bits (int32/uint32 words, see sbw.h)."""
+    N = lengths.numel()
+    if out_bits.element_size() != 4 or out_bits.numel() < sbw_detect_bits_words(N, tokens.numel()):
+        raise TypeError("out_bits must hold sbw_detect_bits_words(N, total) 32-bit words")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().sbw_detect_bits(_ptr(tokens), _ptr(lengths), _ptr(offsets), N, tokens.numel(), ctx_width, key,
+                               gamma, scheme, _ptr(out_counts), _ptr(out_T), _ptr(out_z), _ptr(out_bits),
+                               _ptr(workspace), ws_bytes, _stream(stream))
+    _check("sbw_detect_bits", rc)
+    return out_bits
+
+
+def sbw_window_z(bits: torch.Tensor, lengths: torch.Tensor, offsets: torch.Tensor, total_tokens: int,
+                 window: int, gamma: float, prefix_scratch: torch.Tensor, out_count: torch.Tensor,
+                 out_start: torch.Tensor, out_z: torch.Tensor, *, ctx_width: int = 1, stream=None):
+    """Best window of ``window`` scored positions per sequence from stored green bits."""
+    N = lengths.numel()
+    if offsets.dtype != torch.int64 or offsets.numel() < N + 1:
+        raise TypeError("offsets must be int64 with N + 1 entries")
+    rc = lib().sbw_window_z(_ptr(bits), _ptr(lengths), _ptr(offsets), N, total_tokens, ctx_width, window, gamma,
+                            _ptr(prefix_scratch), _ptr(out_count), _ptr(out_start), _ptr(out_z),
+                            _stream(stream))
+    _check("sbw_window_z", rc)
+    return out_count, out_start, out_z
 
 
 PROBE_KINDS = {"mulwide": (0, 1), "lop3": (1, 1), "iadd3": (2, 1), "imad": (3, 1), "philox": (4, 4),

@@ -42,6 +42,7 @@ struct DetectArgs {
     int32_t *out_counts;
     int32_t *out_T;
     double *out_z;
+    uint32_t *out_bits;   // nullable: per-token green bits, see sbw_detect_bits in sbw.h
     Weyl weyl;   // Philox key-schedule increments (see sbw_hash.cuh)
 };
 
@@ -120,7 +121,7 @@ scan_offsets(const int32_t *lengths, int64_t N, const int64_t *tile_sums, int64_
 // width at compile time (loops unrolled), WIDTH = 0 reads it from the arguments.
 template <int SCHEME, int WIDTH, bool TAIL>
 __device__ __forceinline__ int score_trip(const DetectArgs &a, const int32_t *tok, int base, int len,
-                                          int lane) {
+                                          int lane, uint32_t *bits) {
     const int width = WIDTH > 0 ? WIDTH : a.W;
     uint32_t v[kDetectIlp];
     uint64_t r[kDetectIlp];
@@ -153,8 +154,12 @@ __device__ __forceinline__ int score_trip(const DetectArgs &a, const int32_t *to
     philox_word0_n<kDetectIlp>(v, r, x, a.weyl);
     int count = 0;
 #pragma unroll
-    for (int u = 0; u < kDetectIlp; ++u)
-        count += __popc(__ballot_sync(0xffffffffu, valid[u] && x[u] <= a.thr_m1));
+    for (int u = 0; u < kDetectIlp; ++u) {
+        const unsigned greens = __ballot_sync(0xffffffffu, valid[u] && x[u] <= a.thr_m1);
+        count += __popc(greens);
+        // the ballot is the bit mask of 32 consecutive scored positions: keep it if asked to
+        if (bits && lane == 0 && (!TAIL || base + u * 32 < len)) bits[((base - width) >> 5) + u] = greens;
+    }
     return count;
 }
 
@@ -176,8 +181,10 @@ detect_kernel(const DetectArgs a) {
     int count = 0;
     int base = width;
     // written as a difference so that lengths near 2^31 cannot overflow the trip counter
-    for (; len - base >= kTrip; base += kTrip) count += score_trip<SCHEME, WIDTH, false>(a, tok, base, len, lane);
-    if (base < len) count += score_trip<SCHEME, WIDTH, true>(a, tok, base, len, lane);
+    uint32_t *bits = a.out_bits ? a.out_bits + (off >> 5) + 2 * seq : nullptr;
+    for (; len - base >= kTrip; base += kTrip)
+        count += score_trip<SCHEME, WIDTH, false>(a, tok, base, len, lane, bits);
+    if (base < len) count += score_trip<SCHEME, WIDTH, true>(a, tok, base, len, lane, bits);
 
     if (lane == 0) {
         const int T = len > width ? len - width : 0;
@@ -214,11 +221,12 @@ extern "C" size_t sbw_detect_workspace_bytes(int64_t N) {
            sbw::align_up(tiles * sizeof(int64_t), 256);
 }
 
-extern "C" int sbw_detect(const int32_t *tokens, const int32_t *lengths, const int64_t *offsets,
-                          int64_t N, int64_t total_tokens, int ctx_width, uint64_t key, double gamma,
-                          int scheme, int32_t *out_counts, int32_t *out_T, double *out_z,
-                          void *workspace, size_t workspace_bytes, void *stream) {
-    using namespace sbw;
+namespace sbw {
+namespace {
+int detect_impl(const int32_t *tokens, const int32_t *lengths, const int64_t *offsets, int64_t N,
+                int64_t total_tokens, int ctx_width, uint64_t key, double gamma, int scheme,
+                int32_t *out_counts, int32_t *out_T, double *out_z, uint32_t *out_bits, void *workspace,
+                size_t workspace_bytes, void *stream) {
     if (!valid_common(SBW_DTYPE_F32, ctx_width, gamma, scheme)) return SBW_ERR_INVALID_ARG;
     if (N < 0 || total_tokens < 0) return SBW_ERR_INVALID_ARG;
     if (N == 0) return SBW_OK;
@@ -240,6 +248,7 @@ extern "C" int sbw_detect(const int32_t *tokens, const int32_t *lengths, const i
     a.out_counts = out_counts;
     a.out_T = out_T;
     a.out_z = out_z;
+    a.out_bits = out_bits;
     a.weyl = make_weyl();
 
     if (!offsets) {
@@ -259,5 +268,114 @@ extern "C" int sbw_detect(const int32_t *tokens, const int32_t *lengths, const i
     const unsigned grid = static_cast<unsigned>((N + kDetectThreads / 32 - 1) / (kDetectThreads / 32));
     SBW_CUDA_TRY(scheme == SBW_SCHEME_CONTEXT ? launch_detect<SBW_SCHEME_CONTEXT>(a, grid, s)
                                               : launch_detect<SBW_SCHEME_SELFSALT>(a, grid, s));
+    return SBW_OK;
+}
+
+// ---- windowed detection on the stored green bits ----
+// One warp per sequence.  First the exclusive prefix counts of the sequence's bit words (32 words
+// per trip, warp scan, running carry), kept in `prefix` with the layout of the bits; then every
+// lane evaluates window starts lane, lane + 32, ...: greens in [start, start + w) is the
+// difference of two prefix counts, each one word load, one prefix load and a masked popcount.
+__device__ __forceinline__ int greens_before(const uint32_t *bits, const uint32_t *prefix, int p) {
+    const int word = p >> 5, bit = p & 31;
+    return static_cast<int>(prefix[word]) + (bit ? __popc(bits[word] & ((1u << bit) - 1u)) : 0);
+}
+
+__global__ void __launch_bounds__(kDetectThreads)
+window_kernel(const uint32_t *all_bits, uint32_t *all_prefix, const int32_t *lengths, const int64_t *offsets,
+              int64_t N, int64_t total_tokens, int W, int window, double gamma, int32_t *out_count,
+              int32_t *out_start, double *out_z) {
+    const int lane = threadIdx.x & 31;
+    const int64_t seq = static_cast<int64_t>(blockIdx.x) * (kDetectThreads / 32) + (threadIdx.x >> 5);
+    if (seq >= N) return;
+    const int64_t off = offsets[seq];
+    int64_t L = clamp_len(lengths[seq]);
+    if (off < 0 || off >= total_tokens) L = 0;
+    else if (off + L > total_tokens) L = total_tokens - off;
+    const int T = L > W ? static_cast<int>(L - W) : 0;
+    const uint32_t *bits = all_bits + (off >> 5) + 2 * seq;
+    uint32_t *prefix = all_prefix + (off >> 5) + 2 * seq;
+    const int nwords = (T + 31) >> 5;
+    // the region of a sequence has a word to spare: prefix[nwords] is written too, so that a
+    // window ending exactly at T needs no special case
+    unsigned carry = 0;
+    for (int k0 = 0; k0 <= nwords; k0 += 32) {
+        const int k = k0 + lane;
+        const unsigned c = k < nwords ? __popc(bits[k]) : 0u;
+        unsigned incl = c;
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned up = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += up;
+        }
+        if (k <= nwords) prefix[k] = carry + incl - c;
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    __syncwarp();
+    const int w = window < T ? window : T;
+    int best = 0, best_start = 0;
+    if (w > 0) {
+        for (int start = lane; start + w <= T; start += 32) {
+            const int g = greens_before(bits, prefix, start + w) - greens_before(bits, prefix, start);
+            if (g > best) { best = g; best_start = start; }       // strict: earliest start per lane
+        }
+        for (int d = 16; d > 0; d >>= 1) {
+            const int og = __shfl_down_sync(0xffffffffu, best, d);
+            const int os = __shfl_down_sync(0xffffffffu, best_start, d);
+            if (og > best || (og == best && os < best_start)) { best = og; best_start = os; }
+        }
+    }
+    if (lane == 0) {
+        out_count[seq] = best;
+        out_start[seq] = best > 0 ? best_start : 0;
+        double z = 0.0;
+        if (w > 0) {
+            const double num = __dsub_rn(static_cast<double>(best), __dmul_rn(gamma, static_cast<double>(w)));
+            const double var = __dmul_rn(__dmul_rn(static_cast<double>(w), gamma), __dsub_rn(1.0, gamma));
+            z = __ddiv_rn(num, __dsqrt_rn(var));
+        }
+        out_z[seq] = z;
+    }
+}
+
+}  // namespace
+}  // namespace sbw
+
+extern "C" int sbw_detect(const int32_t *tokens, const int32_t *lengths, const int64_t *offsets,
+                          int64_t N, int64_t total_tokens, int ctx_width, uint64_t key, double gamma,
+                          int scheme, int32_t *out_counts, int32_t *out_T, double *out_z,
+                          void *workspace, size_t workspace_bytes, void *stream) {
+    return sbw::detect_impl(tokens, lengths, offsets, N, total_tokens, ctx_width, key, gamma, scheme,
+                            out_counts, out_T, out_z, nullptr, workspace, workspace_bytes, stream);
+}
+
+extern "C" size_t sbw_detect_bits_words(int64_t N, int64_t total_tokens) {
+    if (N <= 0 || total_tokens < 0) return 0;
+    return static_cast<size_t>(total_tokens / 32 + 2 * N + 2);
+}
+
+extern "C" int sbw_detect_bits(const int32_t *tokens, const int32_t *lengths, const int64_t *offsets,
+                               int64_t N, int64_t total_tokens, int ctx_width, uint64_t key, double gamma,
+                               int scheme, int32_t *out_counts, int32_t *out_T, double *out_z,
+                               uint32_t *out_bits, void *workspace, size_t workspace_bytes, void *stream) {
+    if (N > 0 && !out_bits) return SBW_ERR_INVALID_ARG;
+    return sbw::detect_impl(tokens, lengths, offsets, N, total_tokens, ctx_width, key, gamma, scheme,
+                            out_counts, out_T, out_z, out_bits, workspace, workspace_bytes, stream);
+}
+
+extern "C" int sbw_window_z(const uint32_t *bits, const int32_t *lengths, const int64_t *offsets, int64_t N,
+                            int64_t total_tokens, int ctx_width, int64_t window, double gamma,
+                            uint32_t *prefix_scratch, int32_t *out_count, int32_t *out_start, double *out_z,
+                            void *stream) {
+    using namespace sbw;
+    if (ctx_width < 1 || ctx_width > SBW_MAX_CTX_WIDTH || !(gamma > 0.0 && gamma < 1.0)) return SBW_ERR_INVALID_ARG;
+    if (N < 0 || total_tokens < 0 || window < 1) return SBW_ERR_INVALID_ARG;
+    if (N == 0) return SBW_OK;
+    if (!bits || !lengths || !offsets || !prefix_scratch || !out_count || !out_start || !out_z)
+        return SBW_ERR_INVALID_ARG;
+    const int w = window > 0x7fffffffLL ? 0x7fffffff : static_cast<int>(window);
+    const unsigned grid = static_cast<unsigned>((N + kDetectThreads / 32 - 1) / (kDetectThreads / 32));
+    window_kernel<<<grid, kDetectThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        bits, prefix_scratch, lengths, offsets, N, total_tokens, ctx_width, w, gamma, out_count, out_start, out_z);
+    SBW_CUDA_TRY(cudaGetLastError());
     return SBW_OK;
 }
