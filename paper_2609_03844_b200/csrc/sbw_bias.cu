@@ -16,6 +16,8 @@
 // stream before it touches memory, so stream order is preserved.
 #include <cuda_bf16.h>
 
+#include <atomic>
+
 #include "sbw_common.cuh"
 #include "sbw_hash.cuh"
 
@@ -214,7 +216,7 @@ int launch(const BiasArgs &a, cudaStream_t stream) {
     DeviceInfo di;
     int rc = current_device_info(&di);
     if (rc != SBW_OK) return rc;
-    static int blocks_per_sm = 0;  // same kernel on every device of a process: B200 only
+    static std::atomic<int> blocks_per_sm{0};  // a property of the compiled kernel, equal on every sm_100a device
     if (blocks_per_sm == 0) {
         int n = 0;
         SBW_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, bias_kernel<DTYPE, SCHEME, VECTOR>,

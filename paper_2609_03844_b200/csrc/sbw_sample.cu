@@ -24,6 +24,7 @@
 // order.  The per-row finish (merging chunk partials, p = exp(.)/Z) is fp64.
 #include <cuda_bf16.h>
 
+#include <atomic>
 #include <cfloat>
 #include <climits>
 #include <mutex>
@@ -529,7 +530,7 @@ int launch_one(SampleArgs &a, int64_t nslot, size_t partial_bytes, cudaStream_t 
     DeviceInfo di;
     const int rc = current_device_info(&di);
     if (rc != SBW_OK) return rc;
-    static int blocks_per_sm = 0;
+    static std::atomic<int> blocks_per_sm{0};  // a property of the compiled kernel, equal on every sm_100a device
     if (blocks_per_sm == 0) {
         int n = 0;
         SBW_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, sample_kernel<DTYPE, SCHEME, VECTOR>,
