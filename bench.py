@@ -465,7 +465,7 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
     return out
 
 
-PROFILE_CASES = ("bias_bf16_context", "bias_bf16_selfsalt", "bias_fp32_context", "bias_fp32_selfsalt",
+PROFILE_CASES = ("topk40_fp32_selfsalt", "bias_bf16_context", "bias_bf16_selfsalt", "bias_fp32_context", "bias_fp32_selfsalt",
                  "detect_context", "detect_selfsalt", "sample_bf16_context", "sample_bf16_selfsalt")
 
 
@@ -493,7 +493,9 @@ def run_profile_case(name: str, launches: int) -> None:
         B, V, dtype = (512, V2, torch.bfloat16) if dt == "bf16" else (256, 151936, torch.float32)
         x = inputs.logits_normal(B, V, 4.0, dtype, seed=1, device=dev)
         ctx = inputs.uniform_tokens((B, 1), V, seed=2, device=dev)
-        if kind == "bias":
+        if kind == "topk40":
+            fn = lambda i: sbw.sbw_bias_logits_topk(x, ctx, KEY, 0.25, 4.0, scheme, 40)  # noqa: E731
+        elif kind == "bias":
             fn = lambda i: sbw.sbw_bias_logits(x, ctx, KEY, 0.5, 2.0, scheme)  # noqa: E731
         else:
             ids = torch.empty(B, dtype=torch.int32, device=dev)
