@@ -27,14 +27,10 @@ int bias_logits_impl(void *logits, int dtype, int64_t B, int64_t V, int64_t ld, 
 
 namespace {
 
-#ifndef SBW_TOPK_CTAS_PER_SM
-#define SBW_TOPK_CTAS_PER_SM 1
-#endif
-constexpr int kTopkThreads = 1024;
-constexpr int kTopkWarps = kTopkThreads / 32;
-constexpr int kGroups = kTopkThreads / 4;   // maxima of disjoint column sets used for the lower bound
+// CTA size: 1024 threads (one CTA per SM) when there are fewer rows than SMs can take two of,
+// 512 threads (two CTAs per SM, twice the rows in flight) for larger batches.
 constexpr int kCap = 2048;                  // candidate list entries
-constexpr int kPrefixPerThread = 32;        // columns per thread in the pass that finds the bound
+constexpr int kPrefixColumns = 32768;        // leading columns read by the pass that finds the bound
 
 struct TopkArgs {
     void *logits;
@@ -58,7 +54,7 @@ __device__ __forceinline__ uint64_t composite(uint32_t code, uint32_t col) {
 }
 
 // Calls f(column, code) for the columns of one row that this thread owns.
-template <int DTYPE, typename F>
+template <int DTYPE, int kTopkThreads, typename F>
 __device__ __forceinline__ void for_each_code(const char *row_ptr, uint32_t V, bool vector, F f) {
     // V here is the number of leading columns to visit (the whole row or a prefix of it)
     constexpr int VEC = DTYPE == SBW_DTYPE_F32 ? 4 : 8;
@@ -116,6 +112,7 @@ __device__ __noinline__ void bias_column(const TopkArgs &a, int64_t row, char *r
     }
 }
 
+template <int kTopkWarps>
 __device__ __forceinline__ uint64_t block_max_u64(uint64_t x, uint64_t *sh_red, uint64_t *sh_out) {
     for (int d = 16; d > 0; d >>= 1) {
         const uint64_t o = __shfl_xor_sync(0xffffffffu, x, d);
@@ -132,10 +129,12 @@ __device__ __forceinline__ uint64_t block_max_u64(uint64_t x, uint64_t *sh_red, 
     return *sh_out;
 }
 
-template <int DTYPE, int SCHEME>
+template <int DTYPE, int SCHEME, int kTopkThreads>
 __global__ void __launch_bounds__(kTopkThreads)
 topk_kernel(const TopkArgs a) {
     constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
+    constexpr int kTopkWarps = kTopkThreads / 32;
+    constexpr int kGroups = kTopkThreads / 4;   // maxima of disjoint column sets used for the lower bound
     __shared__ uint32_t sh_max[kGroups];
     __shared__ uint64_t sh_cand[kCap];
     __shared__ uint64_t sh_red[kTopkWarps];
@@ -149,9 +148,9 @@ topk_kernel(const TopkArgs a) {
         char *row_ptr = static_cast<char *>(a.logits) + row * a.ld * ESIZE;
 
         // 1. lower bound of the k-th largest code from a prefix of the row
-        const uint32_t prefix = min(V, static_cast<uint32_t>(kPrefixPerThread * kTopkThreads));
+        const uint32_t prefix = min(V, static_cast<uint32_t>(kPrefixColumns));
         uint32_t mx = 0;
-        for_each_code<DTYPE>(row_ptr, prefix, a.vector, [&](uint32_t, uint32_t code) { mx = max(mx, code); });
+        for_each_code<DTYPE, kTopkThreads>(row_ptr, prefix, a.vector, [&](uint32_t, uint32_t code) { mx = max(mx, code); });
         mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
         mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
         if ((threadIdx.x & 3) == 0) sh_max[threadIdx.x >> 2] = mx;
@@ -173,7 +172,7 @@ topk_kernel(const TopkArgs a) {
         const uint32_t floor_code = sh_floor;
 
         // 2. candidates: every column of the row that reaches the bound
-        for_each_code<DTYPE>(row_ptr, V, a.vector, [&](uint32_t col, uint32_t code) {
+        for_each_code<DTYPE, kTopkThreads>(row_ptr, V, a.vector, [&](uint32_t col, uint32_t code) {
             if (code >= floor_code) {
                 const unsigned pos = atomicAdd(&sh_count, 1u);
                 if (pos < kCap) sh_cand[pos] = composite(code, col);
@@ -199,14 +198,14 @@ topk_kernel(const TopkArgs a) {
             const uint32_t rounds = k < V ? k : V;
             for (uint32_t r = 0; r < rounds; ++r) {
                 uint64_t best = 0;
-                for_each_code<DTYPE>(row_ptr, V, a.vector, [&](uint32_t col, uint32_t code) {
+                for_each_code<DTYPE, kTopkThreads>(row_ptr, V, a.vector, [&](uint32_t col, uint32_t code) {
                     const uint64_t c = composite(code, col);
                     if ((r == 0 || c < prev) && c > best) best = c;
                 });
-                prev = block_max_u64(best, sh_red, &sh_best);
+                prev = block_max_u64<kTopkWarps>(best, sh_red, &sh_best);
             }
             const uint64_t kth = prev;
-            for_each_code<DTYPE>(row_ptr, V, a.vector, [&](uint32_t col, uint32_t code) {
+            for_each_code<DTYPE, kTopkThreads>(row_ptr, V, a.vector, [&](uint32_t col, uint32_t code) {
                 if (composite(code, col) >= kth) bias_column<DTYPE, SCHEME>(a, row, row_ptr, col);
             });
         }
@@ -219,9 +218,16 @@ int launch(const TopkArgs &a, cudaStream_t s) {
     DeviceInfo di;
     const int rc = current_device_info(&di);
     if (rc != SBW_OK) return rc;
-    const int64_t cap = static_cast<int64_t>(di.sm_count) * SBW_TOPK_CTAS_PER_SM;
-    const unsigned grid = static_cast<unsigned>(a.B < cap ? a.B : cap);
-    topk_kernel<DTYPE, SCHEME><<<grid, kTopkThreads, 0, s>>>(a);
+    // more rows than SMs: two 512-thread CTAs per SM keep twice as many rows in flight (that
+    // kernel has 128 groups, so its fast path needs k <= 128); otherwise one 1024-thread CTA per row
+    if (a.B > di.sm_count && a.k <= 128) {
+        const int64_t cap = static_cast<int64_t>(di.sm_count) * 2;
+        const unsigned grid = static_cast<unsigned>(a.B < cap ? a.B : cap);
+        topk_kernel<DTYPE, SCHEME, 512><<<grid, 512, 0, s>>>(a);
+    } else {
+        const unsigned grid = static_cast<unsigned>(a.B < di.sm_count ? a.B : di.sm_count);
+        topk_kernel<DTYPE, SCHEME, 1024><<<grid, 1024, 0, s>>>(a);
+    }
     SBW_CUDA_TRY(cudaGetLastError());
     return SBW_OK;
 }

@@ -90,3 +90,15 @@ def test_k_at_least_v_is_the_full_vocabulary_scheme_and_small_vocabularies():
     L = sbw.lib()
     assert L.sbw_bias_logits_topk(a.data_ptr(), 1, 3, 4096, 4096, 0, ctx.to(dev).data_ptr(), 1, KEY, 0.25, 2.0, 1,
                                   0, None) == -1
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("k", [40, 128, 200])
+def test_batches_larger_than_the_sm_count(dtype, k):
+    """More rows than SMs selects the 512-thread kernel (k <= 128) -- same results, incl. ties."""
+    B, V = 200, 20011
+    x = inputs.logits_normal(B, V, 4.0, dtype, seed=81)
+    x[3, :] = 2.5
+    x[7, 1000:] = float("-inf")
+    ctx = inputs.uniform_tokens((B, 4), V, seed=82)
+    _check(x, V, ctx, KEY, 0.25, 2.0, sbw.SCHEME_SELFSALT, k)
