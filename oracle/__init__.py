@@ -83,6 +83,12 @@ def lib() -> ctypes.CDLL:
         L.sbw_oracle_detect_bits.argtypes = [vp, vp, i64, i32, u64, c.c_double, i32, vp]
         L.sbw_oracle_window_z.restype = None
         L.sbw_oracle_window_z.argtypes = [vp, vp, i64, i32, i64, c.c_double, vp, vp, vp]
+        L.sbw_oracle_detect_unique.restype = None
+        L.sbw_oracle_detect_unique.argtypes = [vp, vp, i64, i32, u64, c.c_double, i32, vp, vp, vp, i32]
+        L.sbw_oracle_prefix_z.restype = None
+        L.sbw_oracle_prefix_z.argtypes = [vp, vp, vp, i64, i32, c.c_double, vp, vp, vp]
+        L.sbw_oracle_roc_auc.restype = c.c_double
+        L.sbw_oracle_roc_auc.argtypes = [vp, vp, i64, vp, i32]
         L.sbw_oracle_zscore.restype = c.c_double
         L.sbw_oracle_zscore.argtypes = [i64, i64, c.c_double]
         L.sbw_oracle_log.restype = c.c_float
@@ -211,6 +217,43 @@ def window_z(green, lengths, window, gamma, ctx_width=1):
     bz = np.zeros(N, dtype=np.float64)
     lib().sbw_oracle_window_z(_ptr(g), _ptr(lens), N, ctx_width, window, gamma, _ptr(bc), _ptr(bs), _ptr(bz))
     return bc, bs, bz
+
+
+def detect_unique(tokens, lengths, key, gamma, scheme, ctx_width=1, threads=1):
+    """Detection that scores each distinct (context, token) tuple once: (counts, T, z)."""
+    tok = np.ascontiguousarray(np.asarray(tokens, dtype=np.int32))
+    lens = np.ascontiguousarray(np.asarray(lengths, dtype=np.int32))
+    N = lens.shape[0]
+    counts = np.zeros(N, dtype=np.int32)
+    T = np.zeros(N, dtype=np.int32)
+    z = np.zeros(N, dtype=np.float64)
+    lib().sbw_oracle_detect_unique(_ptr(tok), _ptr(lens), N, ctx_width, key, gamma, scheme,
+                                   _ptr(counts), _ptr(T), _ptr(z), threads)
+    return counts, T, z
+
+
+def prefix_z(green, lengths, keep, gamma, ctx_width=1):
+    """Detection on the first ``keep[s]`` tokens of each sequence: (counts, T, z)."""
+    g = np.ascontiguousarray(np.asarray(green, dtype=np.uint8))
+    lens = np.ascontiguousarray(np.asarray(lengths, dtype=np.int32))
+    kp = np.ascontiguousarray(np.asarray(keep, dtype=np.int32))
+    N = lens.shape[0]
+    counts = np.zeros(N, dtype=np.int32)
+    T = np.zeros(N, dtype=np.int32)
+    z = np.zeros(N, dtype=np.float64)
+    lib().sbw_oracle_prefix_z(_ptr(g), _ptr(lens), _ptr(kp), N, ctx_width, gamma, _ptr(counts),
+                              _ptr(T), _ptr(z))
+    return counts, T, z
+
+
+def roc_auc(z, labels, threads=1):
+    """ROC-AUC of z against 0/1 labels and the pair statistics {greater, equal, n_pos, n_neg}."""
+    zz = np.ascontiguousarray(np.asarray(z, dtype=np.float64))
+    lb = np.ascontiguousarray(np.asarray(labels, dtype=np.uint8))
+    assert zz.shape == lb.shape and zz.ndim == 1
+    stats = np.zeros(4, dtype=np.uint64)
+    auc = float(lib().sbw_oracle_roc_auc(_ptr(zz), _ptr(lb), zz.shape[0], _ptr(stats), threads))
+    return auc, stats
 
 
 def zscore(G: int, T: int, gamma: float) -> float:

@@ -367,6 +367,118 @@ void sbw_oracle_window_z(const uint8_t *green, const int32_t *lengths, int64_t N
     }
 }
 
+/* Detection that scores every distinct (context, token) tuple of a sequence once -- the option
+ * KGW-family detectors call "ignore repeated n-grams" (Section 3 takes the Y_t as independent;
+ * repeated text repeats the same trial).  Position t >= W counts iff no earlier scored position
+ * t' in [W, t) has tok[t'-W .. t'] equal to tok[t-W .. t] element by element; T is the number of
+ * such positions, G the green ones among them; Eq. 5 on (G, T). */
+void sbw_oracle_detect_unique(const int32_t *tokens, const int32_t *lengths, int64_t N, int ctx_width,
+                              uint64_t key, double gamma, int scheme, int32_t *counts, int32_t *T,
+                              double *z, int threads)
+{
+    uint64_t thr = sbw_oracle_threshold(gamma);
+    int64_t *offsets = (int64_t *)malloc((size_t)(N + 1) * sizeof(int64_t));
+    if (!offsets)
+        return;
+    offsets[0] = 0;
+    for (int64_t s = 0; s < N; ++s)
+        offsets[s + 1] = offsets[s] + (lengths[s] > 0 ? lengths[s] : 0);
+    if (threads < 1)
+        threads = 1;
+#pragma omp parallel for num_threads(threads) schedule(dynamic, 16)
+    for (int64_t s = 0; s < N; ++s) {
+        const int32_t *tok = tokens + offsets[s];
+        int64_t L = lengths[s] > 0 ? lengths[s] : 0;
+        int64_t G = 0, Tu = 0;
+        for (int64_t t = ctx_width; t < L; ++t) {
+            int seen = 0;
+            for (int64_t e = ctx_width; e < t && !seen; ++e) {
+                int same = 1;
+                for (int i = 0; i <= ctx_width; ++i)
+                    if (tok[e - i] != tok[t - i])
+                        same = 0;
+                seen = same;
+            }
+            if (seen)
+                continue;
+            uint32_t v = (uint32_t)tok[t];
+            uint64_t r = seed_for(scheme, key, tok + (t - ctx_width), ctx_width, v);
+            G += sbw_oracle_green(r, v, thr);
+            Tu += 1;
+        }
+        counts[s] = (int32_t)G;
+        if (T)
+            T[s] = (int32_t)Tu;
+        z[s] = sbw_oracle_zscore(G, Tu, gamma);
+    }
+    free(offsets);
+}
+
+/* Detection on a truncated copy of each sequence (the truncation attacks of Appendix G keep a
+ * prefix of the text): only the first keep[s] tokens of sequence s count, keep clamped to
+ * [0, length].  green is the per-token array sbw_oracle_detect_bits wrote for the whole text. */
+void sbw_oracle_prefix_z(const uint8_t *green, const int32_t *lengths, const int32_t *keep, int64_t N,
+                         int ctx_width, double gamma, int32_t *counts, int32_t *T, double *z)
+{
+    int64_t off = 0;
+    for (int64_t s = 0; s < N; ++s) {
+        int64_t L = lengths[s] > 0 ? lengths[s] : 0;
+        int64_t K = keep[s] < 0 ? 0 : (keep[s] > L ? L : keep[s]);
+        int64_t G = 0;
+        for (int64_t t = ctx_width; t < K; ++t)
+            G += green[off + t];
+        int64_t Tk = K > ctx_width ? K - ctx_width : 0;
+        counts[s] = (int32_t)G;
+        if (T)
+            T[s] = (int32_t)Tk;
+        z[s] = sbw_oracle_zscore(G, Tk, gamma);
+        off += L;
+    }
+}
+
+/* Section 4.4: area under the ROC curve of the z-score as a detector of label 1 against label 0,
+ * written as the probability that a watermarked text outscores an unmarked one, ties counting a
+ * half (equal to the trapezoid area under the curve swept over all thresholds).  NaN scores are
+ * left out of both classes.  stats (nullable) receives {pairs with z_pos > z_neg, pairs with
+ * z_pos == z_neg, n_pos, n_neg}.  Returns NaN when a class is empty. */
+double sbw_oracle_roc_auc(const double *z, const uint8_t *labels, int64_t n, uint64_t stats[4], int threads)
+{
+    uint64_t greater = 0, equal = 0, npos = 0, nneg = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        if (z[i] != z[i])
+            continue;
+        if (labels[i])
+            npos += 1;
+        else
+            nneg += 1;
+    }
+    if (threads < 1)
+        threads = 1;
+#pragma omp parallel for num_threads(threads) reduction(+ : greater, equal) schedule(static)
+    for (int64_t i = 0; i < n; ++i) {
+        if (!labels[i] || z[i] != z[i])
+            continue;
+        for (int64_t j = 0; j < n; ++j) {
+            if (labels[j] || z[j] != z[j])
+                continue;
+            if (z[i] > z[j])
+                greater += 1;
+            else if (z[i] == z[j])
+                equal += 1;
+        }
+    }
+    if (stats) {
+        stats[0] = greater;
+        stats[1] = equal;
+        stats[2] = npos;
+        stats[3] = nneg;
+    }
+    if (npos == 0 || nneg == 0)
+        return NAN;
+    /* (2 greater + equal) / (2 npos nneg): numerator and denominator are exact integers */
+    return (double)(2 * greater + equal) / (double)(2 * npos * nneg);
+}
+
 /* ------------------------------------------------------------------ R8: sampler ---- */
 /*
  * Specified fp32 natural logarithm for positive normal x (every step one IEEE operation):

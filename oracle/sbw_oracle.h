@@ -18,6 +18,9 @@
  *   bias add           pinned: numpy float32 / torch bfloat16 adds           (test_oracle_bias)
  *   top-k restriction  pinned: torch.topk, brute force on ties, k >= V case  (test_oracle_topk)
  *   detect             pinned: brute force, closed forms, null law of Eq. 5  (test_oracle_detect)
+ *   detect_unique,     pinned: Python set of tuples, closed forms; slices of  (test_oracle_eval)
+ *   prefix_z, roc_auc  the plain detector; scikit-learn's roc_auc_score,
+ *                      exact threshold sweep in rationals, binormal closed form
  *   log / gumbel /     pinned: fp64 log, chi-square of sampled ids against    (test_oracle_sample)
  *   sample             softmax, scipy softmax / logsumexp, closed form
  *   bit compatibility with the paper authors' own package: PARITY UNPINNED (the paper
@@ -100,6 +103,18 @@ void sbw_oracle_detect_bits(const int32_t *tokens, const int32_t *lengths, int64
 void sbw_oracle_window_z(const uint8_t *green, const int32_t *lengths, int64_t N, int ctx_width,
                          int64_t window, double gamma, int32_t *best_count, int32_t *best_start,
                          double *best_z);
+/* "Ignore repeated n-grams" detection: every distinct (context, token) tuple of a sequence is
+ * scored once; T counts the distinct tuples, counts the green ones among them. */
+void sbw_oracle_detect_unique(const int32_t *tokens, const int32_t *lengths, int64_t N, int ctx_width,
+                              uint64_t key, double gamma, int scheme, int32_t *counts, int32_t *T,
+                              double *z, int threads);
+/* Detection on the first keep[s] tokens of each sequence (truncated text, Appendix G), from the
+ * per-token array of sbw_oracle_detect_bits. */
+void sbw_oracle_prefix_z(const uint8_t *green, const int32_t *lengths, const int32_t *keep, int64_t N,
+                         int ctx_width, double gamma, int32_t *counts, int32_t *T, double *z);
+/* Section 4.4: ROC-AUC of z against binary labels = P(z_pos > z_neg) + P(z_pos == z_neg) / 2 over
+ * all (positive, negative) pairs.  stats (nullable): {greater, equal, n_pos, n_neg}. */
+double sbw_oracle_roc_auc(const double *z, const uint8_t *labels, int64_t n, uint64_t stats[4], int threads);
 /* Eq. 5 alone. */
 double sbw_oracle_zscore(int64_t G, int64_t T, double gamma);
 
