@@ -262,6 +262,54 @@ int sbw_window_z(const uint32_t *bits, const int32_t *lengths, const int64_t *of
                  uint32_t *prefix_scratch, int32_t *out_count, int32_t *out_start, double *out_z,
                  void *stream);
 
+/*
+ * sbw_prefix_z -- detection on truncated text (the paper's robustness study, Appendix G, cuts
+ * text to a prefix): Eq. 5 over the first keep[s] tokens of sequence s only, from the bits
+ * sbw_detect_bits stored.  keep is clamped to [0, length]; T = max(keep - W, 0); T = 0 gives z 0.
+ *   bits, lengths, offsets (required, device), total_tokens, ctx_width  as used by sbw_detect_bits.
+ *   keep        device [N] int32.
+ *   out_counts  device [N] int32;  out_T  device [N] int32 or NULL;  out_z  device [N] double.
+ */
+int sbw_prefix_z(const uint32_t *bits, const int32_t *lengths, const int64_t *offsets, const int32_t *keep,
+                 int64_t N, int64_t total_tokens, int ctx_width, double gamma, int32_t *out_counts,
+                 int32_t *out_T, double *out_z, void *stream);
+
+/*
+ * sbw_detect_unique -- sbw_detect that scores every distinct (context, token) tuple of a sequence
+ * once (what KGW-family detectors call "ignore repeated n-grams"; Section 3 of the paper treats the
+ * indicators Y_i as independent trials, which repeated text is not).  A scored position t counts
+ * iff no earlier scored position of the same sequence has the same W + 1 tokens tok[t-W .. t];
+ * out_T is the number of such positions, out_counts the green ones among them, out_z Eq. 5 on
+ * the two.  Arguments as for sbw_detect, plus
+ *   max_length  an upper bound on every length.  Sequences with more than 1536 scored tokens keep
+ *               their hash set in the workspace; the workspace holds room for that only if
+ *               max_length says such sequences exist.  A sequence longer than max_length that
+ *               needs that room is not scored: count -1, T -1, z NaN.
+ *   workspace   device, 256-byte aligned, at least
+ *               sbw_detect_unique_workspace_bytes(N, total_tokens, max_length) bytes (always
+ *               required; 16 bytes per token more when max_length > 1537).
+ */
+size_t sbw_detect_unique_workspace_bytes(int64_t N, int64_t total_tokens, int64_t max_length);
+int sbw_detect_unique(const int32_t *tokens, const int32_t *lengths, const int64_t *offsets, int64_t N,
+                      int64_t total_tokens, int64_t max_length, int ctx_width, uint64_t key, double gamma,
+                      int scheme, int32_t *out_counts, int32_t *out_T, double *out_z, void *workspace,
+                      size_t workspace_bytes, void *stream);
+
+/*
+ * sbw_roc_auc -- Section 4.4: area under the ROC curve of z-scores as a detector of label 1
+ * (watermarked) against label 0, computed exactly as the pair statistic
+ *   AUC = (2 #{z_pos > z_neg} + #{z_pos == z_neg}) / (2 n_pos n_neg),
+ * which equals the trapezoid area under the (FPR, TPR) curve swept over every threshold.  NaN
+ * scores are left out of both classes; -0 and +0 tie.
+ *   z          device [n] double;  labels  device [n] uint8 (0 or non-zero);  n <= 2^31.
+ *   out_auc    device double[1]; NaN when a class is empty.
+ *   out_stats  device uint64[4] or NULL: {pairs greater, pairs equal, n_pos, n_neg}.
+ *   workspace  device, 256-byte aligned, at least sbw_roc_auc_workspace_bytes(n) bytes.
+ */
+size_t sbw_roc_auc_workspace_bytes(int64_t n);
+int sbw_roc_auc(const double *z, const uint8_t *labels, int64_t n, double *out_auc, uint64_t *out_stats,
+                void *workspace, size_t workspace_bytes, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

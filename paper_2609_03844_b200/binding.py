@@ -30,7 +30,8 @@ EXPORTS = ("sbw_version", "sbw_last_cuda_error", "sbw_bias_logits",
            "sbw_sample_workspace_bytes", "sbw_bias_sample", "sbw_detect_workspace_bytes",
            "sbw_detect", "sbw_int_probe", "sbw_bias_sample_noalloc", "sbw_bias_logits_topk",
            "sbw_bias_sample_shard", "sbw_sample_combine", "sbw_detect_bits_words", "sbw_detect_bits",
-           "sbw_window_z")
+           "sbw_window_z", "sbw_prefix_z", "sbw_detect_unique_workspace_bytes", "sbw_detect_unique",
+           "sbw_roc_auc_workspace_bytes", "sbw_roc_auc")
 
 _lib = None
 
@@ -102,6 +103,17 @@ def lib() -> ctypes.CDLL:
                                       sz, vp]
         L.sbw_window_z.restype = i32
         L.sbw_window_z.argtypes = [vp, vp, vp, i64, i64, i32, i64, c.c_double, vp, vp, vp, vp, vp]
+        L.sbw_prefix_z.restype = i32
+        L.sbw_prefix_z.argtypes = [vp, vp, vp, vp, i64, i64, i32, c.c_double, vp, vp, vp, vp]
+        L.sbw_detect_unique_workspace_bytes.restype = sz
+        L.sbw_detect_unique_workspace_bytes.argtypes = [i64, i64, i64]
+        L.sbw_detect_unique.restype = i32
+        L.sbw_detect_unique.argtypes = [vp, vp, vp, i64, i64, i64, i32, u64, c.c_double, i32, vp, vp, vp,
+                                        vp, sz, vp]
+        L.sbw_roc_auc_workspace_bytes.restype = sz
+        L.sbw_roc_auc_workspace_bytes.argtypes = [i64]
+        L.sbw_roc_auc.restype = i32
+        L.sbw_roc_auc.argtypes = [vp, vp, i64, vp, vp, vp, sz, vp]
         L.sbw_int_probe.restype = i32
         L.sbw_int_probe.argtypes = [i32, i32, i32, i32, vp, vp, vp]
         _lib = L
@@ -344,6 +356,62 @@ def sbw_window_z(bits: torch.Tensor, lengths: torch.Tensor, offsets: torch.Tenso
                             _stream(stream))
     _check("sbw_window_z", rc)
     return out_count, out_start, out_z
+
+
+def sbw_prefix_z(bits: torch.Tensor, lengths: torch.Tensor, offsets: torch.Tensor, keep: torch.Tensor,
+                 total_tokens: int, gamma: float, out_counts: torch.Tensor, out_z: torch.Tensor, *,
+                 out_T: torch.Tensor | None = None, ctx_width: int = 1, stream=None):
+    """Detection on the first ``keep[s]`` tokens of each sequence, from stored green bits."""
+    N = lengths.numel()
+    if offsets.dtype != torch.int64 or offsets.numel() < N + 1:
+        raise TypeError("offsets must be int64 with N + 1 entries")
+    if keep.dtype != torch.int32 or keep.numel() != N:
+        raise TypeError("keep must be int32 with N entries")
+    rc = lib().sbw_prefix_z(_ptr(bits), _ptr(lengths), _ptr(offsets), _ptr(keep), N, total_tokens, ctx_width,
+                            gamma, _ptr(out_counts), _ptr(out_T), _ptr(out_z), _stream(stream))
+    _check("sbw_prefix_z", rc)
+    return out_counts, out_z
+
+
+def sbw_detect_unique_workspace_bytes(N: int, total_tokens: int, max_length: int) -> int:
+    return int(lib().sbw_detect_unique_workspace_bytes(N, total_tokens, max_length))
+
+
+def sbw_detect_unique(tokens: torch.Tensor, lengths: torch.Tensor, max_length: int, key: int, gamma: float,
+                      scheme: int, out_counts: torch.Tensor, out_z: torch.Tensor, workspace: torch.Tensor, *,
+                      out_T: torch.Tensor | None = None, offsets: torch.Tensor | None = None,
+                      ctx_width: int = 1, stream=None):
+    """Batch detection that scores each distinct (context, token) tuple of a sequence once."""
+    N = lengths.numel()
+    if tokens.dtype != torch.int32 or lengths.dtype != torch.int32:
+        raise TypeError("tokens and lengths must be int32")
+    if out_counts.dtype != torch.int32 or out_z.dtype != torch.float64:
+        raise TypeError("out_counts must be int32 and out_z float64")
+    if offsets is not None and (offsets.dtype != torch.int64 or offsets.numel() != N + 1):
+        raise TypeError("offsets must be int64 with N + 1 entries")
+    rc = lib().sbw_detect_unique(_ptr(tokens), _ptr(lengths), _ptr(offsets), N, tokens.numel(), max_length,
+                                 ctx_width, key, gamma, scheme, _ptr(out_counts), _ptr(out_T), _ptr(out_z),
+                                 _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                 _stream(stream))
+    _check("sbw_detect_unique", rc)
+    return out_counts, out_z
+
+
+def sbw_roc_auc_workspace_bytes(n: int) -> int:
+    return int(lib().sbw_roc_auc_workspace_bytes(n))
+
+
+def sbw_roc_auc(z: torch.Tensor, labels: torch.Tensor, out_auc: torch.Tensor, workspace: torch.Tensor, *,
+                out_stats: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """ROC-AUC of float64 scores against uint8 labels into ``out_auc`` (float64[1], CUDA)."""
+    if z.dtype != torch.float64 or labels.dtype != torch.uint8 or z.numel() != labels.numel():
+        raise TypeError("z must be float64 and labels uint8, of equal length")
+    if out_auc.dtype != torch.float64 or (out_stats is not None and out_stats.dtype != torch.int64):
+        raise TypeError("out_auc must be float64 and out_stats int64 (four 64-bit counters)")
+    rc = lib().sbw_roc_auc(_ptr(z), _ptr(labels), z.numel(), _ptr(out_auc), _ptr(out_stats), _ptr(workspace),
+                           workspace.numel() * workspace.element_size(), _stream(stream))
+    _check("sbw_roc_auc", rc)
+    return out_auc
 
 
 PROBE_KINDS = {"mulwide": (0, 1), "lop3": (1, 1), "iadd3": (2, 1), "imad": (3, 1), "philox": (4, 4),

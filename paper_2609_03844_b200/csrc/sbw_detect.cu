@@ -48,6 +48,14 @@ struct DetectArgs {
 
 __device__ __forceinline__ int64_t clamp_len(int32_t l) { return l > 0 ? l : 0; }
 
+// Eq. 5, every operation rounded separately; 0 where it is 0/0.
+__device__ __forceinline__ double zscore(int G, int T, double gamma) {
+    if (T <= 0) return 0.0;
+    const double num = __dsub_rn(static_cast<double>(G), __dmul_rn(gamma, static_cast<double>(T)));
+    const double var = __dmul_rn(__dmul_rn(static_cast<double>(T), gamma), __dsub_rn(1.0, gamma));
+    return __ddiv_rn(num, __dsqrt_rn(var));
+}
+
 // ---- exclusive scan of the lengths: tile sums, then per-tile scan with a look-back sum ----
 __global__ void __launch_bounds__(kScanThreads)
 scan_tile_sums(const int32_t *lengths, int64_t N, int64_t *tile_sums) {
@@ -116,16 +124,15 @@ scan_offsets(const int32_t *lengths, int64_t N, const int64_t *tile_sums, int64_
 }
 
 // ---- the detector ----
-// Scores the kDetectIlp * 32 positions base + u*32 + lane (u = 0..kDetectIlp-1) of one sequence.
-// TAIL = false: every position is inside the sequence, no masking.  WIDTH > 0 fixes the context
-// width at compile time (loops unrolled), WIDTH = 0 reads it from the arguments.
+// A trip covers the kDetectIlp * 32 positions base + u*32 + lane (u = 0..kDetectIlp-1) of one
+// sequence.  TAIL = false: every position is inside the sequence, no masking.  WIDTH > 0 fixes the
+// context width at compile time (loops unrolled), WIDTH = 0 reads it from the arguments.
+// load_trip reads the tokens and derives their seeds; score_trip hashes them and counts.
 template <int SCHEME, int WIDTH, bool TAIL>
-__device__ __forceinline__ int score_trip(const DetectArgs &a, const int32_t *tok, int base, int len,
-                                          int lane, uint32_t *bits) {
+__device__ __forceinline__ void load_trip(const DetectArgs &a, const int32_t *tok, int base, int len, int lane,
+                                          uint32_t (&v)[kDetectIlp], uint64_t (&r)[kDetectIlp],
+                                          bool (&valid)[kDetectIlp]) {
     const int width = WIDTH > 0 ? WIDTH : a.W;
-    uint32_t v[kDetectIlp];
-    uint64_t r[kDetectIlp];
-    bool valid[kDetectIlp];
 #pragma unroll
     for (int u = 0; u < kDetectIlp; ++u) {
         const int t = base + u * 32 + lane;
@@ -150,6 +157,16 @@ __device__ __forceinline__ int score_trip(const DetectArgs &a, const int32_t *to
             r[u] = seed_selfsalt(a.key, jmin, v[u]);
         }
     }
+}
+
+template <int SCHEME, int WIDTH, bool TAIL>
+__device__ __forceinline__ int score_trip(const DetectArgs &a, const int32_t *tok, int base, int len,
+                                          int lane, uint32_t *bits) {
+    const int width = WIDTH > 0 ? WIDTH : a.W;
+    uint32_t v[kDetectIlp];
+    uint64_t r[kDetectIlp];
+    bool valid[kDetectIlp];
+    load_trip<SCHEME, WIDTH, TAIL>(a, tok, base, len, lane, v, r, valid);
     uint32_t x[kDetectIlp];
     philox_word0_n<kDetectIlp>(v, r, x, a.weyl);
     int count = 0;
@@ -190,14 +207,7 @@ detect_kernel(const DetectArgs a) {
         const int T = len > width ? len - width : 0;
         a.out_counts[seq] = count;
         if (a.out_T) a.out_T[seq] = T;
-        double z = 0.0;
-        if (T > 0) {
-            // Eq. 5, every operation rounded separately
-            const double num = __dsub_rn(static_cast<double>(count), __dmul_rn(a.gamma, static_cast<double>(T)));
-            const double var = __dmul_rn(__dmul_rn(static_cast<double>(T), a.gamma), __dsub_rn(1.0, a.gamma));
-            z = __ddiv_rn(num, __dsqrt_rn(var));
-        }
-        a.out_z[seq] = z;
+        a.out_z[seq] = zscore(count, T, a.gamma);
     }
 }
 
@@ -223,6 +233,20 @@ extern "C" size_t sbw_detect_workspace_bytes(int64_t N) {
 
 namespace sbw {
 namespace {
+// Exclusive scan of the lengths into the start of `workspace` (int64[N + 1], then the tile sums).
+int scan_lengths(const int32_t *lengths, int64_t N, void *workspace, int64_t **out_offsets, cudaStream_t s) {
+    int64_t *ws_offsets = static_cast<int64_t *>(workspace);
+    int64_t *tile_sums = reinterpret_cast<int64_t *>(
+        static_cast<char *>(workspace) + align_up((static_cast<size_t>(N) + 1) * sizeof(int64_t), 256));
+    const unsigned tiles = static_cast<unsigned>((N + kScanTile - 1) / kScanTile);
+    scan_tile_sums<<<tiles, kScanThreads, 0, s>>>(lengths, N, tile_sums);
+    SBW_CUDA_TRY(cudaGetLastError());
+    scan_offsets<<<tiles, kScanThreads, 0, s>>>(lengths, N, tile_sums, ws_offsets);
+    SBW_CUDA_TRY(cudaGetLastError());
+    *out_offsets = ws_offsets;
+    return SBW_OK;
+}
+
 int detect_impl(const int32_t *tokens, const int32_t *lengths, const int64_t *offsets, int64_t N,
                 int64_t total_tokens, int ctx_width, uint64_t key, double gamma, int scheme,
                 int32_t *out_counts, int32_t *out_T, double *out_z, uint32_t *out_bits, void *workspace,
@@ -255,14 +279,9 @@ int detect_impl(const int32_t *tokens, const int32_t *lengths, const int64_t *of
         const size_t need = sbw_detect_workspace_bytes(N);
         if (!workspace || workspace_bytes < need || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
             return SBW_ERR_WORKSPACE;
-        int64_t *ws_offsets = static_cast<int64_t *>(workspace);
-        int64_t *tile_sums = reinterpret_cast<int64_t *>(
-            static_cast<char *>(workspace) + align_up((static_cast<size_t>(N) + 1) * sizeof(int64_t), 256));
-        const unsigned tiles = static_cast<unsigned>((N + kScanTile - 1) / kScanTile);
-        scan_tile_sums<<<tiles, kScanThreads, 0, s>>>(lengths, N, tile_sums);
-        SBW_CUDA_TRY(cudaGetLastError());
-        scan_offsets<<<tiles, kScanThreads, 0, s>>>(lengths, N, tile_sums, ws_offsets);
-        SBW_CUDA_TRY(cudaGetLastError());
+        int64_t *ws_offsets = nullptr;
+        const int rc = scan_lengths(lengths, N, workspace, &ws_offsets, s);
+        if (rc != SBW_OK) return rc;
         a.offsets = ws_offsets;
     }
     const unsigned grid = static_cast<unsigned>((N + kDetectThreads / 32 - 1) / (kDetectThreads / 32));
@@ -327,14 +346,165 @@ window_kernel(const uint32_t *all_bits, uint32_t *all_prefix, const int32_t *len
     if (lane == 0) {
         out_count[seq] = best;
         out_start[seq] = best > 0 ? best_start : 0;
-        double z = 0.0;
-        if (w > 0) {
-            const double num = __dsub_rn(static_cast<double>(best), __dmul_rn(gamma, static_cast<double>(w)));
-            const double var = __dmul_rn(__dmul_rn(static_cast<double>(w), gamma), __dsub_rn(1.0, gamma));
-            z = __ddiv_rn(num, __dsqrt_rn(var));
-        }
-        out_z[seq] = z;
+        out_z[seq] = zscore(best, w, gamma);
     }
+}
+
+
+// ---- detection on truncated text: popcount of the first kept bits ----
+__global__ void __launch_bounds__(kDetectThreads)
+prefix_kernel(const uint32_t *all_bits, const int32_t *lengths, const int64_t *offsets, const int32_t *keep,
+              int64_t N, int64_t total_tokens, int W, double gamma, int32_t *out_count, int32_t *out_T,
+              double *out_z) {
+    const int lane = threadIdx.x & 31;
+    const int64_t seq = static_cast<int64_t>(blockIdx.x) * (kDetectThreads / 32) + (threadIdx.x >> 5);
+    if (seq >= N) return;
+    const int64_t off = offsets[seq];
+    int64_t L = clamp_len(lengths[seq]);
+    if (off < 0 || off >= total_tokens) L = 0;
+    else if (off + L > total_tokens) L = total_tokens - off;
+    int64_t K = clamp_len(keep[seq]);
+    if (K > L) K = L;
+    const int T = K > W ? static_cast<int>(K - W) : 0;
+    const uint32_t *bits = all_bits + (off >> 5) + 2 * seq;
+    const int nfull = T >> 5, rem = T & 31;
+    int count = 0;
+    for (int k = lane; k < nfull; k += 32) count += __popc(bits[k]);
+    if (lane == 0 && rem) count += __popc(bits[nfull] & ((1u << rem) - 1u));
+    for (int d = 16; d > 0; d >>= 1) count += __shfl_down_sync(0xffffffffu, count, d);
+    if (lane == 0) {
+        out_count[seq] = count;
+        if (out_T) out_T[seq] = T;
+        out_z[seq] = zscore(count, T, gamma);
+    }
+}
+
+// ---- detection over the distinct (context, token) tuples of a sequence ----
+// One warp per sequence, as in detect_kernel, plus a hash set of the tuples seen so far: open
+// addressing with linear probing over a power-of-two table of token positions (0 = empty; scored
+// positions start at W >= 1).  A lane claims a slot with one compare-and-swap; a lane that finds
+// the slot taken compares its tuple with the tuple at the stored position and either stops
+// (duplicate) or probes on.  Entries are never removed, so concurrent inserts by the lanes of
+// the warp are safe: whichever lane claims a tuple first, every other occurrence meets it on its
+// probe path.  Which occurrence represents a tuple does not matter -- equal tuples have equal
+// green bits -- so counts are deterministic.  The table lives in shared memory (kUniqueSlots
+// slots per warp) for sequences with at most kUniqueSmemMaxT scored tokens, otherwise in the
+// caller's workspace at 4 * offset (the smallest power of two >= 2T is below 4T slots).
+constexpr int kUniqueSlots = 2048;
+constexpr int kUniqueSmemMaxT = 1536;
+
+template <int WIDTH>
+__device__ __forceinline__ uint32_t tuple_hash(const int32_t *tok, int t, int width) {
+    uint32_t h = static_cast<uint32_t>(tok[t]) * 0x9E3779B1u;
+#pragma unroll
+    for (int i = 1; i <= (WIDTH > 0 ? WIDTH : SBW_MAX_CTX_WIDTH); ++i)
+        if (i <= width) h = (h + static_cast<uint32_t>(tok[t - i])) * 0x85EBCA77u;
+    return (h ^ (h >> 15)) * 0x9E3779B1u;
+}
+
+template <int WIDTH>
+__device__ __forceinline__ bool same_tuple(const int32_t *tok, int p, int q, int width) {
+    bool same = true;
+#pragma unroll
+    for (int i = 0; i <= (WIDTH > 0 ? WIDTH : SBW_MAX_CTX_WIDTH); ++i)
+        if (i <= width) same = same && tok[p - i] == tok[q - i];
+    return same;
+}
+
+// true if position t is the one that enters its tuple into the set
+template <int WIDTH>
+__device__ __forceinline__ bool insert_tuple(uint32_t *table, uint32_t mask, int shift, const int32_t *tok,
+                                             int t, int width) {
+    uint32_t slot = tuple_hash<WIDTH>(tok, t, width) >> shift;
+    for (uint32_t n = 0; n <= mask; ++n) {           // bounded: the table always has a free slot
+        const uint32_t prev = atomicCAS(&table[slot], 0u, static_cast<uint32_t>(t));
+        if (prev == 0u) return true;
+        if (same_tuple<WIDTH>(tok, static_cast<int>(prev), t, width)) return false;
+        slot = (slot + 1u) & mask;
+    }
+    return true;
+}
+
+template <int SCHEME, int WIDTH, bool TAIL>
+__device__ __forceinline__ void unique_trip(const DetectArgs &a, const int32_t *tok, int base, int len, int lane,
+                                            uint32_t *table, uint32_t mask, int shift, int &count, int &distinct) {
+    const int width = WIDTH > 0 ? WIDTH : a.W;
+    uint32_t v[kDetectIlp];
+    uint64_t r[kDetectIlp];
+    bool first[kDetectIlp];
+    load_trip<SCHEME, WIDTH, TAIL>(a, tok, base, len, lane, v, r, first);
+#pragma unroll
+    for (int u = 0; u < kDetectIlp; ++u)
+        first[u] = first[u] && insert_tuple<WIDTH>(table, mask, shift, tok, base + u * 32 + lane, width);
+    uint32_t x[kDetectIlp];
+    philox_word0_n<kDetectIlp>(v, r, x, a.weyl);
+#pragma unroll
+    for (int u = 0; u < kDetectIlp; ++u) {
+        distinct += __popc(__ballot_sync(0xffffffffu, first[u]));
+        count += __popc(__ballot_sync(0xffffffffu, first[u] && x[u] <= a.thr_m1));
+    }
+}
+
+template <int SCHEME, int WIDTH>
+__global__ void __launch_bounds__(kDetectThreads)
+detect_unique_kernel(const DetectArgs a, uint32_t *global_tables) {
+    __shared__ __align__(16) uint32_t smem_tables[kDetectThreads / 32][kUniqueSlots];
+    const int lane = threadIdx.x & 31;
+    const int64_t seq = static_cast<int64_t>(blockIdx.x) * (kDetectThreads / 32) + (threadIdx.x >> 5);
+    if (seq >= a.N) return;
+    const int64_t off = a.offsets[seq];
+    int64_t L = clamp_len(a.lengths[seq]);
+    if (off < 0 || off >= a.total_tokens) L = 0;
+    else if (off + L > a.total_tokens) L = a.total_tokens - off;
+    const int width = WIDTH > 0 ? WIDTH : a.W;
+    const int32_t *tok = a.tokens + off;
+    const int len = static_cast<int>(L);
+    const int T = len > width ? len - width : 0;
+    constexpr int kTrip = 32 * kDetectIlp;
+
+    uint32_t *table = smem_tables[threadIdx.x >> 5];
+    uint32_t slots = 64;
+    if (T > kUniqueSmemMaxT) {
+        if (!global_tables) {                        // longer than the caller said any sequence is
+            if (lane == 0) {
+                a.out_counts[seq] = -1;
+                if (a.out_T) a.out_T[seq] = -1;
+                a.out_z[seq] = __longlong_as_double(0x7ff8000000000000LL);
+            }
+            return;
+        }
+        table = global_tables + 4 * off;
+        while (slots < 2u * static_cast<uint32_t>(T)) slots <<= 1;
+    } else {
+        while (slots < 2u * static_cast<uint32_t>(T) && slots < kUniqueSlots) slots <<= 1;
+    }
+    const uint32_t mask = slots - 1u;
+    const int shift = __clz(slots) + 1;               // 32 - log2(slots)
+    for (uint32_t i = lane * 4u; i < slots; i += 128u)
+        *reinterpret_cast<uint4 *>(table + i) = make_uint4(0u, 0u, 0u, 0u);
+    __syncwarp();
+
+    int count = 0, distinct = 0;
+    int base = width;
+    for (; len - base >= kTrip; base += kTrip)
+        unique_trip<SCHEME, WIDTH, false>(a, tok, base, len, lane, table, mask, shift, count, distinct);
+    if (base < len) unique_trip<SCHEME, WIDTH, true>(a, tok, base, len, lane, table, mask, shift, count, distinct);
+
+    if (lane == 0) {
+        a.out_counts[seq] = count;
+        if (a.out_T) a.out_T[seq] = distinct;
+        a.out_z[seq] = zscore(count, distinct, a.gamma);
+    }
+}
+
+template <int SCHEME>
+cudaError_t launch_detect_unique(const DetectArgs &a, uint32_t *tables, unsigned grid, cudaStream_t s) {
+    switch (a.W) {
+        case 1: detect_unique_kernel<SCHEME, 1><<<grid, kDetectThreads, 0, s>>>(a, tables); break;
+        case 4: detect_unique_kernel<SCHEME, 4><<<grid, kDetectThreads, 0, s>>>(a, tables); break;
+        default: detect_unique_kernel<SCHEME, 0><<<grid, kDetectThreads, 0, s>>>(a, tables); break;
+    }
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -377,5 +547,74 @@ extern "C" int sbw_window_z(const uint32_t *bits, const int32_t *lengths, const 
     window_kernel<<<grid, kDetectThreads, 0, static_cast<cudaStream_t>(stream)>>>(
         bits, prefix_scratch, lengths, offsets, N, total_tokens, ctx_width, w, gamma, out_count, out_start, out_z);
     SBW_CUDA_TRY(cudaGetLastError());
+    return SBW_OK;
+}
+
+extern "C" int sbw_prefix_z(const uint32_t *bits, const int32_t *lengths, const int64_t *offsets,
+                            const int32_t *keep, int64_t N, int64_t total_tokens, int ctx_width, double gamma,
+                            int32_t *out_counts, int32_t *out_T, double *out_z, void *stream) {
+    using namespace sbw;
+    if (ctx_width < 1 || ctx_width > SBW_MAX_CTX_WIDTH || !(gamma > 0.0 && gamma < 1.0)) return SBW_ERR_INVALID_ARG;
+    if (N < 0 || total_tokens < 0) return SBW_ERR_INVALID_ARG;
+    if (N == 0) return SBW_OK;
+    if (!bits || !lengths || !offsets || !keep || !out_counts || !out_z) return SBW_ERR_INVALID_ARG;
+    const unsigned grid = static_cast<unsigned>((N + kDetectThreads / 32 - 1) / (kDetectThreads / 32));
+    prefix_kernel<<<grid, kDetectThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        bits, lengths, offsets, keep, N, total_tokens, ctx_width, gamma, out_counts, out_T, out_z);
+    SBW_CUDA_TRY(cudaGetLastError());
+    return SBW_OK;
+}
+
+extern "C" size_t sbw_detect_unique_workspace_bytes(int64_t N, int64_t total_tokens, int64_t max_length) {
+    if (N <= 0 || total_tokens < 0) return 0;
+    size_t bytes = sbw::align_up(sbw_detect_workspace_bytes(N), 256);
+    if (max_length - 1 > sbw::kUniqueSmemMaxT) bytes += 16 * static_cast<size_t>(total_tokens);
+    return bytes;
+}
+
+extern "C" int sbw_detect_unique(const int32_t *tokens, const int32_t *lengths, const int64_t *offsets, int64_t N,
+                                 int64_t total_tokens, int64_t max_length, int ctx_width, uint64_t key,
+                                 double gamma, int scheme, int32_t *out_counts, int32_t *out_T, double *out_z,
+                                 void *workspace, size_t workspace_bytes, void *stream) {
+    using namespace sbw;
+    if (!valid_common(SBW_DTYPE_F32, ctx_width, gamma, scheme)) return SBW_ERR_INVALID_ARG;
+    if (N < 0 || total_tokens < 0 || max_length < 0) return SBW_ERR_INVALID_ARG;
+    if (N == 0) return SBW_OK;
+    if (N > (int64_t(1) << 31) * (kDetectThreads / 32) - 1) return SBW_ERR_UNSUPPORTED;
+    if (!lengths || !out_counts || !out_z) return SBW_ERR_INVALID_ARG;
+    if (!tokens && total_tokens > 0) return SBW_ERR_INVALID_ARG;
+    const size_t need = sbw_detect_unique_workspace_bytes(N, total_tokens, max_length);
+    if (!workspace || workspace_bytes < need || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
+        return SBW_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t scan_bytes = align_up(sbw_detect_workspace_bytes(N), 256);
+    uint32_t *tables = max_length - 1 > kUniqueSmemMaxT
+                           ? reinterpret_cast<uint32_t *>(static_cast<char *>(workspace) + scan_bytes)
+                           : nullptr;
+
+    DetectArgs a;
+    a.tokens = tokens;
+    a.lengths = lengths;
+    a.offsets = offsets;
+    a.N = N;
+    a.total_tokens = total_tokens;
+    a.W = ctx_width;
+    a.key = key;
+    a.thr_m1 = threshold_minus_one(gamma);
+    a.gamma = gamma;
+    a.out_counts = out_counts;
+    a.out_T = out_T;
+    a.out_z = out_z;
+    a.out_bits = nullptr;
+    a.weyl = make_weyl();
+    if (!offsets) {
+        int64_t *ws_offsets = nullptr;
+        const int rc = scan_lengths(lengths, N, workspace, &ws_offsets, s);
+        if (rc != SBW_OK) return rc;
+        a.offsets = ws_offsets;
+    }
+    const unsigned grid = static_cast<unsigned>((N + kDetectThreads / 32 - 1) / (kDetectThreads / 32));
+    SBW_CUDA_TRY(scheme == SBW_SCHEME_CONTEXT ? launch_detect_unique<SBW_SCHEME_CONTEXT>(a, tables, grid, s)
+                                              : launch_detect_unique<SBW_SCHEME_SELFSALT>(a, tables, grid, s));
     return SBW_OK;
 }
