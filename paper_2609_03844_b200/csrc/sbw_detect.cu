@@ -389,9 +389,12 @@ prefix_kernel(const uint32_t *all_bits, const int32_t *lengths, const int64_t *o
 // probe path.  Which occurrence represents a tuple does not matter -- equal tuples have equal
 // green bits -- so counts are deterministic.  The table lives in shared memory (kUniqueSlots
 // slots per warp) for sequences with at most kUniqueSmemMaxT scored tokens, otherwise in the
-// caller's workspace at 4 * offset (the smallest power of two >= 2T is below 4T slots).
-constexpr int kUniqueSlots = 2048;
+// caller's workspace at 4 * offset (the smallest power of two >= 2T is below 4T slots).  The
+// compare-and-swap insert below serves the workspace tables; shared-memory tables use the
+// atomic-free scheme of insert_trip_shared.
+constexpr int kUniqueSlots = 4096;
 constexpr int kUniqueSmemMaxT = 1536;
+static_assert(kUniqueSmemMaxT + SBW_MAX_CTX_WIDTH < 2048, "positions on the shared path must fit 11 bits");
 
 template <int WIDTH>
 __device__ __forceinline__ uint32_t tuple_hash(const int32_t *tok, int t, int width) {
@@ -425,17 +428,85 @@ __device__ __forceinline__ bool insert_tuple(uint32_t *table, uint32_t mask, int
     return true;
 }
 
-template <int SCHEME, int WIDTH, bool TAIL>
+// The shared-memory table is filled without atomics.  An entry is 16 bits, (fingerprint << 11) |
+// position: the low 5 bits of the tuple's hash and the token position (below 2048 on this path),
+// so most foreign entries are told apart without touching the tokens, and kUniqueSlots of them
+// keep the load factor at or below 3/8.  The warp inserts the positions of
+// a trip in rounds of three phases separated by __syncwarp: (1) every pending position walks its
+// probe path over the table as the last round left it, until it meets its own tuple (duplicate,
+// done) or an empty slot; (2) those at an empty slot store their entry -- several may hit the
+// same slot, one store lands; (3) each reads the slot back: the one that finds its own entry has
+// entered the tuple, the others stay pending and meet the winner in the next round.  Equal
+// tuples of one trip walk the same path over the same table state, so they always collide in
+// phase 2 and exactly one of them wins.
+constexpr int kUniquePosBits = 11;
+
+template <int WIDTH, bool TAIL>
+__device__ __forceinline__ void insert_trip_shared(volatile uint16_t *table, uint32_t mask, int shift,
+                                                   const int32_t *tok, int base, int lane, int width,
+                                                   bool (&first)[kDetectIlp]) {
+    uint32_t slot[kDetectIlp], mine[kDetectIlp];
+    bool pending[kDetectIlp], writer[kDetectIlp];
+#pragma unroll
+    for (int u = 0; u < kDetectIlp; ++u) {
+        const int t = base + u * 32 + lane;
+        pending[u] = first[u];                           // on entry: the position exists
+        const uint32_t h = tuple_hash<WIDTH>(tok, pending[u] ? t : width, width);
+        slot[u] = h >> shift;
+        mine[u] = ((h << kUniquePosBits) | static_cast<uint32_t>(t)) & 0xFFFFu;
+    }
+    for (int round = 0; round < 32 * kDetectIlp + 1; ++round) {   // every round settles a position
+#pragma unroll
+        for (int u = 0; u < kDetectIlp; ++u) {
+            writer[u] = false;
+            if (!pending[u]) continue;
+            const int t = base + u * 32 + lane;
+            for (uint32_t n = 0; n <= mask; ++n) {       // bounded: the table always has a free slot
+                const uint32_t e = table[slot[u]];
+                if (e == 0u) {
+                    writer[u] = true;
+                    break;
+                }
+                if (((e ^ mine[u]) >> kUniquePosBits) == 0u &&
+                    same_tuple<WIDTH>(tok, static_cast<int>(e & ((1u << kUniquePosBits) - 1u)), t, width)) {
+                    pending[u] = false;
+                    first[u] = false;
+                    break;
+                }
+                slot[u] = (slot[u] + 1u) & mask;
+            }
+        }
+        __syncwarp();
+#pragma unroll
+        for (int u = 0; u < kDetectIlp; ++u)
+            if (writer[u]) table[slot[u]] = static_cast<uint16_t>(mine[u]);
+        __syncwarp();
+        bool more = false;
+#pragma unroll
+        for (int u = 0; u < kDetectIlp; ++u) {
+            if (writer[u] && table[slot[u]] == mine[u]) pending[u] = false;
+            more = more || pending[u];
+        }
+        if (!__any_sync(0xffffffffu, more)) break;
+    }
+}
+
+template <int SCHEME, int WIDTH, bool TAIL, bool SHARED>
 __device__ __forceinline__ void unique_trip(const DetectArgs &a, const int32_t *tok, int base, int len, int lane,
-                                            uint32_t *table, uint32_t mask, int shift, int &count, int &distinct) {
+                                            void *table, uint32_t mask, int shift, int &count, int &distinct) {
     const int width = WIDTH > 0 ? WIDTH : a.W;
     uint32_t v[kDetectIlp];
     uint64_t r[kDetectIlp];
     bool first[kDetectIlp];
     load_trip<SCHEME, WIDTH, TAIL>(a, tok, base, len, lane, v, r, first);
+    if constexpr (SHARED) {
+        insert_trip_shared<WIDTH, TAIL>(static_cast<uint16_t *>(table), mask, shift, tok, base, lane, width, first);
+    } else {
 #pragma unroll
-    for (int u = 0; u < kDetectIlp; ++u)
-        first[u] = first[u] && insert_tuple<WIDTH>(table, mask, shift, tok, base + u * 32 + lane, width);
+        for (int u = 0; u < kDetectIlp; ++u)
+            first[u] = first[u] && insert_tuple<WIDTH>(static_cast<uint32_t *>(table), mask, shift, tok,
+                                                       base + u * 32 + lane, width);
+    }
     uint32_t x[kDetectIlp];
     philox_word0_n<kDetectIlp>(v, r, x, a.weyl);
 #pragma unroll
@@ -445,64 +516,74 @@ __device__ __forceinline__ void unique_trip(const DetectArgs &a, const int32_t *
     }
 }
 
-template <int SCHEME, int WIDTH>
-__global__ void __launch_bounds__(kDetectThreads)
-detect_unique_kernel(const DetectArgs a, uint32_t *global_tables) {
-    __shared__ __align__(16) uint32_t smem_tables[kDetectThreads / 32][kUniqueSlots];
-    const int lane = threadIdx.x & 31;
-    const int64_t seq = static_cast<int64_t>(blockIdx.x) * (kDetectThreads / 32) + (threadIdx.x >> 5);
-    if (seq >= a.N) return;
-    const int64_t off = a.offsets[seq];
-    int64_t L = clamp_len(a.lengths[seq]);
-    if (off < 0 || off >= a.total_tokens) L = 0;
-    else if (off + L > a.total_tokens) L = a.total_tokens - off;
+template <int SCHEME, int WIDTH, bool SHARED>
+__device__ __forceinline__ void unique_sequence(const DetectArgs &a, const int32_t *tok, int len, int lane,
+                                                void *table, uint32_t slots, int &count, int &distinct) {
     const int width = WIDTH > 0 ? WIDTH : a.W;
-    const int32_t *tok = a.tokens + off;
-    const int len = static_cast<int>(L);
-    const int T = len > width ? len - width : 0;
     constexpr int kTrip = 32 * kDetectIlp;
-
-    uint32_t *table = smem_tables[threadIdx.x >> 5];
-    uint32_t slots = 64;
-    if (T > kUniqueSmemMaxT) {
-        if (!global_tables) {                        // longer than the caller said any sequence is
-            if (lane == 0) {
-                a.out_counts[seq] = -1;
-                if (a.out_T) a.out_T[seq] = -1;
-                a.out_z[seq] = __longlong_as_double(0x7ff8000000000000LL);
-            }
-            return;
-        }
-        table = global_tables + 4 * off;
-        while (slots < 2u * static_cast<uint32_t>(T)) slots <<= 1;
-    } else {
-        while (slots < 2u * static_cast<uint32_t>(T) && slots < kUniqueSlots) slots <<= 1;
-    }
     const uint32_t mask = slots - 1u;
     const int shift = __clz(slots) + 1;               // 32 - log2(slots)
-    for (uint32_t i = lane * 4u; i < slots; i += 128u)
-        *reinterpret_cast<uint4 *>(table + i) = make_uint4(0u, 0u, 0u, 0u);
+    const uint32_t bytes = slots * (SHARED ? 2u : 4u);   // a multiple of 128 (slots >= 64)
+    for (uint32_t i = lane * 16u; i < bytes; i += 512u)
+        *reinterpret_cast<uint4 *>(static_cast<char *>(table) + i) = make_uint4(0u, 0u, 0u, 0u);
     __syncwarp();
-
-    int count = 0, distinct = 0;
     int base = width;
     for (; len - base >= kTrip; base += kTrip)
-        unique_trip<SCHEME, WIDTH, false>(a, tok, base, len, lane, table, mask, shift, count, distinct);
-    if (base < len) unique_trip<SCHEME, WIDTH, true>(a, tok, base, len, lane, table, mask, shift, count, distinct);
+        unique_trip<SCHEME, WIDTH, false, SHARED>(a, tok, base, len, lane, table, mask, shift, count, distinct);
+    if (base < len)
+        unique_trip<SCHEME, WIDTH, true, SHARED>(a, tok, base, len, lane, table, mask, shift, count, distinct);
+}
 
-    if (lane == 0) {
-        a.out_counts[seq] = count;
-        if (a.out_T) a.out_T[seq] = distinct;
-        a.out_z[seq] = zscore(count, distinct, a.gamma);
+// Persistent warps: sequences differ in length by an order of magnitude and a warp's table pins
+// 8 KiB of shared memory, so each warp takes its next sequence from a counter instead of leaving
+// its slot idle until the longest sequence of its CTA is done.
+template <int SCHEME, int WIDTH>
+__global__ void __launch_bounds__(kDetectThreads)
+detect_unique_kernel(const DetectArgs a, uint32_t *global_tables, unsigned long long *next_sequence) {
+    __shared__ __align__(16) uint16_t smem_tables[kDetectThreads / 32][kUniqueSlots];
+    const int lane = threadIdx.x & 31;
+    const int width = WIDTH > 0 ? WIDTH : a.W;
+    for (;;) {
+        unsigned long long ticket = 0;
+        if (lane == 0) ticket = atomicAdd(next_sequence, 1ull);
+        const int64_t seq = static_cast<int64_t>(__shfl_sync(0xffffffffu, ticket, 0));
+        if (seq >= a.N) return;
+        const int64_t off = a.offsets[seq];
+        int64_t L = clamp_len(a.lengths[seq]);
+        if (off < 0 || off >= a.total_tokens) L = 0;
+        else if (off + L > a.total_tokens) L = a.total_tokens - off;
+        const int32_t *tok = a.tokens + off;
+        const int len = static_cast<int>(L);
+        const int T = len > width ? len - width : 0;
+
+        int count = 0, distinct = 0;
+        uint32_t slots = 64;
+        if (T <= kUniqueSmemMaxT) {
+            while (slots < 4u * static_cast<uint32_t>(T) && slots < kUniqueSlots) slots <<= 1;
+            unique_sequence<SCHEME, WIDTH, true>(a, tok, len, lane, smem_tables[threadIdx.x >> 5], slots, count, distinct);
+        } else if (global_tables) {
+            while (slots < 2u * static_cast<uint32_t>(T)) slots <<= 1;
+            unique_sequence<SCHEME, WIDTH, false>(a, tok, len, lane, global_tables + 4 * off, slots, count, distinct);
+        } else {                                     // longer than the caller said any sequence is
+            count = distinct = -1;
+        }
+        if (lane == 0) {
+            a.out_counts[seq] = count;
+            if (a.out_T) a.out_T[seq] = distinct;
+            a.out_z[seq] =
+                distinct < 0 ? __longlong_as_double(0x7ff8000000000000LL) : zscore(count, distinct, a.gamma);
+        }
+        __syncwarp();                                // the table is reused by the next sequence
     }
 }
 
 template <int SCHEME>
-cudaError_t launch_detect_unique(const DetectArgs &a, uint32_t *tables, unsigned grid, cudaStream_t s) {
+cudaError_t launch_detect_unique(const DetectArgs &a, uint32_t *tables, unsigned long long *next,
+                                 unsigned grid, cudaStream_t s) {
     switch (a.W) {
-        case 1: detect_unique_kernel<SCHEME, 1><<<grid, kDetectThreads, 0, s>>>(a, tables); break;
-        case 4: detect_unique_kernel<SCHEME, 4><<<grid, kDetectThreads, 0, s>>>(a, tables); break;
-        default: detect_unique_kernel<SCHEME, 0><<<grid, kDetectThreads, 0, s>>>(a, tables); break;
+        case 1: detect_unique_kernel<SCHEME, 1><<<grid, kDetectThreads, 0, s>>>(a, tables, next); break;
+        case 4: detect_unique_kernel<SCHEME, 4><<<grid, kDetectThreads, 0, s>>>(a, tables, next); break;
+        default: detect_unique_kernel<SCHEME, 0><<<grid, kDetectThreads, 0, s>>>(a, tables, next); break;
     }
     return cudaGetLastError();
 }
@@ -567,7 +648,7 @@ extern "C" int sbw_prefix_z(const uint32_t *bits, const int32_t *lengths, const 
 
 extern "C" size_t sbw_detect_unique_workspace_bytes(int64_t N, int64_t total_tokens, int64_t max_length) {
     if (N <= 0 || total_tokens < 0) return 0;
-    size_t bytes = sbw::align_up(sbw_detect_workspace_bytes(N), 256);
+    size_t bytes = sbw::align_up(sbw_detect_workspace_bytes(N), 256) + 256;   // offsets, sequence counter
     if (max_length - 1 > sbw::kUniqueSmemMaxT) bytes += 16 * static_cast<size_t>(total_tokens);
     return bytes;
 }
@@ -588,9 +669,13 @@ extern "C" int sbw_detect_unique(const int32_t *tokens, const int32_t *lengths, 
         return SBW_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t scan_bytes = align_up(sbw_detect_workspace_bytes(N), 256);
+    unsigned long long *next = reinterpret_cast<unsigned long long *>(static_cast<char *>(workspace) + scan_bytes);
     uint32_t *tables = max_length - 1 > kUniqueSmemMaxT
-                           ? reinterpret_cast<uint32_t *>(static_cast<char *>(workspace) + scan_bytes)
+                           ? reinterpret_cast<uint32_t *>(static_cast<char *>(workspace) + scan_bytes + 256)
                            : nullptr;
+    DeviceInfo di;
+    if (int rc = current_device_info(&di)) return rc;
+    SBW_CUDA_TRY(cudaMemsetAsync(next, 0, sizeof(unsigned long long), s));
 
     DetectArgs a;
     a.tokens = tokens;
@@ -613,8 +698,10 @@ extern "C" int sbw_detect_unique(const int32_t *tokens, const int32_t *lengths, 
         if (rc != SBW_OK) return rc;
         a.offsets = ws_offsets;
     }
-    const unsigned grid = static_cast<unsigned>((N + kDetectThreads / 32 - 1) / (kDetectThreads / 32));
-    SBW_CUDA_TRY(scheme == SBW_SCHEME_CONTEXT ? launch_detect_unique<SBW_SCHEME_CONTEXT>(a, tables, grid, s)
-                                              : launch_detect_unique<SBW_SCHEME_SELFSALT>(a, tables, grid, s));
+    const int64_t blocks = (N + kDetectThreads / 32 - 1) / (kDetectThreads / 32);
+    const int64_t resident = 8LL * di.sm_count;       // more CTAs than fit: the counter balances them
+    const unsigned grid = static_cast<unsigned>(blocks < resident ? blocks : resident);
+    SBW_CUDA_TRY(scheme == SBW_SCHEME_CONTEXT ? launch_detect_unique<SBW_SCHEME_CONTEXT>(a, tables, next, grid, s)
+                                              : launch_detect_unique<SBW_SCHEME_SELFSALT>(a, tables, next, grid, s));
     return SBW_OK;
 }

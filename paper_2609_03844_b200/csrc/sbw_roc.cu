@@ -1,22 +1,25 @@
 // sbw_roc_auc: area under the ROC curve of detection scores (Section 4.4 of the paper) as the
 // exact pair statistic  AUC = (2 #{z_pos > z_neg} + #{z_pos == z_neg}) / (2 n_pos n_neg).
 //
-// Two kernels.  split_kernel copies the scores of each class into its own dense array (slot
+// Three kernels.  split_kernel copies the scores of each class into its own dense array (slot
 // allocation by one atomic per warp and class; the order inside a class does not matter to a
-// count) and drops NaNs.  pairs_kernel walks the (positive tile) x (negative tile) grid with a
-// persistent set of CTAs: every thread keeps kRocPerThread positives in registers, the negatives
-// of the tile sit in shared memory and are read as warp-wide broadcasts, so a pair costs two
-// fp64 compares and two predicated adds.  Counts are integers, so the result does not depend on
-// the order of anything; the last CTA to finish (atomic ticket) forms the quotient.
+// count) and drops NaNs.  sort_tiles_kernel sorts the negatives inside every tile of
+// kRocNegTile scores (bitonic network in shared memory).  pairs_kernel walks the (positive
+// chunk) x (negative tile) grid with a persistent set of CTAs: the sorted tile sits in shared
+// memory and every positive finds #{q < p} and #{q <= p} in it by two branch-free binary
+// searches, kRocPerThread positives per thread interleaved -- 2 log2(tile) probes per
+// (positive, tile) instead of one compare per pair.  Counts are integers, so the result does not
+// depend on the order of anything; the last CTA to finish (atomic ticket) forms the quotient.
 #include "sbw_common.cuh"
 
 namespace sbw {
 namespace {
 
 constexpr int kRocThreads = 256;
-constexpr int kRocPerThread = 4;
-constexpr int kRocPosTile = kRocThreads * kRocPerThread;   // positives per tile
-constexpr int kRocNegTile = 1024;                          // negatives per tile (8 KiB of shared memory)
+constexpr int kRocPerThread = 8;
+constexpr int kRocPosTile = kRocThreads * kRocPerThread;   // positives per work item
+constexpr int kRocNegTile = 2048;                          // negatives per sorted tile (16 KiB of shared memory)
+constexpr int kRocSortThreads = kRocNegTile / 2;
 
 // counters in the workspace
 struct RocCounters {
@@ -49,40 +52,86 @@ split_kernel(const double *z, const uint8_t *labels, int64_t n, double *pos, dou
     }
 }
 
+// Sorts each tile of kRocNegTile negatives in place, ascending; a short last tile is padded with
+// +inf in shared memory and only its own entries are written back (they are its smallest).
+__global__ void __launch_bounds__(kRocSortThreads)
+sort_tiles_kernel(double *neg, const RocCounters *c) {
+    __shared__ double s[kRocNegTile];
+    const unsigned long long n_neg = c->n_neg;
+    const unsigned long long tiles = (n_neg + kRocNegTile - 1) / kRocNegTile;
+    const double inf = __longlong_as_double(0x7ff0000000000000LL);
+    for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+        const unsigned long long base = tile * kRocNegTile;
+        for (int j = threadIdx.x; j < kRocNegTile; j += kRocSortThreads)
+            s[j] = base + j < n_neg ? neg[base + j] : inf;
+        __syncthreads();
+        for (int k = 2; k <= kRocNegTile; k <<= 1) {
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                const int t = threadIdx.x;
+                const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));     // bit j clear
+                const double a = s[i], b = s[i + j];
+                const bool ascending = (i & k) == 0;
+                if ((a > b) == ascending) {
+                    s[i] = b;
+                    s[i + j] = a;
+                }
+                __syncthreads();
+            }
+        }
+        for (int j = threadIdx.x; j < kRocNegTile; j += kRocSortThreads)
+            if (base + j < n_neg) neg[base + j] = s[j];
+        __syncthreads();
+    }
+}
+
 __global__ void __launch_bounds__(kRocThreads)
 pairs_kernel(const double *pos, const double *neg, RocCounters *c, double *out_auc, uint64_t *out_stats) {
     __shared__ double sneg[kRocNegTile];
     __shared__ unsigned long long red[2][kRocThreads / 32];
     __shared__ bool last;
-    const unsigned long long n_pos = c->n_pos, n_neg = c->n_neg;   // written by the previous kernel
+    const unsigned long long n_pos = c->n_pos, n_neg = c->n_neg;   // written by the split kernel
     const unsigned long long tiles_p = (n_pos + kRocPosTile - 1) / kRocPosTile;
     const unsigned long long tiles_n = (n_neg + kRocNegTile - 1) / kRocNegTile;
-    const double nan = __longlong_as_double(0x7ff8000000000000LL);   // compares false both ways: padding
+    const double nan = __longlong_as_double(0x7ff8000000000000LL);
+    const double inf = __longlong_as_double(0x7ff0000000000000LL);
 
     unsigned long long greater = 0, equal = 0;
     for (unsigned long long item = blockIdx.x; item < tiles_p * tiles_n; item += gridDim.x) {
         const unsigned long long tp = item / tiles_n, tn = item % tiles_n;
+        const unsigned long long left = n_neg - tn * kRocNegTile;
+        const unsigned m = left < kRocNegTile ? static_cast<unsigned>(left) : kRocNegTile;   // real entries
         double p[kRocPerThread];
 #pragma unroll
         for (int r = 0; r < kRocPerThread; ++r) {
             const unsigned long long i = tp * kRocPosTile + r * kRocThreads + threadIdx.x;
-            p[r] = i < n_pos ? pos[i] : nan;
+            p[r] = i < n_pos ? pos[i] : nan;             // NaN compares false: counts nothing
         }
         __syncthreads();                                 // the previous tile's readers are done
-        for (int j = threadIdx.x; j < kRocNegTile; j += kRocThreads) {
-            const unsigned long long i = tn * kRocNegTile + j;
-            sneg[j] = i < n_neg ? neg[i] : nan;
-        }
+        for (int j = threadIdx.x; j < kRocNegTile; j += kRocThreads)
+            sneg[j] = static_cast<unsigned>(j) < m ? neg[tn * kRocNegTile + j] : inf;
         __syncthreads();
-        unsigned g = 0, e = 0;                           // at most kRocPerThread * kRocNegTile each
-#pragma unroll 8
-        for (int j = 0; j < kRocNegTile; ++j) {
-            const double q = sneg[j];
+        // lt[r] = #{q < p[r]}, le[r] = #{q <= p[r]} over the sorted tile; padding is +inf and
+        // sorts last, so clamping to m removes it
+        unsigned lt[kRocPerThread], le[kRocPerThread];
+#pragma unroll
+        for (int r = 0; r < kRocPerThread; ++r) lt[r] = le[r] = 0;
+#pragma unroll
+        for (int step = kRocNegTile / 2; step > 0; step >>= 1) {
 #pragma unroll
             for (int r = 0; r < kRocPerThread; ++r) {
-                g += p[r] > q ? 1u : 0u;
-                e += p[r] == q ? 1u : 0u;
+                if (sneg[lt[r] + step - 1] < p[r]) lt[r] += step;
+                if (sneg[le[r] + step - 1] <= p[r]) le[r] += step;
             }
+        }
+        unsigned g = 0, e = 0;
+#pragma unroll
+        for (int r = 0; r < kRocPerThread; ++r) {
+            if (sneg[lt[r]] < p[r]) lt[r] += 1;
+            if (sneg[le[r]] <= p[r]) le[r] += 1;
+            lt[r] = min(lt[r], m);
+            le[r] = min(le[r], m);
+            g += lt[r];
+            e += le[r] - lt[r];
         }
         greater += g;
         equal += e;
@@ -151,6 +200,12 @@ extern "C" int sbw_roc_auc(const double *z, const uint8_t *labels, int64_t n, do
         const int64_t blocks = (n + kRocThreads - 1) / kRocThreads;
         const unsigned grid = static_cast<unsigned>(blocks < 8LL * di.sm_count ? blocks : 8LL * di.sm_count);
         split_kernel<<<grid, kRocThreads, 0, s>>>(z, labels, n, pos, neg, c);
+        SBW_CUDA_TRY(cudaGetLastError());
+    }
+    {
+        const int64_t tiles = (n + kRocNegTile - 1) / kRocNegTile + 1;
+        const int64_t cap = 2LL * di.sm_count;
+        sort_tiles_kernel<<<static_cast<unsigned>(tiles < cap ? tiles : cap), kRocSortThreads, 0, s>>>(neg, c);
         SBW_CUDA_TRY(cudaGetLastError());
     }
     // enough CTAs to fill the machine, never more than the largest possible number of tile pairs
