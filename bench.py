@@ -422,7 +422,18 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
         s = _time_calls(lambda i: sbw.sbw_detect(tokens, lengths, KEY, 0.25, scheme, counts, z, workspace=ws), 30)
         out[f"detect_{name}_N100000"] = {"tokens_per_s": ntok / s, "ms": s * 1e3, "tokens": ntok,
                                          **place(INT_OPS[f"detect_{name}"] * ntok, 4 * ntok + 24 * N, s)}
-    del tokens
+    # evaluation steps on the same streams: distinct-tuple scoring, then ROC-AUC of the z array
+    # against alternating labels (timing only: these streams are all unmarked)
+    wsu = torch.empty(sbw.sbw_detect_unique_workspace_bytes(N, ntok, 1024), dtype=torch.uint8, device=dev)
+    s = _time_calls(lambda i: sbw.sbw_detect_unique(tokens, lengths, 1024, KEY, 0.25, sbw.SCHEME_CONTEXT, counts,
+                                                    z, wsu), 20)
+    out["detect_unique_context_N100000"] = {"tokens_per_s": ntok / s, "ms": s * 1e3, "tokens": ntok}
+    labels = (torch.arange(N, device=dev) % 2).to(torch.uint8)
+    auc = torch.empty(1, dtype=torch.float64, device=dev)
+    wsr = torch.empty(sbw.sbw_roc_auc_workspace_bytes(N), dtype=torch.uint8, device=dev)
+    s = _time_calls(lambda i: sbw.sbw_roc_auc(z, labels, auc, wsr), 20)
+    out["roc_auc_N100000"] = {"ms": s * 1e3, "pairs_per_s": (N / 2) ** 2 / s}
+    del tokens, wsu
     # config 4: fused sampling sweep, bf16, V=128256, tau 0.7
     for B in (1, 8, 32, 128, 512, 1024):
         x = inputs.logits_normal(B, V2, 4.0, torch.bfloat16, seed=600 + B, device=dev)

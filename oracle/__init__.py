@@ -101,6 +101,12 @@ def lib() -> ctypes.CDLL:
         L.sbw_oracle_bias_sample.argtypes = [vp, i32, i64, i64, i64, i64, vp, i32, u64, c.c_double,
                                              c.c_float, i32, c.c_float, u64, u64, vp, vp, vp, vp,
                                              vp, vp, i32]
+        L.sbw_oracle_nucleus_weight.restype = u64
+        L.sbw_oracle_nucleus_weight.argtypes = [c.c_float, c.c_float, i32, c.c_float]
+        L.sbw_oracle_bias_sample_filtered.restype = None
+        L.sbw_oracle_bias_sample_filtered.argtypes = [vp, i32, i64, i64, i64, i64, vp, i32, u64, c.c_double,
+                                                      c.c_float, i32, c.c_float, i64, c.c_double, u64, u64,
+                                                      vp, vp, vp, i32]
         L.sbw_oracle_jenkins_collisions.restype = i64
         L.sbw_oracle_jenkins_collisions.argtypes = []
         L.sbw_oracle_log_max_ulp.restype = c.c_double
@@ -290,6 +296,27 @@ def bias_sample(logits: np.ndarray, V, ctx_tokens, key, gamma, delta, scheme, te
                                  delta, scheme, temperature, rng_seed, rng_step, _ptr(tokens),
                                  _ptr(m), _ptr(Z), _ptr(p), _ptr(probs), _ptr(score), threads)
     return {"tokens": tokens, "max": m, "sumexp": Z, "prob": p, "probs": probs, "score": score}
+
+
+def nucleus_weight(l: float, m: float, is_max: bool, c: float) -> int:
+    return int(lib().sbw_oracle_nucleus_weight(l, m, int(is_max), c))
+
+
+def bias_sample_filtered(logits: np.ndarray, V, ctx_tokens, key, gamma, delta, scheme, temperature,
+                         top_k, top_p, rng_seed, rng_step, vocab_offset=0, want_mask=False, threads=1):
+    """Fused bias + top-k / top-p truncation + Gumbel-max id: dict of tokens, kept counts, mask."""
+    assert logits.ndim == 2 and logits.dtype in (np.float32, np.uint16)
+    x = np.ascontiguousarray(logits)
+    B, ld = x.shape
+    ctx, W = _ctx(ctx_tokens, B)
+    dtype = DTYPE_F32 if x.dtype == np.float32 else DTYPE_BF16
+    tokens = np.zeros(B, dtype=np.int32)
+    kept = np.zeros(B, dtype=np.int32)
+    mask = np.zeros((B, V), dtype=np.uint8) if want_mask else None
+    lib().sbw_oracle_bias_sample_filtered(_ptr(x), dtype, B, V, ld, vocab_offset, _ptr(ctx), W, key, gamma,
+                                          delta, scheme, temperature, top_k, top_p, rng_seed, rng_step,
+                                          _ptr(tokens), _ptr(kept), _ptr(mask), threads)
+    return {"tokens": tokens, "kept": kept, "mask": mask}
 
 
 def jenkins_collisions() -> int:

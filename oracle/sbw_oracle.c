@@ -609,6 +609,125 @@ void sbw_oracle_bias_sample(const void *logits, int dtype, int64_t B, int64_t V,
                    out_sumexp, out_prob, out_probs, out_score);
 }
 
+/* ------------------------------------------------------------------ R10: top-k / top-p ---- */
+/*
+ * Sampling from the truncated distribution (Appendix F of the paper samples with top_p = 0.8;
+ * the paper gives no arithmetic for it, this library fixes one so that the kept set is a pure
+ * function of the biased logits).  Per row, with l' the biased logits of Eq. 2:
+ *   order    candidates sorted by order-encoded bits descending, ties by column ascending (the
+ *            order of the top-k restriction above); m = the first one's value.
+ *   top-k    top_k > 0 keeps the first min(top_k, V) of that order; top_k = 0 keeps all.
+ *   weights  integers, so that sums do not depend on the order of addition:
+ *            c = (float)(log2(e) / (double)temperature);
+ *            a candidate with the bits of m has W = 2^40; otherwise d = l' - m, y = d * c (fp32);
+ *            W = 0 unless y >= -41; n = rintf(y), f = y - n (exact), p = degree-7 Horner in f
+ *            with fmaf over the coefficients (ln 2)^k / k! rounded to fp32, W = trunc(p 2^(n+40)).
+ *   top-p    top_p < 1: with Z the sum of W over the candidates top-k kept, p32 = floor(top_p
+ *            2^32) clamped to [1, 2^32], candidate number i of the order stays iff the weights of
+ *            the candidates before it sum to S with S 2^32 < p32 Z (the candidate that crosses
+ *            top_p stays, as in the usual nucleus rule; the first always stays).
+ *   sample   Gumbel-max over the kept candidates with the stream of sbw_oracle_gumbel:
+ *            argmax fmaf(l', 1/temperature, g), ties to the lowest column.
+ */
+uint64_t sbw_oracle_nucleus_weight(float l, float m, int is_max, float c)
+{
+    static const float K[8] = { 0x1p+0f, 0x1.62e43p-1f, 0x1.ebfbep-3f, 0x1.c6b08ep-5f,
+                                0x1.3b2ab6p-7f, 0x1.5d87fep-10f, 0x1.430912p-13f, 0x1.ffcbfcp-17f };
+    if (is_max)
+        return (uint64_t)1 << 40;
+    float d = l - m;
+    float y = d * c;
+    if (!(y >= -41.0f))
+        return 0;                                    /* also NaN and -inf */
+    if (y > 0.0f)
+        y = 0.0f;                                    /* cannot happen for ordered finite values */
+    float n = rintf(y);
+    float f = y - n;
+    float p = K[7];
+    for (int i = 6; i >= 0; --i)
+        p = fmaf(p, f, K[i]);
+    float scaled = ldexpf(p, (int)n + 40);
+    return (uint64_t)scaled;
+}
+
+void sbw_oracle_bias_sample_filtered(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
+                                     int64_t vocab_offset, const int32_t *ctx_tokens, int ctx_width,
+                                     uint64_t key, double gamma, float delta, int scheme,
+                                     float temperature, int64_t top_k, double top_p, uint64_t rng_seed,
+                                     uint64_t rng_step, int32_t *out_tokens, int32_t *out_kept,
+                                     uint8_t *out_mask, int threads)
+{
+    uint64_t thr = sbw_oracle_threshold(gamma);
+    float inv_tau = 1.0f / temperature;
+    float c = (float)(1.4426950408889634 / (double)temperature);
+    double p_scaled = floor(top_p * 4294967296.0);
+    uint64_t p32 = p_scaled < 1.0 ? 1u : (p_scaled > 4294967296.0 ? (uint64_t)1 << 32 : (uint64_t)p_scaled);
+    if (threads < 1)
+        threads = 1;
+#pragma omp parallel for num_threads(threads) schedule(dynamic, 1)
+    for (int64_t b = 0; b < B; ++b) {
+        const int32_t *ctx = ctx_tokens + b * ctx_width;
+        float *biased = (float *)malloc((size_t)V * sizeof(float));
+        ranked_t *order = (ranked_t *)malloc((size_t)V * sizeof(ranked_t));
+        if (!biased || !order) {
+            free(biased);
+            free(order);
+            continue;
+        }
+        for (int64_t j = 0; j < V; ++j) {
+            uint32_t v = (uint32_t)(vocab_offset + j);
+            int g = sbw_oracle_green(seed_for(scheme, key, ctx, ctx_width, v), v, thr);
+            uint32_t bits;
+            if (dtype == SBW_O_DTYPE_BF16) {
+                uint16_t h = sbw_oracle_bias_elem_bf16(((const uint16_t *)logits)[b * ld + j], delta, g);
+                biased[j] = sbw_oracle_bf16_to_f32(h);
+            } else {
+                biased[j] = sbw_oracle_bias_elem_f32(((const float *)logits)[b * ld + j], delta, g);
+            }
+            memcpy(&bits, &biased[j], sizeof bits);
+            order[j].code = order_code(bits);
+            order[j].col = j;
+        }
+        qsort(order, (size_t)V, sizeof(ranked_t), ranked_cmp);
+        int64_t n1 = (top_k > 0 && top_k < V) ? top_k : V;          /* after top-k */
+        int64_t n2 = n1;                                            /* after top-p */
+        if (top_p < 1.0) {
+            float m = biased[order[0].col];
+            unsigned __int128 Z = 0;
+            for (int64_t i = 0; i < n1; ++i)
+                Z += sbw_oracle_nucleus_weight(biased[order[i].col], m, order[i].code == order[0].code, c);
+            unsigned __int128 S = 0;
+            n2 = 0;
+            for (int64_t i = 0; i < n1; ++i) {
+                if (!((S << 32) < (unsigned __int128)p32 * Z))
+                    break;
+                n2 = i + 1;
+                S += sbw_oracle_nucleus_weight(biased[order[i].col], m, order[i].code == order[0].code, c);
+            }
+        }
+        if (out_mask)
+            memset(out_mask + b * V, 0, (size_t)V);
+        int64_t best = -1;
+        float best_s = -INFINITY;
+        for (int64_t i = 0; i < n2; ++i) {
+            int64_t j = order[i].col;
+            if (out_mask)
+                out_mask[b * V + j] = 1;
+            float g = sbw_oracle_gumbel(rng_seed, rng_step, (uint32_t)b, (uint32_t)(vocab_offset + j));
+            float sc = fmaf(biased[j], inv_tau, g);
+            if (best < 0 || sc > best_s || (sc == best_s && j < best)) {
+                best_s = sc;
+                best = j;
+            }
+        }
+        out_tokens[b] = (int32_t)best;
+        if (out_kept)
+            out_kept[b] = (int32_t)n2;
+        free(biased);
+        free(order);
+    }
+}
+
 /* ------------------------------------------------------------------ exhaustive checks */
 int64_t sbw_oracle_jenkins_collisions(void)
 {

@@ -23,6 +23,8 @@
  *                      exact threshold sweep in rationals, binormal closed form
  *   log / gumbel /     pinned: fp64 log, chi-square of sampled ids against    (test_oracle_sample)
  *   sample             softmax, scipy softmax / logsumexp, closed form
+ *   top-k / top-p      pinned: fp64 softmax + cumulative sums (numpy), torch.topk,  (test_oracle_filter)
+ *   sampling           2^f in fp64, closed forms, chi-square of sampled ids
  *   bit compatibility with the paper authors' own package: PARITY UNPINNED (the paper
  *   prints no hash input/output pair; the constants below are this library's frozen
  *   reading, "SBW-spec v1").
@@ -130,6 +132,18 @@ void sbw_oracle_bias_sample(const void *logits, int dtype, int64_t B, int64_t V,
                             float temperature, uint64_t rng_seed, uint64_t rng_step,
                             int32_t *out_tokens, double *out_max, double *out_sumexp,
                             double *out_prob, double *out_probs, float *out_score, int threads);
+
+/* Fused sampling from the top-k / top-p truncated distribution (Appendix F samples with top_p = 0.8;
+ * the integer-weight arithmetic is this library's, see sbw_oracle.c).  top_k = 0 and top_p >= 1 switch
+ * the filters off.  out_kept (nullable) [B]: candidates left per row; out_mask (nullable) [B, V]: 1
+ * for kept candidates. */
+uint64_t sbw_oracle_nucleus_weight(float l, float m, int is_max, float c);
+void sbw_oracle_bias_sample_filtered(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
+                                     int64_t vocab_offset, const int32_t *ctx_tokens, int ctx_width,
+                                     uint64_t key, double gamma, float delta, int scheme,
+                                     float temperature, int64_t top_k, double top_p, uint64_t rng_seed,
+                                     uint64_t rng_step, int32_t *out_tokens, int32_t *out_kept,
+                                     uint8_t *out_mask, int threads);
 
 /* Exhaustive checks that are too slow from Python; each returns a summary. */
 /* Number of 32-bit values hit more than once by jenkins over all 2^32 inputs (0 = bijection).
