@@ -310,6 +310,38 @@ size_t sbw_roc_auc_workspace_bytes(int64_t n);
 int sbw_roc_auc(const double *z, const uint8_t *labels, int64_t n, double *out_auc, uint64_t *out_stats,
                 void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * sbw_bias_sample_filtered -- sbw_bias_sample on the top-k / top-p truncated distribution (the
+ * paper's Appendix F samples with temperature 0.7 and top_p = 0.8; the paper gives no arithmetic
+ * for the truncation, the one below is this library's).  Per row, with l' the biased logits of Eq. 2:
+ *   order    candidates are ranked by order-encoded bit pattern, descending, ties to the lowest
+ *            column (the order of sbw_bias_logits_topk); m is the first one's value.
+ *   top_k    > 0 keeps the first min(top_k, V) of the order; 0 switches the filter off.
+ *   top_p    < 1 keeps candidate i of what top_k left iff the integer weights of the candidates
+ *            before it sum to S with S 2^32 < floor(top_p 2^32) Z, Z being the sum over all of
+ *            them; >= 1 switches the filter off; must be > 0.  The weight of a candidate is 2^40
+ *            for the bits of m, else with c = (float)(log2(e) / (double)temperature), y = (l' - m) c
+ *            in fp32: 0 if not y >= -41, else trunc(2^(40 + n) P(y - n)), n = rintf(y), P the
+ *            degree-7 Taylor polynomial of 2^f with coefficients rounded to fp32, evaluated by
+ *            Horner's rule with fused multiply-adds.  The sums are exact, so the kept set does
+ *            not depend on the order of addition.
+ *   sample   arg max over the kept candidates of fmaf(l', 1 / temperature, g), g the Gumbel
+ *            variate sbw_bias_sample draws for (rng_seed, rng_step, row, vocab_offset + column),
+ *            ties to the lowest column.  With both filters off the ids equal sbw_bias_sample's.
+ * Arguments as for sbw_bias_sample (logits are not modified), plus
+ *   out_tokens  device [B] int32: the sampled column per row.
+ *   out_kept    device [B] int32 or NULL: the number of candidates left per row.
+ *   workspace   device, 256-byte aligned, at least sbw_sample_filtered_workspace_bytes(dtype, B, V)
+ *               bytes (a biased copy of the logits); contents undefined afterwards.
+ * Rows that contain NaN are not supported (the result is some kept column).
+ */
+size_t sbw_sample_filtered_workspace_bytes(int dtype, int64_t B, int64_t V);
+int sbw_bias_sample_filtered(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
+                             int64_t vocab_offset, const int32_t *ctx_tokens, int ctx_width, uint64_t key,
+                             double gamma, float delta, int scheme, float temperature, int64_t top_k,
+                             double top_p, uint64_t rng_seed, uint64_t rng_step, int32_t *out_tokens,
+                             int32_t *out_kept, void *workspace, size_t workspace_bytes, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -31,7 +31,8 @@ EXPORTS = ("sbw_version", "sbw_last_cuda_error", "sbw_bias_logits",
            "sbw_detect", "sbw_int_probe", "sbw_bias_sample_noalloc", "sbw_bias_logits_topk",
            "sbw_bias_sample_shard", "sbw_sample_combine", "sbw_detect_bits_words", "sbw_detect_bits",
            "sbw_window_z", "sbw_prefix_z", "sbw_detect_unique_workspace_bytes", "sbw_detect_unique",
-           "sbw_roc_auc_workspace_bytes", "sbw_roc_auc")
+           "sbw_roc_auc_workspace_bytes", "sbw_roc_auc", "sbw_sample_filtered_workspace_bytes",
+           "sbw_bias_sample_filtered")
 
 _lib = None
 
@@ -114,6 +115,12 @@ def lib() -> ctypes.CDLL:
         L.sbw_roc_auc_workspace_bytes.argtypes = [i64]
         L.sbw_roc_auc.restype = i32
         L.sbw_roc_auc.argtypes = [vp, vp, i64, vp, vp, vp, sz, vp]
+        L.sbw_sample_filtered_workspace_bytes.restype = sz
+        L.sbw_sample_filtered_workspace_bytes.argtypes = [i32, i64, i64]
+        L.sbw_bias_sample_filtered.restype = i32
+        L.sbw_bias_sample_filtered.argtypes = [vp, i32, i64, i64, i64, i64, vp, i32, u64, c.c_double,
+                                               c.c_float, i32, c.c_float, i64, c.c_double, u64, u64, vp, vp,
+                                               vp, sz, vp]
         L.sbw_int_probe.restype = i32
         L.sbw_int_probe.argtypes = [i32, i32, i32, i32, vp, vp, vp]
         _lib = L
@@ -241,6 +248,32 @@ def sbw_bias_sample(logits: torch.Tensor, ctx_tokens: torch.Tensor, key: int, ga
                                _ptr(out_sumexp), _ptr(out_prob), _ptr(out_probs), _ptr(workspace),
                                workspace.numel() * workspace.element_size(), _stream(stream))
     _check("sbw_bias_sample", rc)
+    return out_tokens
+
+
+def sbw_sample_filtered_workspace_bytes(dtype: torch.dtype, B: int, V: int) -> int:
+    code = DTYPE_F32 if dtype == torch.float32 else DTYPE_BF16
+    return int(lib().sbw_sample_filtered_workspace_bytes(code, B, V))
+
+
+def sbw_bias_sample_filtered(logits: torch.Tensor, ctx_tokens: torch.Tensor, key: int, gamma: float,
+                             delta: float, scheme: int, temperature: float, top_k: int, top_p: float,
+                             rng_seed: int, rng_step: int, out_tokens: torch.Tensor, workspace: torch.Tensor,
+                             *, out_kept: torch.Tensor | None = None, V: int | None = None,
+                             vocab_offset: int = 0, stream=None) -> torch.Tensor:
+    """Fused bias + top-k / top-p truncation + Gumbel-max id (``top_k`` 0 and ``top_p`` >= 1 switch
+    the filters off).  Returns ``out_tokens`` (int32 CUDA)."""
+    B, V, ld = _row_layout(logits, V)
+    W = _ctx(ctx_tokens, B)
+    for name, t in (("out_tokens", out_tokens), ("out_kept", out_kept)):
+        if t is not None and (t.dtype != torch.int32 or not t.is_cuda or not t.is_contiguous()):
+            raise TypeError(f"{name} must be a contiguous CUDA int32 tensor")
+    rc = lib().sbw_bias_sample_filtered(_ptr(logits), _dtype_code(logits), B, V, ld, vocab_offset,
+                                        _ptr(ctx_tokens), W, key, gamma, delta, scheme, temperature, top_k,
+                                        top_p, rng_seed, rng_step, _ptr(out_tokens), _ptr(out_kept),
+                                        _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                        _stream(stream))
+    _check("sbw_bias_sample_filtered", rc)
     return out_tokens
 
 

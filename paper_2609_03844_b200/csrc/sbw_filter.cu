@@ -1,0 +1,489 @@
+// sbw_bias_sample_filtered: bias (Eq. 2 of the paper) + top-k / top-p truncation + Gumbel-max
+// sampling (the paper's Appendix F samples with temperature 0.7 and top_p = 0.8).
+//
+// The biased logits l' are produced once -- the row is copied into the workspace and biased
+// there by the full-vocabulary bias kernel -- and everything after that is memory traffic over
+// that copy, one CTA per row:
+//   order    candidates are ranked by order-encoded bits, ties by column; with key_m the code of
+//            the row maximum, a candidate is the 64-bit composite (key_m - code) << 32 | column,
+//            and "kept" is always "composite <= boundary".
+//   weights  integers W = trunc(2^(40 + (l' - m) c)) from a fixed fp32 2^f (see nucleus_weight),
+//            so sums are exact and the kept set does not depend on the order of addition.
+//   select   the boundary is found by a radix descent over the distance key_m - code: a pass
+//            histograms the candidates of the current range into 2048 bins (weight and number),
+//            a block scan finds the bin in which the running weight crosses the target (top-k: k
+//            candidates; top-p: ceil(p32 Z / 2^32) of weight, Z being the total of the first
+//            histogram), and the range narrows to that bin.  When the bin holds at most kListCap
+//            candidates they are gathered, sorted and scanned in shared memory, which gives the
+//            boundary directly; a range of one distance that is still too full is a group of
+//            equal logits, cut by column with one ordered counting pass.
+//   sample   one last pass draws Gumbel variates for the kept candidates only and takes the
+//            arg max of fmaf(l', 1/tau, g), ties to the lowest column.
+#include <cuda_bf16.h>
+
+#include "sbw_common.cuh"
+#include "sbw_gumbel.cuh"
+#include "sbw_hash.cuh"
+
+namespace sbw {
+
+int bias_logits_impl(void *logits, int dtype, int64_t B, int64_t V, int64_t ld, int64_t vocab_offset,
+                     const int32_t *ctx_tokens, int ctx_width, uint64_t key, double gamma, float delta,
+                     int scheme, cudaStream_t stream);
+
+namespace {
+
+constexpr int kFilterThreads = 512;
+constexpr int kFilterWarps = kFilterThreads / 32;
+constexpr int kBins = 2048;
+constexpr int kBinBits = 11;
+constexpr int kListCap = 2048;
+constexpr uint64_t kAll = ~0ull;
+
+struct FilterArgs {
+    const void *biased;    // [B, ld] biased logits, rows 16-byte aligned
+    int64_t B, V, ld;
+    uint32_t vocab_offset;
+    float inv_tau;         // 1 / temperature, fp32 division
+    float c;               // (float)(log2(e) / temperature)
+    int64_t top_k;         // 0: off
+    uint64_t p32;          // floor(top_p 2^32) in [1, 2^32]; 0: top-p off
+    uint32_t step_lo, step_hi;
+    BlockKeys gkeys;       // Philox round keys of the Gumbel stream
+    int32_t *out_tokens;
+    int32_t *out_kept;     // nullable
+};
+
+struct FilterShared {
+    unsigned long long hist_w[kBins];
+    unsigned int hist_c[kBins];
+    unsigned long long list[kListCap];
+    unsigned long long red[kFilterWarps];
+    unsigned long long bcast[4];
+    unsigned int list_n;
+    unsigned int red32[kFilterWarps];
+};
+
+__device__ __forceinline__ uint32_t order_code(uint32_t bits) {
+    return (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+}
+__device__ __forceinline__ uint32_t order_decode(uint32_t code) {
+    return (code & 0x80000000u) ? (code & 0x7fffffffu) : ~code;
+}
+
+// Codes are compared in units of one representable value of the logits' type: 32 significant
+// bits for fp32, the upper 16 for bf16 (whose lower 16 bits are always zero).
+template <int DTYPE>
+__device__ __forceinline__ uint32_t code_of_bits(uint32_t bits32) {
+    const uint32_t c = order_code(bits32);
+    return DTYPE == SBW_DTYPE_F32 ? c : c >> 16;
+}
+template <int DTYPE>
+__device__ __forceinline__ float value_of_code(uint32_t code) {
+    if constexpr (DTYPE == SBW_DTYPE_F32) return __uint_as_float(order_decode(code));
+    // 16-bit code: undo the order map on 16 bits, then widen (the low 16 bits of the value are 0)
+    const uint32_t b16 = (code & 0x8000u) ? (code & 0x7fffu) : (~code & 0xffffu);
+    return __uint_as_float(b16 << 16);
+}
+
+// Integer softmax weight of a candidate at distance `dist` below the maximum code (see the oracle
+// of this library for the same steps): 2^40 at the maximum, trunc(2^(40 + (l' - m) c)) below it.
+__device__ __forceinline__ unsigned long long nucleus_weight(float l, float m, bool is_max, float c) {
+    if (is_max) return 1ull << 40;
+    const float d = __fsub_rn(l, m);
+    float y = __fmul_rn(d, c);
+    if (!(y >= -41.0f)) return 0ull;
+    if (y > 0.0f) y = 0.0f;
+    const float n = rintf(y);
+    const float f = __fsub_rn(y, n);
+    float p = 0x1.ffcbfcp-17f;
+    p = __fmaf_rn(p, f, 0x1.430912p-13f);
+    p = __fmaf_rn(p, f, 0x1.5d87fep-10f);
+    p = __fmaf_rn(p, f, 0x1.3b2ab6p-7f);
+    p = __fmaf_rn(p, f, 0x1.c6b08ep-5f);
+    p = __fmaf_rn(p, f, 0x1.ebfbep-3f);
+    p = __fmaf_rn(p, f, 0x1.62e43p-1f);
+    p = __fmaf_rn(p, f, 0x1p+0f);
+    // p 2^(n + 40): n + 40 lies in [-1, 40], so the scale is a normal power of two and exact
+    const float scale = __uint_as_float(static_cast<uint32_t>(static_cast<int>(n) + 40 + 127) << 23);
+    return __float2ull_rz(__fmul_rn(p, scale));
+}
+
+// Calls f(column, code) for every column of the row, 16 bytes per load, several loads in flight.
+template <int DTYPE, typename F>
+__device__ __forceinline__ void for_each(const char *row_ptr, uint32_t V, F f) {
+    constexpr int VEC = DTYPE == SBW_DTYPE_F32 ? 4 : 8;
+    constexpr int kInFlight = 4;
+    const uint32_t nvec = (V + VEC - 1) / VEC;        // the row is padded to whole vectors
+    for (uint32_t j0 = threadIdx.x; j0 < nvec; j0 += kInFlight * kFilterThreads) {
+        uint4 w[kInFlight];
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+            const uint32_t j = j0 + u * kFilterThreads;
+            w[u] = j < nvec ? reinterpret_cast<const uint4 *>(row_ptr)[j] : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+            const uint32_t j = j0 + u * kFilterThreads;
+            if (j >= nvec) break;
+            const uint32_t *e = reinterpret_cast<const uint32_t *>(&w[u]);
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                uint32_t bits;
+                if constexpr (DTYPE == SBW_DTYPE_F32) bits = e[i];
+                else bits = (i & 1) ? (e[i >> 1] & 0xffff0000u) : (e[i >> 1] << 16);
+                const uint32_t col = j * VEC + i;
+                if (col < V) f(col, code_of_bits<DTYPE>(bits));
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ unsigned long long warp_sum(unsigned long long x) {
+    for (int d = 16; d > 0; d >>= 1) x += __shfl_xor_sync(0xffffffffu, x, d);
+    return x;
+}
+
+// Sum over the CTA, returned to every thread.  Uses sh.red and sh.bcast[3].
+__device__ __forceinline__ unsigned long long block_sum(unsigned long long x, FilterShared &sh) {
+    x = warp_sum(x);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sh.red[threadIdx.x >> 5] = x;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long t = 0;
+        for (int w = 0; w < kFilterWarps; ++w) t += sh.red[w];
+        sh.bcast[3] = t;
+    }
+    __syncthreads();
+    return sh.bcast[3];
+}
+
+// Exclusive prefix over the CTA in thread order.  Uses sh.red.
+__device__ __forceinline__ unsigned long long block_exclusive_scan(unsigned long long x, FilterShared &sh) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned long long incl = x;
+    for (int d = 1; d < 32; d <<= 1) {
+        const unsigned long long up = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += up;
+    }
+    __syncthreads();
+    if (lane == 31) sh.red[warp] = incl;
+    __syncthreads();
+    unsigned long long before = 0;
+    for (int w = 0; w < warp; ++w) before += sh.red[w];
+    return before + incl - x;
+}
+
+
+enum { kModeCount = 0, kModeMass = 1 };
+
+// Bitonic sort of sh.list[0 .. len), len a power of two >= 2, ascending.
+__device__ __forceinline__ void sort_list(FilterShared &sh, int len) {
+    for (int k = 2; k <= len; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int t = threadIdx.x; t < len / 2; t += kFilterThreads) {
+                const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+                const unsigned long long a = sh.list[i], b = sh.list[i + j];
+                if ((a > b) == ((i & k) == 0)) {
+                    sh.list[i] = b;
+                    sh.list[i + j] = a;
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+// The composite of the last kept candidate: the first one, in the order of the composites, at
+// which the running weight reaches the target.  MODE count: every candidate weighs 1 and
+// `target` is the number to keep.  MODE mass: candidates weigh nucleus_weight, `target` is p32 and
+// the weight to reach is ceil(p32 Z / 2^32), Z being the weight of everything at or below `limit`.
+// s0: all candidates with a weight lie at distances below 2^s0.
+template <int DTYPE, int MODE>
+__device__ unsigned long long select_boundary(const char *row_ptr, uint32_t V, uint32_t key_m, float m, float c,
+                                              unsigned long long limit, unsigned long long target, int s0,
+                                              FilterShared &sh) {
+    auto weight = [&](uint32_t dist) -> unsigned long long {
+        if (MODE == kModeCount) return 1ull;
+        return nucleus_weight(value_of_code<DTYPE>(key_m - dist), m, dist == 0u, c);
+    };
+    uint32_t r0 = 0;
+    int s = s0;
+    unsigned long long acc = 0;
+    for (int iter = 0; iter < 5; ++iter) {           // the range loses 11 bits per iteration
+        const int sub = s > kBinBits ? s - kBinBits : 0;
+        for (int i = threadIdx.x; i < kBins; i += kFilterThreads) {
+            sh.hist_w[i] = 0ull;
+            sh.hist_c[i] = 0u;
+        }
+        if (threadIdx.x == 0) sh.bcast[0] = kBins;
+        __syncthreads();
+        for_each<DTYPE>(row_ptr, V, [&](uint32_t col, uint32_t code) {
+            const uint32_t dist = key_m - code;
+            if (((static_cast<unsigned long long>(dist) << 32) | col) > limit) return;
+            const uint32_t rel = dist - r0;           // wraps to a large value below the range
+            if (s < 32 && (rel >> s) != 0u) return;
+            const unsigned long long w = weight(dist);
+            if (w == 0ull) return;
+            const uint32_t bin = rel >> sub;
+            atomicAdd(&sh.hist_w[bin], w);
+            atomicAdd(&sh.hist_c[bin], 1u);
+        });
+        __syncthreads();
+        // every thread owns kBins / kFilterThreads consecutive bins
+        constexpr int kOwn = kBins / kFilterThreads;
+        unsigned long long own[kOwn], sum = 0;
+#pragma unroll
+        for (int i = 0; i < kOwn; ++i) {
+            own[i] = sh.hist_w[threadIdx.x * kOwn + i];
+            sum += own[i];
+        }
+        if (MODE == kModeMass && iter == 0) {
+            const unsigned long long Z = block_sum(sum, sh);
+            const unsigned long long lo = target * Z, hi = __umul64hi(target, Z);
+            target = (hi << 32) | (lo >> 32);
+            if (lo & 0xffffffffull) target += 1;
+        }
+        unsigned long long run = acc + block_exclusive_scan(sum, sh);
+#pragma unroll
+        for (int i = 0; i < kOwn; ++i) {
+            if (run < target && run + own[i] >= target) {
+                sh.bcast[0] = threadIdx.x * kOwn + i;
+                sh.bcast[1] = run;
+                sh.bcast[2] = sh.hist_c[threadIdx.x * kOwn + i];
+            }
+            run += own[i];
+        }
+        __syncthreads();
+        const unsigned long long b = sh.bcast[0];
+        if (b >= kBins) return limit;                 // target beyond the total: everything stays
+        acc = sh.bcast[1];
+        const unsigned long long cnt = sh.bcast[2];
+        r0 += static_cast<uint32_t>(b) << sub;
+        s = sub;
+        __syncthreads();
+
+        if (cnt <= kListCap) {
+            // gather the candidates of the range, sort them, walk the weights
+            if (threadIdx.x == 0) sh.list_n = 0u;
+            __syncthreads();
+            for_each<DTYPE>(row_ptr, V, [&](uint32_t col, uint32_t code) {
+                const uint32_t dist = key_m - code;
+                const unsigned long long comp = (static_cast<unsigned long long>(dist) << 32) | col;
+                if (comp > limit) return;
+                const uint32_t rel = dist - r0;
+                if (s < 32 && (rel >> s) != 0u) return;
+                if (weight(dist) == 0ull) return;
+                const unsigned idx = atomicAdd(&sh.list_n, 1u);
+                if (idx < kListCap) sh.list[idx] = comp;
+            });
+            __syncthreads();
+            const int n = static_cast<int>(min(sh.list_n, static_cast<unsigned>(kListCap)));
+            int len = 2;
+            while (len < n) len <<= 1;
+            for (int i = n + threadIdx.x; i < len; i += kFilterThreads) sh.list[i] = kAll;
+            __syncthreads();
+            sort_list(sh, len);
+            constexpr int kPer = kListCap / kFilterThreads;
+            unsigned long long w[kPer], mine = 0;
+#pragma unroll
+            for (int i = 0; i < kPer; ++i) {
+                const int idx = threadIdx.x * kPer + i;
+                w[i] = idx < n ? weight(static_cast<uint32_t>(sh.list[idx] >> 32)) : 0ull;
+                mine += w[i];
+            }
+            if (threadIdx.x == 0) sh.bcast[0] = limit;
+            unsigned long long at = acc + block_exclusive_scan(mine, sh);
+#pragma unroll
+            for (int i = 0; i < kPer; ++i) {
+                if (at < target && at + w[i] >= target) sh.bcast[0] = sh.list[threadIdx.x * kPer + i];
+                at += w[i];
+            }
+            __syncthreads();
+            const unsigned long long boundary = sh.bcast[0];
+            __syncthreads();
+            return boundary;
+        }
+        if (s == 0) {
+            // more equal logits than the list holds: keep the first `need` of them by column
+            const unsigned long long wt = weight(r0);
+            const unsigned long long need = (target - acc + wt - 1) / wt;     // >= 1
+            constexpr int VEC = DTYPE == SBW_DTYPE_F32 ? 4 : 8;
+            const uint32_t nvec = (V + VEC - 1) / VEC;
+            unsigned long long seen = 0;
+            if (threadIdx.x == 0) sh.bcast[0] = limit;
+            for (uint32_t base = 0; base < nvec && seen < need; base += kFilterThreads) {
+                const uint32_t j = base + threadIdx.x;
+                uint32_t match = 0;                    // bit i: column j VEC + i belongs to the group
+                if (j < nvec) {
+                    const uint4 q = reinterpret_cast<const uint4 *>(row_ptr)[j];
+                    const uint32_t *e = reinterpret_cast<const uint32_t *>(&q);
+#pragma unroll
+                    for (int i = 0; i < VEC; ++i) {
+                        uint32_t bits;
+                        if constexpr (DTYPE == SBW_DTYPE_F32) bits = e[i];
+                        else bits = (i & 1) ? (e[i >> 1] & 0xffff0000u) : (e[i >> 1] << 16);
+                        const uint32_t col = j * VEC + i;
+                        const uint32_t dist = key_m - code_of_bits<DTYPE>(bits);
+                        if (col < V && dist == r0 && ((static_cast<unsigned long long>(dist) << 32) | col) <= limit)
+                            match |= 1u << i;
+                    }
+                }
+                const unsigned long long cntm = __popc(match);
+                const unsigned long long before = seen + block_exclusive_scan(cntm, sh);
+                if (before < need && before + cntm >= need) {
+                    uint32_t left = static_cast<uint32_t>(need - before);   // 1-based rank inside `match`
+                    uint32_t mm = match;
+                    while (left > 1) {
+                        mm &= mm - 1;
+                        --left;
+                    }
+                    sh.bcast[0] = (static_cast<unsigned long long>(r0) << 32) | (j * VEC + (__ffs(mm) - 1));
+                }
+                seen += block_sum(cntm, sh);
+            }
+            __syncthreads();
+            const unsigned long long boundary = sh.bcast[0];
+            __syncthreads();
+            return boundary;
+        }
+    }
+    return limit;
+}
+
+template <int DTYPE>
+__global__ void __launch_bounds__(kFilterThreads)
+filter_sample_kernel(const FilterArgs a) {
+    constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
+    constexpr int kCodeBits = DTYPE == SBW_DTYPE_F32 ? 32 : 16;
+    __shared__ FilterShared sh;
+    const uint32_t V = static_cast<uint32_t>(a.V);
+    for (int64_t row = blockIdx.x; row < a.B; row += gridDim.x) {
+        const char *row_ptr = static_cast<const char *>(a.biased) + row * a.ld * ESIZE;
+        // the row maximum in code space
+        uint32_t best_code = 0;
+        for_each<DTYPE>(row_ptr, V, [&](uint32_t, uint32_t code) { best_code = max(best_code, code); });
+        for (int d = 16; d > 0; d >>= 1) best_code = max(best_code, __shfl_xor_sync(0xffffffffu, best_code, d));
+        __syncthreads();
+        if ((threadIdx.x & 31) == 0) sh.red32[threadIdx.x >> 5] = best_code;
+        __syncthreads();
+        uint32_t key_m = 0;
+        for (int w = 0; w < kFilterWarps; ++w) key_m = max(key_m, sh.red32[w]);
+        const float m = value_of_code<DTYPE>(key_m);
+
+        unsigned long long boundary = kAll;
+        if (a.top_k > 0 && a.top_k < a.V)
+            boundary = select_boundary<DTYPE, kModeCount>(row_ptr, V, key_m, m, a.c, kAll,
+                                                          static_cast<unsigned long long>(a.top_k), kCodeBits, sh);
+        if (a.p32 != 0ull) {
+            // candidates with a weight lie within 41 / c of the maximum
+            int s0 = 0;
+            if (m == m && fabsf(m) != __int_as_float(0x7f800000)) {
+                const float l_lo = __fsub_rn(m, __fdiv_rn(42.0f, a.c));
+                const uint32_t span = key_m - code_of_bits<DTYPE>(__float_as_uint(l_lo));
+                s0 = 32 - __clz(span);
+            }
+            boundary = select_boundary<DTYPE, kModeMass>(row_ptr, V, key_m, m, a.c, boundary, a.p32, s0, sh);
+        }
+
+        // Gumbel-max over the kept candidates
+        unsigned long long best = 0;                  // (encoded score << 32) | ~column
+        unsigned long long kept = 0;
+        const uint32_t rowb = static_cast<uint32_t>(row);
+        for_each<DTYPE>(row_ptr, V, [&](uint32_t col, uint32_t code) {
+            const uint32_t dist = key_m - code;
+            if (((static_cast<unsigned long long>(dist) << 32) | col) > boundary) return;
+            kept += 1;
+            const uint32_t v = a.vocab_offset + col;
+            const uint4 r = philox4x32_10(v >> 2, rowb, a.step_lo, a.step_hi, a.gkeys);
+            const uint32_t k = v & 3u;
+            const uint32_t y = k == 0 ? r.x : k == 1 ? r.y : k == 2 ? r.z : r.w;
+            const float sc = __fmaf_rn(value_of_code<DTYPE>(code), a.inv_tau, gumbel_of_word(y));
+            const uint32_t sb = __float_as_uint(sc);
+            const uint32_t enc = (sb & 0x80000000u) ? ~sb : (sb | 0x80000000u);
+            const unsigned long long cand = (static_cast<unsigned long long>(enc) << 32) | (0xFFFFFFFFu - col);
+            best = cand > best ? cand : best;
+        });
+        for (int d = 16; d > 0; d >>= 1) {
+            const unsigned long long o = __shfl_xor_sync(0xffffffffu, best, d);
+            best = o > best ? o : best;
+        }
+        __syncthreads();
+        if ((threadIdx.x & 31) == 0) sh.red[threadIdx.x >> 5] = best;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned long long top = 0;
+            for (int w = 0; w < kFilterWarps; ++w) top = sh.red[w] > top ? sh.red[w] : top;
+            a.out_tokens[row] = static_cast<int32_t>(0xFFFFFFFFu - static_cast<uint32_t>(top));
+        }
+        const unsigned long long total = block_sum(kept, sh);
+        if (threadIdx.x == 0 && a.out_kept) a.out_kept[row] = static_cast<int32_t>(total);
+        __syncthreads();
+    }
+}
+
+}  // namespace
+}  // namespace sbw
+
+extern "C" size_t sbw_sample_filtered_workspace_bytes(int dtype, int64_t B, int64_t V) {
+    if (B <= 0 || V <= 0 || (dtype != SBW_DTYPE_F32 && dtype != SBW_DTYPE_BF16)) return 0;
+    const size_t es = dtype == SBW_DTYPE_F32 ? 4 : 2;
+    const size_t vp = sbw::align_up(static_cast<size_t>(V), 8);
+    return sbw::align_up(static_cast<size_t>(B) * vp * es, 256);
+}
+
+extern "C" int sbw_bias_sample_filtered(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
+                                        int64_t vocab_offset, const int32_t *ctx_tokens, int ctx_width,
+                                        uint64_t key, double gamma, float delta, int scheme, float temperature,
+                                        int64_t top_k, double top_p, uint64_t rng_seed, uint64_t rng_step,
+                                        int32_t *out_tokens, int32_t *out_kept, void *workspace,
+                                        size_t workspace_bytes, void *stream) {
+    using namespace sbw;
+    if (!valid_common(dtype, ctx_width, gamma, scheme)) return SBW_ERR_INVALID_ARG;
+    if (B < 0 || V < 1 || ld < V || vocab_offset < 0 || top_k < 0) return SBW_ERR_INVALID_ARG;
+    if (!(temperature > 0.0f) || !(top_p > 0.0)) return SBW_ERR_INVALID_ARG;
+    if (B == 0) return SBW_OK;
+    if (!logits || !ctx_tokens || !out_tokens) return SBW_ERR_INVALID_ARG;
+    if (V > 0x7fffffffLL || B > 0xffffffffLL) return SBW_ERR_UNSUPPORTED;
+    const size_t need = sbw_sample_filtered_workspace_bytes(dtype, B, V);
+    if (!workspace || workspace_bytes < need || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
+        return SBW_ERR_WORKSPACE;
+    DeviceInfo di;
+    if (int rc = current_device_info(&di)) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t es = dtype == SBW_DTYPE_F32 ? 4 : 2;
+    const int64_t vp = static_cast<int64_t>(align_up(static_cast<size_t>(V), 8));
+
+    // l' of Eq. 2, in the logits' precision, into the workspace
+    SBW_CUDA_TRY(cudaMemcpy2DAsync(workspace, vp * es, logits, ld * es, V * es, B, cudaMemcpyDeviceToDevice, s));
+    if (int rc = bias_logits_impl(workspace, dtype, B, V, vp, vocab_offset, ctx_tokens, ctx_width, key, gamma,
+                                  delta, scheme, s))
+        return rc;
+
+    FilterArgs a;
+    a.biased = workspace;
+    a.B = B;
+    a.V = V;
+    a.ld = vp;
+    a.vocab_offset = static_cast<uint32_t>(vocab_offset);
+    a.inv_tau = 1.0f / temperature;
+    a.c = static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
+    a.top_k = top_k;
+    a.p32 = 0;
+    if (top_p < 1.0) {
+        const double scaled = std::floor(top_p * 4294967296.0);
+        a.p32 = scaled < 1.0 ? 1ull : static_cast<uint64_t>(scaled);
+    }
+    a.step_lo = static_cast<uint32_t>(rng_step);
+    a.step_hi = static_cast<uint32_t>(rng_step >> 32);
+    a.gkeys = make_block_keys(static_cast<uint32_t>(rng_seed), static_cast<uint32_t>(rng_seed >> 32));
+    a.out_tokens = out_tokens;
+    a.out_kept = out_kept;
+    const int64_t cap = 2LL * di.sm_count;
+    const unsigned grid = static_cast<unsigned>(B < cap ? B : cap);
+    if (dtype == SBW_DTYPE_F32) filter_sample_kernel<SBW_DTYPE_F32><<<grid, kFilterThreads, 0, s>>>(a);
+    else filter_sample_kernel<SBW_DTYPE_BF16><<<grid, kFilterThreads, 0, s>>>(a);
+    SBW_CUDA_TRY(cudaGetLastError());
+    return SBW_OK;
+}
