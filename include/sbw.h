@@ -333,7 +333,8 @@ int sbw_roc_auc(const double *z, const uint8_t *labels, int64_t n, double *out_a
  *   out_kept    device [B] int32 or NULL: the number of candidates left per row.
  *   workspace   device, 256-byte aligned, at least sbw_sample_filtered_workspace_bytes(dtype, B, V)
  *               bytes (a biased copy of the logits); contents undefined afterwards.
- * Rows that contain NaN are not supported (the result is some kept column).
+ * Rows that contain NaN are not supported (the result is some kept column).  V <= 2^21
+ * (SBW_ERR_UNSUPPORTED beyond: the weight histogram's counters hold that many candidates).
  */
 size_t sbw_sample_filtered_workspace_bytes(int dtype, int64_t B, int64_t V);
 int sbw_bias_sample_filtered(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld,

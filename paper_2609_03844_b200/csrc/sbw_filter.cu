@@ -54,10 +54,22 @@ struct FilterArgs {
     int32_t *out_kept;     // nullable
 };
 
+// Weights go into the histogram as four 11-bit limbs, each its own array of 32-bit counters:
+// native 32-bit shared-memory adds instead of 64-bit compare-and-swap loops, which crawl when the
+// candidates crowd into a few bins (bf16 logits have a few hundred distinct values near the top).
+// A limb counter holds up to 2^21 candidates' worth.  The list reuses the histogram's space.
+constexpr int kLimbs = 4;
+constexpr int kLimbBits = 11;
+constexpr int64_t kMaxFilterV = int64_t(1) << 21;
+
 struct FilterShared {
-    unsigned long long hist_w[kBins];
-    unsigned int hist_c[kBins];
-    unsigned long long list[kListCap];
+    union {
+        struct {
+            unsigned int hist_c[kBins];
+            unsigned int hist_l[kLimbs][kBins];
+        };
+        unsigned long long list[kListCap];
+    };
     unsigned long long red[kFilterWarps];
     unsigned long long bcast[4];
     unsigned int list_n;
@@ -214,8 +226,9 @@ __device__ unsigned long long select_boundary(const char *row_ptr, uint32_t V, u
     for (int iter = 0; iter < 5; ++iter) {           // the range loses 11 bits per iteration
         const int sub = s > kBinBits ? s - kBinBits : 0;
         for (int i = threadIdx.x; i < kBins; i += kFilterThreads) {
-            sh.hist_w[i] = 0ull;
             sh.hist_c[i] = 0u;
+#pragma unroll
+            for (int l = 0; l < kLimbs; ++l) sh.hist_l[l][i] = 0u;
         }
         if (threadIdx.x == 0) sh.bcast[0] = kBins;
         __syncthreads();
@@ -227,8 +240,14 @@ __device__ unsigned long long select_boundary(const char *row_ptr, uint32_t V, u
             const unsigned long long w = weight(dist);
             if (w == 0ull) return;
             const uint32_t bin = rel >> sub;
-            atomicAdd(&sh.hist_w[bin], w);
             atomicAdd(&sh.hist_c[bin], 1u);
+            if (MODE == kModeMass) {
+#pragma unroll
+                for (int l = 0; l < kLimbs; ++l) {
+                    const unsigned int part = static_cast<unsigned int>(w >> (l * kLimbBits)) & ((1u << kLimbBits) - 1u);
+                    if (part) atomicAdd(&sh.hist_l[l][bin], part);
+                }
+            }
         });
         __syncthreads();
         // every thread owns kBins / kFilterThreads consecutive bins
@@ -236,7 +255,15 @@ __device__ unsigned long long select_boundary(const char *row_ptr, uint32_t V, u
         unsigned long long own[kOwn], sum = 0;
 #pragma unroll
         for (int i = 0; i < kOwn; ++i) {
-            own[i] = sh.hist_w[threadIdx.x * kOwn + i];
+            const int bin = threadIdx.x * kOwn + i;
+            if (MODE == kModeCount) {
+                own[i] = sh.hist_c[bin];
+            } else {
+                own[i] = 0ull;
+#pragma unroll
+                for (int l = 0; l < kLimbs; ++l)
+                    own[i] += static_cast<unsigned long long>(sh.hist_l[l][bin]) << (l * kLimbBits);
+            }
             sum += own[i];
         }
         if (MODE == kModeMass && iter == 0) {
@@ -352,59 +379,147 @@ __device__ unsigned long long select_boundary(const char *row_ptr, uint32_t V, u
     return limit;
 }
 
+// Gumbel-max score of one candidate, packed for a max-reduction: (order-encoded score << 32) |
+// ~column, so that the larger score wins and equal scores go to the lower column.
+template <int DTYPE>
+__device__ __forceinline__ unsigned long long packed_score(const FilterArgs &a, uint32_t rowb, uint32_t col,
+                                                           uint32_t code) {
+    const uint32_t v = a.vocab_offset + col;
+    const uint4 r = philox4x32_10(v >> 2, rowb, a.step_lo, a.step_hi, a.gkeys);
+    const uint32_t k = v & 3u;
+    const uint32_t y = k == 0 ? r.x : k == 1 ? r.y : k == 2 ? r.z : r.w;
+    const float sc = __fmaf_rn(value_of_code<DTYPE>(code), a.inv_tau, gumbel_of_word(y));
+    const uint32_t sb = __float_as_uint(sc);
+    const uint32_t enc = (sb & 0x80000000u) ? ~sb : (sb | 0x80000000u);
+    return (static_cast<unsigned long long>(enc) << 32) | (0xFFFFFFFFu - col);
+}
+
+// One CTA per row.  The usual case -- the kept candidates are a few hundred at most -- needs two
+// passes over the row and no histogram: pass A finds every thread's largest code; the r-th
+// largest of those maxima is a floor that at least r candidates reach; pass B gathers everything
+// at or above the floor into the shared-memory list (and adds up the weights of the whole row);
+// the sorted list is then the head of the row's order, complete down to the floor, and if the
+// top-k cut and the top-p crossing both fall inside it, the sample is drawn from the list.
+// Otherwise (a deep nucleus, flat or tied rows, a large top_k) the radix descent above finds the
+// boundary and one more pass over the row draws the sample.
 template <int DTYPE>
 __global__ void __launch_bounds__(kFilterThreads)
 filter_sample_kernel(const FilterArgs a) {
     constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
     constexpr int kCodeBits = DTYPE == SBW_DTYPE_F32 ? 32 : 16;
+    constexpr int kPer = kListCap / kFilterThreads;
     __shared__ FilterShared sh;
     const uint32_t V = static_cast<uint32_t>(a.V);
+    const bool use_k = a.top_k > 0 && a.top_k < a.V;
+    const bool use_p = a.p32 != 0ull;
     for (int64_t row = blockIdx.x; row < a.B; row += gridDim.x) {
         const char *row_ptr = static_cast<const char *>(a.biased) + row * a.ld * ESIZE;
-        // the row maximum in code space
-        uint32_t best_code = 0;
-        for_each<DTYPE>(row_ptr, V, [&](uint32_t, uint32_t code) { best_code = max(best_code, code); });
-        for (int d = 16; d > 0; d >>= 1) best_code = max(best_code, __shfl_xor_sync(0xffffffffu, best_code, d));
+        const uint32_t rowb = static_cast<uint32_t>(row);
+        // pass A: per-thread maxima, sorted descending (as ~code ascending) in the list area
+        uint32_t my_max = 0;
+        for_each<DTYPE>(row_ptr, V, [&](uint32_t, uint32_t code) { my_max = max(my_max, code); });
+        sh.list[threadIdx.x] = static_cast<unsigned long long>(~my_max);
+        if (threadIdx.x == 0) sh.list_n = 0u;
         __syncthreads();
-        if ((threadIdx.x & 31) == 0) sh.red32[threadIdx.x >> 5] = best_code;
-        __syncthreads();
-        uint32_t key_m = 0;
-        for (int w = 0; w < kFilterWarps; ++w) key_m = max(key_m, sh.red32[w]);
+        sort_list(sh, kFilterThreads);
+        const uint32_t key_m = ~static_cast<uint32_t>(sh.list[0]);
+        const int rank = use_k ? static_cast<int>(min(a.top_k, static_cast<int64_t>(kFilterThreads))) : 384;
+        const uint32_t floor_code = ~static_cast<uint32_t>(sh.list[rank - 1]);
         const float m = value_of_code<DTYPE>(key_m);
+        __syncthreads();
 
-        unsigned long long boundary = kAll;
-        if (a.top_k > 0 && a.top_k < a.V)
-            boundary = select_boundary<DTYPE, kModeCount>(row_ptr, V, key_m, m, a.c, kAll,
-                                                          static_cast<unsigned long long>(a.top_k), kCodeBits, sh);
-        if (a.p32 != 0ull) {
-            // candidates with a weight lie within 41 / c of the maximum
-            int s0 = 0;
-            if (m == m && fabsf(m) != __int_as_float(0x7f800000)) {
-                const float l_lo = __fsub_rn(m, __fdiv_rn(42.0f, a.c));
-                const uint32_t span = key_m - code_of_bits<DTYPE>(__float_as_uint(l_lo));
-                s0 = 32 - __clz(span);
+        // candidates with a weight lie within 41 / c of the maximum: code_lo is below all of them
+        uint32_t code_lo = key_m;
+        if (m == m && fabsf(m) != __int_as_float(0x7f800000))
+            code_lo = code_of_bits<DTYPE>(__float_as_uint(__fsub_rn(m, __fdiv_rn(42.0f, a.c))));
+
+        // pass B: gather the head of the order; total weight of the row when top-p works on all of it
+        unsigned long long z_local = 0;
+        if (use_k || use_p) {
+            for_each<DTYPE>(row_ptr, V, [&](uint32_t col, uint32_t code) {
+                const uint32_t dist = key_m - code;
+                if (use_p && !use_k && code >= code_lo)
+                    z_local += nucleus_weight(value_of_code<DTYPE>(code), m, dist == 0u, a.c);
+                if (code >= floor_code && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= kListCap) {
+                    const unsigned idx = atomicAdd(&sh.list_n, 1u);
+                    if (idx < kListCap) sh.list[idx] = (static_cast<unsigned long long>(dist) << 32) | col;
+                }
+            });
+        }
+        __syncthreads();
+        const unsigned gathered = sh.list_n;
+        bool resolved = (use_k || use_p) && gathered <= kListCap;
+        int n2 = 0;                                   // candidates kept, a prefix of the sorted list
+        if (resolved) {
+            const int n = static_cast<int>(gathered);
+            int len = 2;
+            while (len < n) len <<= 1;
+            __syncthreads();
+            for (int i = n + threadIdx.x; i < len; i += kFilterThreads) sh.list[i] = kAll;
+            __syncthreads();
+            sort_list(sh, len);
+            int n1 = n;
+            if (use_k) {
+                if (a.top_k <= n) n1 = static_cast<int>(a.top_k);
+                else resolved = false;
             }
-            boundary = select_boundary<DTYPE, kModeMass>(row_ptr, V, key_m, m, a.c, boundary, a.p32, s0, sh);
+            n2 = n1;
+            if (resolved && use_p) {
+                unsigned long long w[kPer], mine = 0;
+#pragma unroll
+                for (int i = 0; i < kPer; ++i) {
+                    const int idx = threadIdx.x * kPer + i;
+                    const uint32_t dist = static_cast<uint32_t>(sh.list[idx < len ? idx : 0] >> 32);
+                    w[i] = idx < n1 ? nucleus_weight(value_of_code<DTYPE>(key_m - dist), m, dist == 0u, a.c) : 0ull;
+                    mine += w[i];
+                }
+                const unsigned long long in_list = block_sum(mine, sh);
+                const unsigned long long Z = use_k ? in_list : block_sum(z_local, sh);
+                const unsigned long long lo = a.p32 * Z, hi = __umul64hi(a.p32, Z);
+                unsigned long long target = (hi << 32) | (lo >> 32);
+                if (lo & 0xffffffffull) target += 1;
+                if (threadIdx.x == 0) sh.bcast[0] = kAll;
+                unsigned long long at = block_exclusive_scan(mine, sh);
+#pragma unroll
+                for (int i = 0; i < kPer; ++i) {
+                    if (at < target && at + w[i] >= target) sh.bcast[0] = threadIdx.x * kPer + i;
+                    at += w[i];
+                }
+                __syncthreads();
+                const unsigned long long cross = sh.bcast[0];
+                __syncthreads();
+                if (cross == kAll) resolved = false;      // the nucleus reaches below the floor
+                else n2 = static_cast<int>(cross) + 1;
+            }
         }
 
-        // Gumbel-max over the kept candidates
-        unsigned long long best = 0;                  // (encoded score << 32) | ~column
-        unsigned long long kept = 0;
-        const uint32_t rowb = static_cast<uint32_t>(row);
-        for_each<DTYPE>(row_ptr, V, [&](uint32_t col, uint32_t code) {
-            const uint32_t dist = key_m - code;
-            if (((static_cast<unsigned long long>(dist) << 32) | col) > boundary) return;
-            kept += 1;
-            const uint32_t v = a.vocab_offset + col;
-            const uint4 r = philox4x32_10(v >> 2, rowb, a.step_lo, a.step_hi, a.gkeys);
-            const uint32_t k = v & 3u;
-            const uint32_t y = k == 0 ? r.x : k == 1 ? r.y : k == 2 ? r.z : r.w;
-            const float sc = __fmaf_rn(value_of_code<DTYPE>(code), a.inv_tau, gumbel_of_word(y));
-            const uint32_t sb = __float_as_uint(sc);
-            const uint32_t enc = (sb & 0x80000000u) ? ~sb : (sb | 0x80000000u);
-            const unsigned long long cand = (static_cast<unsigned long long>(enc) << 32) | (0xFFFFFFFFu - col);
-            best = cand > best ? cand : best;
-        });
+        unsigned long long best = 0, kept = 0;
+        if (resolved) {
+            for (int i = threadIdx.x; i < n2; i += kFilterThreads) {
+                const unsigned long long comp = sh.list[i];
+                const unsigned long long cand = packed_score<DTYPE>(a, rowb, static_cast<uint32_t>(comp),
+                                                                    key_m - static_cast<uint32_t>(comp >> 32));
+                best = cand > best ? cand : best;
+            }
+            kept = threadIdx.x == 0 ? n2 : 0;
+        } else {
+            __syncthreads();
+            unsigned long long boundary = kAll;
+            if (use_k)
+                boundary = select_boundary<DTYPE, kModeCount>(row_ptr, V, key_m, m, a.c, kAll,
+                                                              static_cast<unsigned long long>(a.top_k), kCodeBits, sh);
+            if (use_p) {
+                const int s0 = 32 - __clz(key_m - code_lo);
+                boundary = select_boundary<DTYPE, kModeMass>(row_ptr, V, key_m, m, a.c, boundary, a.p32, s0, sh);
+            }
+            for_each<DTYPE>(row_ptr, V, [&](uint32_t col, uint32_t code) {
+                const uint32_t dist = key_m - code;
+                if (((static_cast<unsigned long long>(dist) << 32) | col) > boundary) return;
+                kept += 1;
+                const unsigned long long cand = packed_score<DTYPE>(a, rowb, col, code);
+                best = cand > best ? cand : best;
+            });
+        }
         for (int d = 16; d > 0; d >>= 1) {
             const unsigned long long o = __shfl_xor_sync(0xffffffffu, best, d);
             best = o > best ? o : best;
@@ -445,7 +560,7 @@ extern "C" int sbw_bias_sample_filtered(const void *logits, int dtype, int64_t B
     if (!(temperature > 0.0f) || !(top_p > 0.0)) return SBW_ERR_INVALID_ARG;
     if (B == 0) return SBW_OK;
     if (!logits || !ctx_tokens || !out_tokens) return SBW_ERR_INVALID_ARG;
-    if (V > 0x7fffffffLL || B > 0xffffffffLL) return SBW_ERR_UNSUPPORTED;
+    if (V > kMaxFilterV || B > 0xffffffffLL) return SBW_ERR_UNSUPPORTED;
     const size_t need = sbw_sample_filtered_workspace_bytes(dtype, B, V);
     if (!workspace || workspace_bytes < need || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
         return SBW_ERR_WORKSPACE;
