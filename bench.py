@@ -477,7 +477,8 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
 
 
 PROFILE_CASES = ("topk40_fp32_selfsalt", "bias_bf16_context", "bias_bf16_selfsalt", "bias_fp32_context", "bias_fp32_selfsalt",
-                 "detect_context", "detect_selfsalt", "sample_bf16_context", "sample_bf16_selfsalt")
+                 "detect_context", "detect_selfsalt", "sample_bf16_context", "sample_bf16_selfsalt",
+                 "detectunique_context", "filtered_bf16_context")
 
 
 def run_profile_case(name: str, launches: int) -> None:
@@ -491,15 +492,27 @@ def run_profile_case(name: str, launches: int) -> None:
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
     kind, dt, scheme_name = (name.split("_") + [""])[:3] if not name.startswith("detect") else \
-        ("detect", "", name.split("_")[1])
+        (name.split("_")[0], "", name.split("_")[1])
     scheme = sbw.SCHEME_SELFSALT if scheme_name == "selfsalt" else sbw.SCHEME_CONTEXT
-    if kind == "detect":
+    if kind in ("detect", "detectunique"):
         N = 100000
         tokens, lengths = inputs.null_token_streams(N, 64, 1024, V2, seed=500, device=dev)
         counts = torch.empty(N, dtype=torch.int32, device=dev)
         z = torch.empty(N, dtype=torch.float64, device=dev)
-        ws = torch.empty(sbw.sbw_detect_workspace_bytes(N), dtype=torch.uint8, device=dev)
-        fn = lambda i: sbw.sbw_detect(tokens, lengths, KEY, 0.25, scheme, counts, z, workspace=ws)  # noqa: E731
+        if kind == "detect":
+            ws = torch.empty(sbw.sbw_detect_workspace_bytes(N), dtype=torch.uint8, device=dev)
+            fn = lambda i: sbw.sbw_detect(tokens, lengths, KEY, 0.25, scheme, counts, z, workspace=ws)  # noqa: E731
+        else:
+            ws = torch.empty(sbw.sbw_detect_unique_workspace_bytes(N, tokens.numel(), 1024), dtype=torch.uint8,
+                             device=dev)
+            fn = lambda i: sbw.sbw_detect_unique(tokens, lengths, 1024, KEY, 0.25, scheme, counts, z, ws)  # noqa: E731
+    elif kind == "filtered":
+        B = 512
+        x = inputs.logits_normal(B, V2, 4.0, torch.bfloat16, seed=1, device=dev)
+        ctx = inputs.uniform_tokens((B, 1), V2, seed=2, device=dev)
+        ids = torch.empty(B, dtype=torch.int32, device=dev)
+        ws = torch.empty(sbw.sbw_sample_filtered_workspace_bytes(x.dtype, B, V2), dtype=torch.uint8, device=dev)
+        fn = lambda i: sbw.sbw_bias_sample_filtered(x, ctx, KEY, 0.25, 2.0, scheme, 0.7, 0, 0.8, 0xC4, i, ids, ws)  # noqa: E731
     else:
         B, V, dtype = (512, V2, torch.bfloat16) if dt == "bf16" else (256, 151936, torch.float32)
         x = inputs.logits_normal(B, V, 4.0, dtype, seed=1, device=dev)
