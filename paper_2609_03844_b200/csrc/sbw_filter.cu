@@ -19,6 +19,7 @@
 //            equal logits, cut by column with one ordered counting pass.
 //   sample   one last pass draws Gumbel variates for the kept candidates only and takes the
 //            arg max of fmaf(l', 1/tau, g), ties to the lowest column.
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
 #include "sbw_common.cuh"
@@ -74,6 +75,9 @@ struct FilterShared {
     unsigned long long bcast[4];
     unsigned int list_n;
     unsigned int red32[kFilterWarps];
+    // what the CTAs of a cluster tell each other about their parts of the row
+    unsigned int part_max, part_floor;
+    unsigned long long part_z;
 };
 
 __device__ __forceinline__ uint32_t order_code(uint32_t bits) {
@@ -121,13 +125,18 @@ __device__ __forceinline__ unsigned long long nucleus_weight(float l, float m, b
     return __float2ull_rz(__fmul_rn(p, scale));
 }
 
-// Calls f(column, code) for every column of the row, 16 bytes per load, several loads in flight.
+// The row is padded to whole 16-byte vectors; loads are 16 bytes wide, several in flight.
+template <int DTYPE>
+__device__ __forceinline__ uint32_t vectors_of(uint32_t V) {
+    return (V + (DTYPE == SBW_DTYPE_F32 ? 4 : 8) - 1) / (DTYPE == SBW_DTYPE_F32 ? 4 : 8);
+}
+
+// Calls f(column, code) for the columns of 16-byte vectors [vec_begin, nvec) of the row.
 template <int DTYPE, typename F>
-__device__ __forceinline__ void for_each(const char *row_ptr, uint32_t V, F f) {
+__device__ __forceinline__ void for_each(const char *row_ptr, uint32_t V, uint32_t vec_begin, uint32_t nvec, F f) {
     constexpr int VEC = DTYPE == SBW_DTYPE_F32 ? 4 : 8;
     constexpr int kInFlight = 4;
-    const uint32_t nvec = (V + VEC - 1) / VEC;        // the row is padded to whole vectors
-    for (uint32_t j0 = threadIdx.x; j0 < nvec; j0 += kInFlight * kFilterThreads) {
+    for (uint32_t j0 = vec_begin + threadIdx.x; j0 < nvec; j0 += kInFlight * kFilterThreads) {
         uint4 w[kInFlight];
 #pragma unroll
         for (int u = 0; u < kInFlight; ++u) {
@@ -149,6 +158,11 @@ __device__ __forceinline__ void for_each(const char *row_ptr, uint32_t V, F f) {
             }
         }
     }
+}
+
+template <int DTYPE, typename F>
+__device__ __forceinline__ void for_each(const char *row_ptr, uint32_t V, F f) {
+    for_each<DTYPE>(row_ptr, V, 0u, vectors_of<DTYPE>(V), f);
 }
 
 __device__ __forceinline__ unsigned long long warp_sum(unsigned long long x) {
@@ -394,39 +408,64 @@ __device__ __forceinline__ unsigned long long packed_score(const FilterArgs &a, 
     return (static_cast<unsigned long long>(enc) << 32) | (0xFFFFFFFFu - col);
 }
 
-// One CTA per row.  The usual case -- the kept candidates are a few hundred at most -- needs two
-// passes over the row and no histogram: pass A finds every thread's largest code; the r-th
-// largest of those maxima is a floor that at least r candidates reach; pass B gathers everything
-// at or above the floor into the shared-memory list (and adds up the weights of the whole row);
-// the sorted list is then the head of the row's order, complete down to the floor, and if the
-// top-k cut and the top-p crossing both fall inside it, the sample is drawn from the list.
-// Otherwise (a deep nucleus, flat or tied rows, a large top_k) the radix descent above finds the
-// boundary and one more pass over the row draws the sample.
-template <int DTYPE>
+// One CTA per row (CS = 1), or a cluster of CS CTAs per row for small batches.  The usual case --
+// the kept candidates are a few hundred at most -- needs two passes over the row and no
+// histogram: pass A finds every thread's largest code; the r-th largest of those maxima is a
+// floor that at least r candidates reach; pass B gathers everything at or above the floor into
+// the shared-memory list (and adds up the weights of the whole row); the sorted list is then the
+// head of the row's order, complete down to the floor, and if the top-k cut and the top-p
+// crossing both fall inside it, the sample is drawn from the list.  Otherwise (a deep nucleus,
+// flat or tied rows, a large top_k) the radix descent above finds the boundary and one more pass
+// over the row draws the sample.
+// In a cluster every CTA runs the two passes on its own CS-th of the row; the CTAs exchange their
+// maxima and floors (the smallest of the local floors, each reached by r / CS local candidates,
+// is reached by r candidates of the row), then CTA 0 pulls the other lists and weight sums over
+// distributed shared memory and finishes the row alone.  All CTAs pass the same three cluster
+// barriers whatever the data; nothing spins.
+template <int DTYPE, int CS>
 __global__ void __launch_bounds__(kFilterThreads)
 filter_sample_kernel(const FilterArgs a) {
     constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
     constexpr int kCodeBits = DTYPE == SBW_DTYPE_F32 ? 32 : 16;
     constexpr int kPer = kListCap / kFilterThreads;
     __shared__ FilterShared sh;
+    namespace cg = cooperative_groups;
     const uint32_t V = static_cast<uint32_t>(a.V);
+    const uint32_t nvec = vectors_of<DTYPE>(V);
     const bool use_k = a.top_k > 0 && a.top_k < a.V;
     const bool use_p = a.p32 != 0ull;
-    for (int64_t row = blockIdx.x; row < a.B; row += gridDim.x) {
+    const unsigned part = CS > 1 ? blockIdx.x % CS : 0u;          // this CTA's part of the row
+    const int64_t first_row = CS > 1 ? blockIdx.x / CS : blockIdx.x;
+    const int64_t row_step = CS > 1 ? a.B : gridDim.x;            // a cluster handles exactly one row
+    for (int64_t row = first_row; row < a.B; row += row_step) {
         const char *row_ptr = static_cast<const char *>(a.biased) + row * a.ld * ESIZE;
         const uint32_t rowb = static_cast<uint32_t>(row);
+        const uint32_t vec_lo = static_cast<uint32_t>(static_cast<uint64_t>(nvec) * part / CS);
+        const uint32_t vec_hi = static_cast<uint32_t>(static_cast<uint64_t>(nvec) * (part + 1) / CS);
         // pass A: per-thread maxima, sorted descending (as ~code ascending) in the list area
         uint32_t my_max = 0;
-        for_each<DTYPE>(row_ptr, V, [&](uint32_t, uint32_t code) { my_max = max(my_max, code); });
+        for_each<DTYPE>(row_ptr, V, vec_lo, vec_hi, [&](uint32_t, uint32_t code) { my_max = max(my_max, code); });
         sh.list[threadIdx.x] = static_cast<unsigned long long>(~my_max);
         if (threadIdx.x == 0) sh.list_n = 0u;
         __syncthreads();
         sort_list(sh, kFilterThreads);
-        const uint32_t key_m = ~static_cast<uint32_t>(sh.list[0]);
-        const int rank = use_k ? static_cast<int>(min(a.top_k, static_cast<int64_t>(kFilterThreads))) : 384;
-        const uint32_t floor_code = ~static_cast<uint32_t>(sh.list[rank - 1]);
-        const float m = value_of_code<DTYPE>(key_m);
+        uint32_t key_m = ~static_cast<uint32_t>(sh.list[0]);
+        const int want = use_k ? static_cast<int>(min(a.top_k, static_cast<int64_t>(kFilterThreads))) : 384;
+        uint32_t floor_code = ~static_cast<uint32_t>(sh.list[(want + CS - 1) / CS - 1]);
         __syncthreads();
+        if constexpr (CS > 1) {
+            if (threadIdx.x == 0) {
+                sh.part_max = key_m;
+                sh.part_floor = floor_code;
+            }
+            cg::this_cluster().sync();
+            for (unsigned r = 0; r < CS; ++r) {
+                const FilterShared *other = cg::this_cluster().map_shared_rank(&sh, r);
+                key_m = max(key_m, other->part_max);
+                floor_code = min(floor_code, other->part_floor);
+            }
+        }
+        const float m = value_of_code<DTYPE>(key_m);
 
         // candidates with a weight lie within 41 / c of the maximum: code_lo is below all of them
         uint32_t code_lo = key_m;
@@ -436,7 +475,7 @@ filter_sample_kernel(const FilterArgs a) {
         // pass B: gather the head of the order; total weight of the row when top-p works on all of it
         unsigned long long z_local = 0;
         if (use_k || use_p) {
-            for_each<DTYPE>(row_ptr, V, [&](uint32_t col, uint32_t code) {
+            for_each<DTYPE>(row_ptr, V, vec_lo, vec_hi, [&](uint32_t col, uint32_t code) {
                 const uint32_t dist = key_m - code;
                 if (use_p && !use_k && code >= code_lo)
                     z_local += nucleus_weight(value_of_code<DTYPE>(code), m, dist == 0u, a.c);
@@ -446,8 +485,27 @@ filter_sample_kernel(const FilterArgs a) {
                 }
             });
         }
+        unsigned long long z_all = (use_p && !use_k) ? block_sum(z_local, sh) : 0ull;
         __syncthreads();
-        const unsigned gathered = sh.list_n;
+        unsigned gathered = sh.list_n;
+        if constexpr (CS > 1) {
+            if (threadIdx.x == 0) sh.part_z = z_all;
+            cg::this_cluster().sync();
+            if (part == 0) {
+                // pull the other parts: list entries behind the own ones, weight sums added up
+                for (unsigned r = 1; r < CS; ++r) {
+                    const FilterShared *other = cg::this_cluster().map_shared_rank(&sh, r);
+                    const unsigned n_r = other->list_n;
+                    if (gathered <= kListCap && n_r <= kListCap && gathered + n_r <= kListCap)
+                        for (unsigned i = threadIdx.x; i < n_r; i += kFilterThreads) sh.list[gathered + i] = other->list[i];
+                    gathered = (gathered > kListCap || n_r > kListCap) ? kListCap + 1 : gathered + n_r;
+                    z_all += other->part_z;
+                }
+            }
+            cg::this_cluster().sync();               // the other CTAs' shared memory has been read
+            if (part != 0) return;
+            __syncthreads();
+        }
         bool resolved = (use_k || use_p) && gathered <= kListCap;
         int n2 = 0;                                   // candidates kept, a prefix of the sorted list
         if (resolved) {
@@ -474,7 +532,7 @@ filter_sample_kernel(const FilterArgs a) {
                     mine += w[i];
                 }
                 const unsigned long long in_list = block_sum(mine, sh);
-                const unsigned long long Z = use_k ? in_list : block_sum(z_local, sh);
+                const unsigned long long Z = use_k ? in_list : z_all;
                 const unsigned long long lo = a.p32 * Z, hi = __umul64hi(a.p32, Z);
                 unsigned long long target = (hi << 32) | (lo >> 32);
                 if (lo & 0xffffffffull) target += 1;
@@ -538,6 +596,27 @@ filter_sample_kernel(const FilterArgs a) {
     }
 }
 
+template <int DTYPE>
+cudaError_t launch_cluster(const FilterArgs &a, int cs, cudaStream_t s) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(a.B * cs));
+    cfg.blockDim = dim3(kFilterThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(cs);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    switch (cs) {
+        case 8: return cudaLaunchKernelEx(&cfg, filter_sample_kernel<DTYPE, 8>, a);
+        case 4: return cudaLaunchKernelEx(&cfg, filter_sample_kernel<DTYPE, 4>, a);
+        default: return cudaLaunchKernelEx(&cfg, filter_sample_kernel<DTYPE, 2>, a);
+    }
+}
+
 }  // namespace
 }  // namespace sbw
 
@@ -595,10 +674,17 @@ extern "C" int sbw_bias_sample_filtered(const void *logits, int dtype, int64_t B
     a.gkeys = make_block_keys(static_cast<uint32_t>(rng_seed), static_cast<uint32_t>(rng_seed >> 32));
     a.out_tokens = out_tokens;
     a.out_kept = out_kept;
+    // small batches: a cluster of CTAs per row, as many as keeps every SM busy with two CTAs
     const int64_t cap = 2LL * di.sm_count;
-    const unsigned grid = static_cast<unsigned>(B < cap ? B : cap);
-    if (dtype == SBW_DTYPE_F32) filter_sample_kernel<SBW_DTYPE_F32><<<grid, kFilterThreads, 0, s>>>(a);
-    else filter_sample_kernel<SBW_DTYPE_BF16><<<grid, kFilterThreads, 0, s>>>(a);
+    const int cs = B * 8 <= cap ? 8 : B * 4 <= cap ? 4 : B * 2 <= cap ? 2 : 1;
+    if (cs == 1) {
+        const unsigned grid = static_cast<unsigned>(B < cap ? B : cap);
+        if (dtype == SBW_DTYPE_F32) filter_sample_kernel<SBW_DTYPE_F32, 1><<<grid, kFilterThreads, 0, s>>>(a);
+        else filter_sample_kernel<SBW_DTYPE_BF16, 1><<<grid, kFilterThreads, 0, s>>>(a);
+    } else {
+        SBW_CUDA_TRY(dtype == SBW_DTYPE_F32 ? launch_cluster<SBW_DTYPE_F32>(a, cs, s)
+                                            : launch_cluster<SBW_DTYPE_BF16>(a, cs, s));
+    }
     SBW_CUDA_TRY(cudaGetLastError());
     return SBW_OK;
 }

@@ -133,3 +133,17 @@ def test_argument_checks():
     with pytest.raises(sbw.SbwError) as e:
         sbw.sbw_bias_sample_filtered(x, ctx, KEY, 0.25, 2.0, 0, 0.7, 0, 0.8, 1, 0, ids, ws[:16])
     assert e.value.code == -3
+
+
+@pytest.mark.parametrize("B", [37, 38, 74, 75, 148, 149, 300])
+def test_every_cluster_size(B):
+    """Small batches split a row over 8, 4 or 2 CTAs; larger ones take one CTA per row."""
+    V = 6007
+    x = inputs.logits_normal(B, V, 1.5, torch.bfloat16, seed=300 + B)
+    x[1] = 0.0                                                  # a flat row: the list overflows, radix path
+    x[2, :3000] = 3.0                                           # a big group of ties at the top
+    ctx = inputs.uniform_tokens((B, 1), V, seed=400 + B)
+    _check(x, ctx, sbw.SCHEME_CONTEXT, 0.7, 0, 0.8)
+    _check(x, ctx, sbw.SCHEME_SELFSALT, 0.7, 40, 0.9)
+    _check(x, ctx, sbw.SCHEME_CONTEXT, 1.0, 700, 1.0)
+    _check(x.float(), ctx, sbw.SCHEME_CONTEXT, 0.7, 0, 0.97)
