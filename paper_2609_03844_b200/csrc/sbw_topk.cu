@@ -14,6 +14,7 @@
 // If the list overflows (rows of equal values, k > 256) the CTA falls back to k rounds of "largest
 // composite below the previous one", a block reduction each, and one pass that biases every
 // column at or above the k-th composite: slow, but it needs no assumption about the data.
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
 #include "sbw_common.cuh"
@@ -53,16 +54,16 @@ __device__ __forceinline__ uint64_t composite(uint32_t code, uint32_t col) {
     return (static_cast<uint64_t>(code) << 32) | (0xFFFFFFFFu - col);
 }
 
-// Calls f(column, code) for the columns of one row that this thread owns.
+// Calls f(column, code) for the columns [begin, end) of one row that this thread owns; begin is a
+// multiple of 8 columns.
 template <int DTYPE, int kTopkThreads, typename F>
-__device__ __forceinline__ void for_each_code(const char *row_ptr, uint32_t V, bool vector, F f) {
-    // V here is the number of leading columns to visit (the whole row or a prefix of it)
+__device__ __forceinline__ void for_each_code(const char *row_ptr, uint32_t begin, uint32_t end, bool vector, F f) {
     constexpr int VEC = DTYPE == SBW_DTYPE_F32 ? 4 : 8;
-    uint32_t done = 0;
+    uint32_t done = begin;
     if (vector) {
-        const uint32_t nfull = V / VEC;
+        const uint32_t nfull = end / VEC;
         constexpr int kInFlight = 8;   // independent 128-bit loads per thread before the first use
-        for (uint32_t j0 = threadIdx.x; j0 < nfull; j0 += kInFlight * kTopkThreads) {
+        for (uint32_t j0 = begin / VEC + threadIdx.x; j0 < nfull; j0 += kInFlight * kTopkThreads) {
             uint4 w[kInFlight];
 #pragma unroll
             for (int u = 0; u < kInFlight; ++u) {
@@ -84,9 +85,9 @@ __device__ __forceinline__ void for_each_code(const char *row_ptr, uint32_t V, b
                 }
             }
         }
-        done = nfull * VEC;
+        done = max(begin, nfull * VEC);
     }
-    for (uint32_t c = done + threadIdx.x; c < V; c += kTopkThreads) {
+    for (uint32_t c = done + threadIdx.x; c < end; c += kTopkThreads) {
         uint32_t bits;
         if constexpr (DTYPE == SBW_DTYPE_F32) bits = reinterpret_cast<const uint32_t *>(row_ptr)[c];
         else bits = static_cast<uint32_t>(reinterpret_cast<const uint16_t *>(row_ptr)[c]) << 16;
@@ -129,7 +130,12 @@ __device__ __forceinline__ uint64_t block_max_u64(uint64_t x, uint64_t *sh_red, 
     return *sh_out;
 }
 
-template <int DTYPE, int SCHEME, int kTopkThreads>
+// CS = 1: one CTA per row.  CS > 1 (small batches): a thread-block cluster per row; every CTA runs
+// steps 1 and 2 on its CS-th of the row with ceil(k / CS) in place of k (the smallest of the local
+// bounds is then reached by at least k columns of the row), the bounds travel through distributed
+// shared memory, CTA 0 pulls the other candidate lists and does step 3 (or the fallback) alone.
+// Every CTA passes the same three cluster barriers; nothing spins.
+template <int DTYPE, int SCHEME, int kTopkThreads, int CS>
 __global__ void __launch_bounds__(kTopkThreads)
 topk_kernel(const TopkArgs a) {
     constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
@@ -141,45 +147,75 @@ topk_kernel(const TopkArgs a) {
     __shared__ uint64_t sh_best;
     __shared__ uint32_t sh_floor;
     __shared__ unsigned sh_count;
+    namespace cg = cooperative_groups;
     const uint32_t V = static_cast<uint32_t>(a.V);
     const uint32_t k = static_cast<uint32_t>(a.k);
+    const uint32_t k_part = (k + CS - 1) / CS;
+    const unsigned part = CS > 1 ? blockIdx.x % CS : 0u;
+    const int64_t first_row = CS > 1 ? blockIdx.x / CS : blockIdx.x;
+    const int64_t row_step = CS > 1 ? a.B : gridDim.x;           // a cluster handles exactly one row
+    // this CTA's columns; part boundaries are multiples of 8 columns
+    const uint32_t c_lo = CS > 1 ? static_cast<uint32_t>(static_cast<uint64_t>(V) * part / CS) & ~7u : 0u;
+    const uint32_t c_hi = CS > 1 && part + 1 < CS ? static_cast<uint32_t>(static_cast<uint64_t>(V) * (part + 1) / CS) & ~7u : V;
 
-    for (int64_t row = blockIdx.x; row < a.B; row += gridDim.x) {
+    for (int64_t row = first_row; row < a.B; row += row_step) {
         char *row_ptr = static_cast<char *>(a.logits) + row * a.ld * ESIZE;
 
-        // 1. lower bound of the k-th largest code from a prefix of the row
-        const uint32_t prefix = min(V, static_cast<uint32_t>(kPrefixColumns));
+        // 1. lower bound of the k-th largest code from a prefix of the columns
+        const uint32_t prefix_end = min(c_hi, c_lo + static_cast<uint32_t>(kPrefixColumns / CS));
         uint32_t mx = 0;
-        for_each_code<DTYPE, kTopkThreads>(row_ptr, prefix, a.vector, [&](uint32_t, uint32_t code) { mx = max(mx, code); });
+        for_each_code<DTYPE, kTopkThreads>(row_ptr, c_lo, prefix_end, a.vector,
+                                           [&](uint32_t, uint32_t code) { mx = max(mx, code); });
         mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
         mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
         if ((threadIdx.x & 3) == 0) sh_max[threadIdx.x >> 2] = mx;
         if (threadIdx.x == 0) {
-            sh_floor = 0;            // k > kGroups: no bound, everything is a candidate
+            sh_floor = 0;            // k_part > kGroups: no bound, everything is a candidate
             sh_count = 0;
         }
         __syncthreads();
-        if (k <= kGroups && threadIdx.x < kGroups) {
+        if (k_part <= kGroups && threadIdx.x < kGroups) {
             const uint32_t mine = sh_max[threadIdx.x];
             uint32_t rank = 0;
             for (int u = 0; u < kGroups; ++u) {
                 const uint32_t o = sh_max[u];
                 rank += (o > mine || (o == mine && u < static_cast<int>(threadIdx.x))) ? 1u : 0u;
             }
-            if (rank == k - 1) sh_floor = mine;
+            if (rank == k_part - 1) sh_floor = mine;
         }
         __syncthreads();
-        const uint32_t floor_code = sh_floor;
+        uint32_t floor_code = sh_floor;
+        if constexpr (CS > 1) {
+            cg::this_cluster().sync();
+            for (unsigned r = 0; r < CS; ++r)
+                floor_code = min(floor_code, *cg::this_cluster().map_shared_rank(&sh_floor, r));
+        }
 
-        // 2. candidates: every column of the row that reaches the bound
-        for_each_code<DTYPE, kTopkThreads>(row_ptr, V, a.vector, [&](uint32_t col, uint32_t code) {
+        // 2. candidates: every column that reaches the bound
+        for_each_code<DTYPE, kTopkThreads>(row_ptr, c_lo, c_hi, a.vector, [&](uint32_t col, uint32_t code) {
             if (code >= floor_code) {
                 const unsigned pos = atomicAdd(&sh_count, 1u);
                 if (pos < kCap) sh_cand[pos] = composite(code, col);
             }
         });
         __syncthreads();
-        const unsigned n = sh_count;
+        unsigned n = sh_count;
+        if constexpr (CS > 1) {
+            cg::this_cluster().sync();
+            if (part == 0) {
+                for (unsigned r = 1; r < CS; ++r) {
+                    const unsigned n_r = *cg::this_cluster().map_shared_rank(&sh_count, r);
+                    if (n <= kCap && n_r <= kCap && n + n_r <= kCap) {
+                        const uint64_t *other = cg::this_cluster().map_shared_rank(&sh_cand[0], r);
+                        for (unsigned i = threadIdx.x; i < n_r; i += kTopkThreads) sh_cand[n + i] = other[i];
+                    }
+                    n = (n > kCap || n_r > kCap) ? kCap + 1 : n + n_r;
+                }
+            }
+            cg::this_cluster().sync();               // the other CTAs' shared memory has been read
+            if (part != 0) return;
+            __syncthreads();
+        }
 
         if (n <= kCap) {
             // 3. rank by counting, bias ranks below k
@@ -198,18 +234,39 @@ topk_kernel(const TopkArgs a) {
             const uint32_t rounds = k < V ? k : V;
             for (uint32_t r = 0; r < rounds; ++r) {
                 uint64_t best = 0;
-                for_each_code<DTYPE, kTopkThreads>(row_ptr, V, a.vector, [&](uint32_t col, uint32_t code) {
+                for_each_code<DTYPE, kTopkThreads>(row_ptr, 0u, V, a.vector, [&](uint32_t col, uint32_t code) {
                     const uint64_t c = composite(code, col);
                     if ((r == 0 || c < prev) && c > best) best = c;
                 });
                 prev = block_max_u64<kTopkWarps>(best, sh_red, &sh_best);
             }
             const uint64_t kth = prev;
-            for_each_code<DTYPE, kTopkThreads>(row_ptr, V, a.vector, [&](uint32_t col, uint32_t code) {
+            for_each_code<DTYPE, kTopkThreads>(row_ptr, 0u, V, a.vector, [&](uint32_t col, uint32_t code) {
                 if (composite(code, col) >= kth) bias_column<DTYPE, SCHEME>(a, row, row_ptr, col);
             });
         }
         __syncthreads();             // shared scratch is reused by the next row
+    }
+}
+
+template <int DTYPE, int SCHEME>
+cudaError_t launch_cluster(const TopkArgs &a, int cs, cudaStream_t s) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(a.B * cs));
+    cfg.blockDim = dim3(512);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(cs);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    switch (cs) {
+        case 8: return cudaLaunchKernelEx(&cfg, topk_kernel<DTYPE, SCHEME, 512, 8>, a);
+        case 4: return cudaLaunchKernelEx(&cfg, topk_kernel<DTYPE, SCHEME, 512, 4>, a);
+        default: return cudaLaunchKernelEx(&cfg, topk_kernel<DTYPE, SCHEME, 512, 2>, a);
     }
 }
 
@@ -220,13 +277,17 @@ int launch(const TopkArgs &a, cudaStream_t s) {
     if (rc != SBW_OK) return rc;
     // more rows than SMs: two 512-thread CTAs per SM keep twice as many rows in flight (that
     // kernel has 128 groups, so its fast path needs k <= 128); otherwise one 1024-thread CTA per row
-    if (a.B > di.sm_count && a.k <= 128) {
-        const int64_t cap = static_cast<int64_t>(di.sm_count) * 2;
+    // small batches: a cluster of 512-thread CTAs per row, as many as keeps two CTAs on every SM
+    const int64_t cap = static_cast<int64_t>(di.sm_count) * 2;
+    const int cs = a.B * 8 <= cap ? 8 : a.B * 4 <= cap ? 4 : a.B * 2 <= cap ? 2 : 1;
+    if (cs > 1 && (a.k + cs - 1) / cs <= 128 && a.V >= 4096) {
+        SBW_CUDA_TRY((launch_cluster<DTYPE, SCHEME>(a, cs, s)));
+    } else if (a.B > di.sm_count && a.k <= 128) {
         const unsigned grid = static_cast<unsigned>(a.B < cap ? a.B : cap);
-        topk_kernel<DTYPE, SCHEME, 512><<<grid, 512, 0, s>>>(a);
+        topk_kernel<DTYPE, SCHEME, 512, 1><<<grid, 512, 0, s>>>(a);
     } else {
         const unsigned grid = static_cast<unsigned>(a.B < di.sm_count ? a.B : di.sm_count);
-        topk_kernel<DTYPE, SCHEME, 1024><<<grid, 1024, 0, s>>>(a);
+        topk_kernel<DTYPE, SCHEME, 1024, 1><<<grid, 1024, 0, s>>>(a);
     }
     SBW_CUDA_TRY(cudaGetLastError());
     return SBW_OK;

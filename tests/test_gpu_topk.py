@@ -102,3 +102,16 @@ def test_batches_larger_than_the_sm_count(dtype, k):
     x[7, 1000:] = float("-inf")
     ctx = inputs.uniform_tokens((B, 4), V, seed=82)
     _check(x, V, ctx, KEY, 0.25, 2.0, sbw.SCHEME_SELFSALT, k)
+
+
+@pytest.mark.parametrize("B", [1, 37, 38, 74, 75, 148, 149])
+def test_every_cluster_size(B):
+    """Small batches give a row to a cluster of 8, 4 or 2 CTAs; ties, flat rows and a ragged tail included."""
+    V = 20011
+    x = inputs.logits_normal(B, V, 4.0, torch.float32, seed=90 + B)
+    x[0, :] = 1.25
+    if B > 2:
+        x[2, 5000:15000] = 9.0
+    ctx = inputs.uniform_tokens((B, 1), V, seed=91)
+    _check(x, V, ctx, KEY, 0.25, 2.0, sbw.SCHEME_SELFSALT, 40)
+    _check(x.to(torch.bfloat16), V, ctx, KEY, 0.25, 2.0, sbw.SCHEME_CONTEXT, 128)
