@@ -42,7 +42,7 @@ namespace {
 constexpr int kSampleThreads = 256;
 constexpr int kSampleWarps = kSampleThreads / 32;
 constexpr int kMaxSplit = 512;         // chunks per row at most
-constexpr int kMinSlotsPerItem = 64;   // two trips of a warp at least
+constexpr int kMinSlotsPerItem = 32;   // one full trip of a warp at least
 constexpr int kMaxExtraParts = 40960;  // partials beyond one per row never needed: ~16 waves of warps
 
 struct __align__(32) Partial {
