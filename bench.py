@@ -444,6 +444,24 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
             s = _time_calls(lambda i: sbw.sbw_bias_sample(x, c, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, wsb), 20)
             out[f"sample_bf16_{name}_B{B}"] = {"gelem_s": B * V2 / s / 1e9, "ms": s * 1e3,
                                                "l2_resident": B * V2 * 2 < 100e6}
+    # Appendix F's sampling setting (temperature 0.7, top_p 0.8) and a top-k one, through the truncated sampler
+    for B in (64, 1024):
+        x = inputs.logits_normal(B, V2, 4.0, torch.bfloat16, seed=600 + B, device=dev)
+        c = inputs.uniform_tokens((B, 1), V2, seed=700 + B, device=dev)
+        ids = torch.empty(B, dtype=torch.int32, device=dev)
+        wsf = torch.empty(sbw.sbw_sample_filtered_workspace_bytes(torch.bfloat16, B, V2), dtype=torch.uint8,
+                          device=dev)
+        for name, top_k, top_p in (("top_p0.8", 0, 0.8), ("top_k50", 50, 1.0)):
+            s = _time_calls(lambda i: sbw.sbw_bias_sample_filtered(x, c, KEY, 0.25, 2.0, sbw.SCHEME_CONTEXT, 0.7,
+                                                                   top_k, top_p, 0xC4, i, ids, wsf), 20)
+            out[f"sample_filtered_bf16_context_{name}_B{B}"] = {"gelem_s": B * V2 / s / 1e9, "ms": s * 1e3}
+    # SBW-ss (self-salt on the top-40 candidates) at the headline shape
+    xs = [inputs.logits_normal(B2, V2, 4.0, torch.bfloat16, seed=650 + i, device=dev) for i in range(16)]
+    cs = [inputs.uniform_tokens((B2, 1), V2, seed=750 + i, device=dev) for i in range(16)]
+    s = _time_calls(lambda i: sbw.sbw_bias_logits_topk(xs[i % 16], cs[i % 16], KEY, 0.25, 2.0, sbw.SCHEME_SELFSALT, 40),
+                    256)
+    out["topk40_bf16_selfsalt_B64_V128256"] = {"gelem_s": B2 * V2 / s / 1e9, "ms": s * 1e3}
+    del xs, cs
     # the paper's isolated-benchmark protocol (Appendix B: fresh (B, 151936) logits, 20 warm-up + 200
     # timed calls, CUDA events, synchronise between calls, p50/p99) on its two full-vocabulary schemes
     # with context width 4 (SBW-4, SBW-ss-V); fp32 logits (the paper does not state its dtype)
