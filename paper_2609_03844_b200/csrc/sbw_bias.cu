@@ -39,6 +39,8 @@ struct BiasArgs {
     float delta;            // fp32 path: delta; bf16 path: delta rounded to bf16, widened
     uint32_t delta_bf16;    // bf16 bits of delta
     Weyl weyl;              // Philox key-schedule increments (see sbw_hash.cuh)
+    const void *src;        // out-of-place variant only: rows are read here and written to `logits`
+    int64_t ld_src;
 };
 
 __device__ __forceinline__ uint32_t add_bf16x2(uint32_t a, uint32_t b) {
@@ -133,7 +135,9 @@ __device__ __forceinline__ void green4x2(const BiasArgs &a, const RowSeed<SCHEME
     for (int i = 0; i < 8; ++i) g[i] = x[i] <= a.thr_m1;
 }
 
-template <int DTYPE, int SCHEME, bool VECTOR>
+// COPY = true is the out-of-place variant used by the truncated sampler: the same pass, reading the
+// rows from a.src (16-byte aligned rows) and writing the biased rows to a.logits.
+template <int DTYPE, int SCHEME, bool VECTOR, bool COPY = false>
 __global__ void __launch_bounds__(kBiasThreads, 2)
 bias_kernel(const BiasArgs a) {
     constexpr int VEC = VECTOR ? (DTYPE == SBW_DTYPE_F32 ? 4 : 8) : 1;
@@ -163,10 +167,13 @@ bias_kernel(const BiasArgs a) {
         } else {
             const uint32_t jf_end = min(j_end, nfull);
             uint4 *slots = reinterpret_cast<uint4 *>(row_ptr);
+            const uint4 *in = slots;
+            if constexpr (COPY)
+                in = reinterpret_cast<const uint4 *>(static_cast<const char *>(a.src) + row * a.ld_src * ESIZE);
             if constexpr (DTYPE == SBW_DTYPE_BF16) {
                 const uint32_t dlo = a.delta_bf16, dhi = a.delta_bf16 << 16;
                 for (uint32_t j = col + threadIdx.x; j < jf_end; j += kBiasThreads) {
-                    uint4 w = slots[j];
+                    uint4 w = in[j];
                     bool g[8];
                     green8<SCHEME>(a, rs, a.vocab_offset + j * 8, g);
                     // adding -0.0 returns the other operand unchanged, so a packed add with
@@ -184,8 +191,8 @@ bias_kernel(const BiasArgs a) {
                 for (uint32_t j = col + threadIdx.x; j < jf_end; j += 2 * kBiasThreads) {
                     const uint32_t j2 = j + kBiasThreads;
                     const bool two = j2 < jf_end;
-                    uint4 w0 = slots[j];
-                    uint4 w1 = two ? slots[j2] : make_uint4(0, 0, 0, 0);
+                    uint4 w0 = in[j];
+                    uint4 w1 = two ? in[j2] : make_uint4(0, 0, 0, 0);
                     bool g[8];
                     green4x2<SCHEME>(a, rs, a.vocab_offset + j * 4, a.vocab_offset + j2 * 4, g);
                     uint32_t *e0 = reinterpret_cast<uint32_t *>(&w0);
@@ -202,8 +209,13 @@ bias_kernel(const BiasArgs a) {
                 }
             }
             // ragged last slot of the row, if this block owns it
-            if (nfull < nslot && j_end == nslot && threadIdx.x == 0)
+            if (nfull < nslot && j_end == nslot && threadIdx.x == 0) {
+                if constexpr (COPY) {
+                    const char *tail = reinterpret_cast<const char *>(in);
+                    for (uint32_t b = nfull * VEC * ESIZE; b < V * ESIZE; ++b) row_ptr[b] = tail[b];
+                }
                 bias_scalar<DTYPE, SCHEME>(a, rs, row_ptr, nfull * VEC, V, 1);
+            }
         }
         left -= seg;
         ++row;
@@ -211,7 +223,7 @@ bias_kernel(const BiasArgs a) {
     }
 }
 
-template <int DTYPE, int SCHEME, bool VECTOR>
+template <int DTYPE, int SCHEME, bool VECTOR, bool COPY = false>
 int launch(const BiasArgs &a, cudaStream_t stream) {
     DeviceInfo di;
     int rc = current_device_info(&di);
@@ -219,14 +231,14 @@ int launch(const BiasArgs &a, cudaStream_t stream) {
     static std::atomic<int> blocks_per_sm{0};  // a property of the compiled kernel, equal on every sm_100a device
     if (blocks_per_sm == 0) {
         int n = 0;
-        SBW_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, bias_kernel<DTYPE, SCHEME, VECTOR>,
+        SBW_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, bias_kernel<DTYPE, SCHEME, VECTOR, COPY>,
                                                                    kBiasThreads, 0));
         blocks_per_sm = n > 0 ? n : 1;
     }
     const int64_t want = (a.total + kBiasThreads - 1) / kBiasThreads;
     const int64_t cap = static_cast<int64_t>(di.sm_count) * blocks_per_sm;
     const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
-    SBW_CUDA_TRY(launch_pdl(bias_kernel<DTYPE, SCHEME, VECTOR>, dim3(grid), dim3(kBiasThreads), stream, a));
+    SBW_CUDA_TRY(launch_pdl(bias_kernel<DTYPE, SCHEME, VECTOR, COPY>, dim3(grid), dim3(kBiasThreads), stream, a));
     return SBW_OK;
 }
 
@@ -237,9 +249,14 @@ int launch_v(const BiasArgs &a, bool vector, cudaStream_t stream) {
 
 }  // namespace
 
-int bias_logits_impl(void *logits, int dtype, int64_t B, int64_t V, int64_t ld, int64_t vocab_offset,
-                     const int32_t *ctx_tokens, int ctx_width, uint64_t key, double gamma, float delta,
-                     int scheme, cudaStream_t stream) {
+// Checks and argument set-up shared by the in-place and the out-of-place entry.  Returns SBW_OK
+// with *run = false when there is nothing to do (empty batch, or a bias that is zero in the
+// logits' precision: the paper's delta = 0 control, which leaves every bit alone -- an IEEE add of
+// +0 would turn -0 into +0).
+static int prepare(BiasArgs &a, void *logits, int dtype, int64_t B, int64_t V, int64_t ld, int64_t vocab_offset,
+                   const int32_t *ctx_tokens, int ctx_width, uint64_t key, double gamma, float delta, int scheme,
+                   bool *run) {
+    *run = false;
     if (!valid_common(dtype, ctx_width, gamma, scheme)) return SBW_ERR_INVALID_ARG;
     if (B < 0 || V <= 0 || ld < V || vocab_offset < 0) return SBW_ERR_INVALID_ARG;
     if (V > 0x7fffffffLL || B > (int64_t(1) << 40)) return SBW_ERR_UNSUPPORTED;
@@ -247,8 +264,6 @@ int bias_logits_impl(void *logits, int dtype, int64_t B, int64_t V, int64_t ld, 
     if (!(delta == delta) || delta - delta != 0.0f) return SBW_ERR_INVALID_ARG;  // NaN or inf
     if (B == 0) return SBW_OK;
     if (!logits || !ctx_tokens) return SBW_ERR_INVALID_ARG;
-
-    BiasArgs a;
     a.logits = logits;
     a.B = B; a.V = V; a.ld = ld;
     a.ctx = ctx_tokens;
@@ -259,16 +274,27 @@ int bias_logits_impl(void *logits, int dtype, int64_t B, int64_t V, int64_t ld, 
     a.delta = delta;
     a.delta_bf16 = 0;
     a.weyl = make_weyl();
-    const int esize = dtype == SBW_DTYPE_F32 ? 4 : 2;
+    a.src = nullptr;
+    a.ld_src = 0;
     if (dtype == SBW_DTYPE_BF16) {
         const __nv_bfloat16 d = __float2bfloat16_rn(delta);
         a.delta_bf16 = static_cast<uint32_t>(__bfloat16_as_ushort(d));
         a.delta = __bfloat162float(d);
     }
-    // A bias that is zero in the logits' precision is the paper's delta = 0 control: the logits
-    // are left alone bit for bit (an IEEE add of +0 would turn -0 into +0).
-    if (a.delta == 0.0f) return SBW_OK;
+    *run = a.delta != 0.0f;
+    return SBW_OK;
+}
 
+int bias_logits_impl(void *logits, int dtype, int64_t B, int64_t V, int64_t ld, int64_t vocab_offset,
+                     const int32_t *ctx_tokens, int ctx_width, uint64_t key, double gamma, float delta,
+                     int scheme, cudaStream_t stream) {
+    BiasArgs a;
+    bool run;
+    if (int rc = prepare(a, logits, dtype, B, V, ld, vocab_offset, ctx_tokens, ctx_width, key, gamma, delta, scheme,
+                         &run))
+        return rc;
+    if (!run) return SBW_OK;
+    const int esize = dtype == SBW_DTYPE_F32 ? 4 : 2;
     const bool vector = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && ((ld * esize) % 16 == 0);
     const int vec = vector ? 16 / esize : 1;
     a.nslot = (V + vec - 1) / vec;
@@ -282,6 +308,37 @@ int bias_logits_impl(void *logits, int dtype, int64_t B, int64_t V, int64_t ld, 
     return scheme == SBW_SCHEME_CONTEXT
                ? launch_v<SBW_DTYPE_BF16, SBW_SCHEME_CONTEXT>(a, vector, stream)
                : launch_v<SBW_DTYPE_BF16, SBW_SCHEME_SELFSALT>(a, vector, stream);
+}
+
+// Out-of-place bias: dst[b, j] = bias(src[b, j]) for j < V in one pass.  *done = false (and nothing
+// launched) when the rows of src or dst are not 16-byte aligned or the bias is zero in the logits'
+// precision; the caller then copies the rows itself and biases them in place.
+int bias_copy_impl(const void *src, int64_t ld_src, void *dst, int dtype, int64_t B, int64_t V, int64_t ld,
+                   int64_t vocab_offset, const int32_t *ctx_tokens, int ctx_width, uint64_t key, double gamma,
+                   float delta, int scheme, cudaStream_t stream, bool *done) {
+    *done = false;
+    BiasArgs a;
+    bool run;
+    if (int rc = prepare(a, dst, dtype, B, V, ld, vocab_offset, ctx_tokens, ctx_width, key, gamma, delta, scheme,
+                         &run))
+        return rc;
+    if (!src || ld_src < V) return SBW_ERR_INVALID_ARG;
+    const int esize = dtype == SBW_DTYPE_F32 ? 4 : 2;
+    const bool aligned = reinterpret_cast<uintptr_t>(dst) % 16 == 0 && (ld * esize) % 16 == 0 &&
+                         reinterpret_cast<uintptr_t>(src) % 16 == 0 && (ld_src * esize) % 16 == 0;
+    if (!run || !aligned) return SBW_OK;
+    a.src = src;
+    a.ld_src = ld_src;
+    const int vec = 16 / esize;
+    a.nslot = (V + vec - 1) / vec;
+    a.total = B * a.nslot;
+    *done = true;
+    if (dtype == SBW_DTYPE_F32) {
+        return scheme == SBW_SCHEME_CONTEXT ? launch<SBW_DTYPE_F32, SBW_SCHEME_CONTEXT, true, true>(a, stream)
+                                            : launch<SBW_DTYPE_F32, SBW_SCHEME_SELFSALT, true, true>(a, stream);
+    }
+    return scheme == SBW_SCHEME_CONTEXT ? launch<SBW_DTYPE_BF16, SBW_SCHEME_CONTEXT, true, true>(a, stream)
+                                        : launch<SBW_DTYPE_BF16, SBW_SCHEME_SELFSALT, true, true>(a, stream);
 }
 
 }  // namespace sbw

@@ -1,9 +1,9 @@
 // sbw_bias_sample_filtered: bias (Eq. 2 of the paper) + top-k / top-p truncation + Gumbel-max
 // sampling (the paper's Appendix F samples with temperature 0.7 and top_p = 0.8).
 //
-// The biased logits l' are produced once -- the row is copied into the workspace and biased
-// there by the full-vocabulary bias kernel -- and everything after that is memory traffic over
-// that copy, one CTA per row:
+// The biased logits l' are produced once -- the full-vocabulary bias kernel writes a biased copy
+// of the rows into the workspace -- and everything after that is memory traffic over that copy,
+// one CTA (or one cluster of CTAs) per row:
 //   order    candidates are ranked by order-encoded bits, ties by column; with key_m the code of
 //            the row maximum, a candidate is the 64-bit composite (key_m - code) << 32 | column,
 //            and "kept" is always "composite <= boundary".
@@ -31,6 +31,9 @@ namespace sbw {
 int bias_logits_impl(void *logits, int dtype, int64_t B, int64_t V, int64_t ld, int64_t vocab_offset,
                      const int32_t *ctx_tokens, int ctx_width, uint64_t key, double gamma, float delta,
                      int scheme, cudaStream_t stream);
+int bias_copy_impl(const void *src, int64_t ld_src, void *dst, int dtype, int64_t B, int64_t V, int64_t ld,
+                   int64_t vocab_offset, const int32_t *ctx_tokens, int ctx_width, uint64_t key, double gamma,
+                   float delta, int scheme, cudaStream_t stream, bool *done);
 
 namespace {
 
@@ -649,11 +652,18 @@ extern "C" int sbw_bias_sample_filtered(const void *logits, int dtype, int64_t B
     const size_t es = dtype == SBW_DTYPE_F32 ? 4 : 2;
     const int64_t vp = static_cast<int64_t>(align_up(static_cast<size_t>(V), 8));
 
-    // l' of Eq. 2, in the logits' precision, into the workspace
-    SBW_CUDA_TRY(cudaMemcpy2DAsync(workspace, vp * es, logits, ld * es, V * es, B, cudaMemcpyDeviceToDevice, s));
-    if (int rc = bias_logits_impl(workspace, dtype, B, V, vp, vocab_offset, ctx_tokens, ctx_width, key, gamma,
-                                  delta, scheme, s))
+    // l' of Eq. 2, in the logits' precision, into the workspace: one out-of-place pass of the bias
+    // kernel when the rows are 16-byte aligned, else a row copy and the in-place kernel
+    bool fused = false;
+    if (int rc = bias_copy_impl(logits, ld, workspace, dtype, B, V, vp, vocab_offset, ctx_tokens, ctx_width, key,
+                                gamma, delta, scheme, s, &fused))
         return rc;
+    if (!fused) {
+        SBW_CUDA_TRY(cudaMemcpy2DAsync(workspace, vp * es, logits, ld * es, V * es, B, cudaMemcpyDeviceToDevice, s));
+        if (int rc = bias_logits_impl(workspace, dtype, B, V, vp, vocab_offset, ctx_tokens, ctx_width, key, gamma,
+                                      delta, scheme, s))
+            return rc;
+    }
 
     FilterArgs a;
     a.biased = workspace;
