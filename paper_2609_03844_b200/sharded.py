@@ -53,3 +53,40 @@ def sharded_bias_sample(logits_shard: torch.Tensor, ctx_tokens: torch.Tensor, ke
     p = torch.empty(B, dtype=torch.float32, device=dev)
     binding.sbw_sample_combine(shards, temperature, tokens, out_max=m, out_sumexp=Z, out_prob=p)
     return tokens, m, Z, p
+
+
+def shard_sequences(N: int, rank: int, world: int) -> tuple[int, int]:
+    """Sequences [lo, hi) of a batch of N owned by ``rank``: contiguous and balanced.  Detection has
+    no cross-sequence dependency, so this is all the sharding it needs."""
+    base, rem = divmod(N, world)
+    lo = rank * base + min(rank, rem)
+    return lo, lo + base + (1 if rank < rem else 0)
+
+
+def gather_ragged(local: torch.Tensor, group=None) -> torch.Tensor:
+    """Concatenation, in rank order, of 1-D tensors whose lengths differ between ranks (two
+    collectives: the lengths, then the padded payloads)."""
+    world = dist.get_world_size(group) if dist.is_initialized() else 1
+    if world == 1:
+        return local.contiguous()
+    n = torch.tensor([local.numel()], dtype=torch.int64, device=local.device)
+    sizes = [torch.zeros_like(n) for _ in range(world)]
+    dist.all_gather(sizes, n, group=group)
+    sizes = [int(s.item()) for s in sizes]
+    width = max(sizes)
+    padded = torch.zeros(width, dtype=local.dtype, device=local.device)
+    padded[:local.numel()] = local
+    parts = [torch.empty_like(padded) for _ in range(world)]
+    dist.all_gather(parts, padded, group=group)
+    return torch.cat([p[:s] for p, s in zip(parts, sizes)])
+
+
+def sharded_roc_auc(z_local: torch.Tensor, labels_local: torch.Tensor, group=None) -> torch.Tensor:
+    """ROC-AUC over the z-scores of all ranks (each rank detected its own sequences): 9 bytes per
+    sequence are all-gathered, then every rank counts the pairs itself.  Returns float64[1]."""
+    z = gather_ragged(z_local, group)
+    labels = gather_ragged(labels_local, group)
+    auc = torch.empty(1, dtype=torch.float64, device=z.device)
+    ws = torch.empty(max(binding.sbw_roc_auc_workspace_bytes(z.numel()), 256), dtype=torch.uint8, device=z.device)
+    binding.sbw_roc_auc(z, labels, auc, ws)
+    return auc

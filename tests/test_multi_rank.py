@@ -135,3 +135,48 @@ def test_shard_columns_partition_is_aligned_and_complete():
             assert parts[0][0] == 0 and parts[-1][1] == V
             assert all(parts[i][1] == parts[i + 1][0] for i in range(world - 1))
             assert all(lo % 8 == 0 or lo == V for lo, _ in parts)
+
+
+def _roc_worker(rank: int, world: int, port: int, out_dir: str):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank),
+                      WORLD_SIZE=str(world), LOCAL_RANK=str(rank))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import oracle
+    from paper_2609_03844_b200 import inputs, sharded
+
+    N = 13                                                      # odd: the ranks hold different numbers
+    tokens, lengths = inputs.null_token_streams(N, 5, 60, 500, seed=11)
+    lo, hi = sharded.shard_sequences(N, rank, world)
+    off = np.concatenate([[0], np.cumsum(lengths.numpy())])
+    _, _, z = oracle.detect(tokens.numpy()[off[lo]:off[hi]], lengths.numpy()[lo:hi], 0x5EED, 0.25, 1)
+    labels = (np.arange(lo, hi) % 3 == 0).astype(np.uint8)
+    all_z = sharded.gather_ragged(torch.from_numpy(z))
+    all_l = sharded.gather_ragged(torch.from_numpy(labels))
+    assert all_z.numel() == N and all_l.numel() == N
+    np.savez(os.path.join(out_dir, f"roc{rank}.npz"), z=all_z.numpy(), l=all_l.numpy())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_gather_scores_for_roc_auc(tmp_path):
+    """Sequence-sharded detection, host side: ranks hold different numbers of z-scores, the ragged
+    all-gather restores the batch order on every rank, and the AUC of the gathered scores is the
+    AUC of the unsharded batch."""
+    world = 2
+    mp.spawn(_roc_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    import oracle
+    from paper_2609_03844_b200 import inputs, sharded
+
+    r0, r1 = np.load(tmp_path / "roc0.npz"), np.load(tmp_path / "roc1.npz")
+    assert np.array_equal(r0["z"], r1["z"]) and np.array_equal(r0["l"], r1["l"])
+    tokens, lengths = inputs.null_token_streams(13, 5, 60, 500, seed=11)
+    _, _, z = oracle.detect(tokens.numpy(), lengths.numpy(), 0x5EED, 0.25, 1)
+    labels = (np.arange(13) % 3 == 0).astype(np.uint8)
+    assert np.array_equal(r0["z"], z) and np.array_equal(r0["l"], labels)
+    assert oracle.roc_auc(r0["z"], r0["l"])[0] == oracle.roc_auc(z, labels)[0]
+    for N in (0, 1, 13, 100):
+        for w in (1, 2, 3, 8):
+            parts = [sharded.shard_sequences(N, r, w) for r in range(w)]
+            assert parts[0][0] == 0 and parts[-1][1] == N
+            assert all(a[1] == b[0] for a, b in zip(parts, parts[1:]))
+            assert max(b - a for a, b in parts) - min(b - a for a, b in parts) <= 1
