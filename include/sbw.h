@@ -311,6 +311,18 @@ int sbw_roc_auc(const double *z, const uint8_t *labels, int64_t n, double *out_a
                 void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * sbw_roc_auc_batched -- M independent ROC-AUCs in one launch (the paper's Table 4 holds one AUC per
+ * configuration, each over 500 watermarked and 500 unmarked texts).  Problem i is the scores and
+ * labels [offsets[i], offsets[i + 1]) of the flat arrays; each result is what sbw_roc_auc gives on
+ * that slice.  One CTA per problem: meant for many problems of up to a few ten thousand scores.
+ *   z, labels   device, flat;  offsets  device int64[M + 1], non-decreasing.
+ *   out_auc     device double[M];  out_stats  device uint64[4 M] or NULL.
+ * Needs no workspace.
+ */
+int sbw_roc_auc_batched(const double *z, const uint8_t *labels, const int64_t *offsets, int64_t M,
+                        double *out_auc, uint64_t *out_stats, void *stream);
+
+/*
  * sbw_bias_sample_filtered -- sbw_bias_sample on the top-k / top-p truncated distribution (the
  * paper's Appendix F samples with temperature 0.7 and top_p = 0.8; the paper gives no arithmetic
  * for the truncation, the one below is this library's).  Per row, with l' the biased logits of Eq. 2:

@@ -32,7 +32,7 @@ EXPORTS = ("sbw_version", "sbw_last_cuda_error", "sbw_bias_logits",
            "sbw_bias_sample_shard", "sbw_sample_combine", "sbw_detect_bits_words", "sbw_detect_bits",
            "sbw_window_z", "sbw_prefix_z", "sbw_detect_unique_workspace_bytes", "sbw_detect_unique",
            "sbw_roc_auc_workspace_bytes", "sbw_roc_auc", "sbw_sample_filtered_workspace_bytes",
-           "sbw_bias_sample_filtered")
+           "sbw_bias_sample_filtered", "sbw_roc_auc_batched")
 
 _lib = None
 
@@ -115,6 +115,8 @@ def lib() -> ctypes.CDLL:
         L.sbw_roc_auc_workspace_bytes.argtypes = [i64]
         L.sbw_roc_auc.restype = i32
         L.sbw_roc_auc.argtypes = [vp, vp, i64, vp, vp, vp, sz, vp]
+        L.sbw_roc_auc_batched.restype = i32
+        L.sbw_roc_auc_batched.argtypes = [vp, vp, vp, i64, vp, vp, vp]
         L.sbw_sample_filtered_workspace_bytes.restype = sz
         L.sbw_sample_filtered_workspace_bytes.argtypes = [i32, i64, i64]
         L.sbw_bias_sample_filtered.restype = i32
@@ -444,6 +446,22 @@ def sbw_roc_auc(z: torch.Tensor, labels: torch.Tensor, out_auc: torch.Tensor, wo
     rc = lib().sbw_roc_auc(_ptr(z), _ptr(labels), z.numel(), _ptr(out_auc), _ptr(out_stats), _ptr(workspace),
                            workspace.numel() * workspace.element_size(), _stream(stream))
     _check("sbw_roc_auc", rc)
+    return out_auc
+
+
+def sbw_roc_auc_batched(z: torch.Tensor, labels: torch.Tensor, offsets: torch.Tensor, out_auc: torch.Tensor, *,
+                        out_stats: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """One ROC-AUC per slice ``[offsets[i], offsets[i + 1])`` of the flat scores and labels."""
+    M = offsets.numel() - 1
+    if z.dtype != torch.float64 or labels.dtype != torch.uint8 or offsets.dtype != torch.int64:
+        raise TypeError("z must be float64, labels uint8, offsets int64")
+    if out_auc.dtype != torch.float64 or out_auc.numel() < M:
+        raise TypeError("out_auc must be float64 with one entry per problem")
+    if out_stats is not None and (out_stats.dtype != torch.int64 or out_stats.numel() < 4 * M):
+        raise TypeError("out_stats must be int64 with four entries per problem")
+    rc = lib().sbw_roc_auc_batched(_ptr(z), _ptr(labels), _ptr(offsets), M, _ptr(out_auc), _ptr(out_stats),
+                                   _stream(stream))
+    _check("sbw_roc_auc_batched", rc)
     return out_auc
 
 

@@ -171,6 +171,108 @@ pairs_kernel(const double *pos, const double *neg, RocCounters *c, double *out_a
     }
 }
 
+
+// Many independent problems at once (the paper's tables hold one AUC per configuration, each over
+// a few hundred texts): one CTA per problem, no workspace.  The problem's scores are walked in
+// windows of kRocNegTile; the negatives of a window are compacted into shared memory (their order
+// does not matter), padded with +inf and sorted, and every positive of the whole problem is then
+// searched in them as in pairs_kernel.
+__global__ void __launch_bounds__(kRocSortThreads)
+batched_kernel(const double *z, const uint8_t *labels, const int64_t *offsets, int64_t M, double *out_auc,
+               uint64_t *out_stats) {
+    __shared__ double s[kRocNegTile];
+    __shared__ unsigned long long red[3][kRocSortThreads / 32];
+    __shared__ unsigned int s_count;
+    const double inf = __longlong_as_double(0x7ff0000000000000LL);
+    const double nan = __longlong_as_double(0x7ff8000000000000LL);
+    for (int64_t prob = blockIdx.x; prob < M; prob += gridDim.x) {
+        const int64_t lo = offsets[prob], hi = offsets[prob + 1];
+        const int64_t n = hi > lo ? hi - lo : 0;
+        const double *zp = z + lo;
+        const uint8_t *lp = labels + lo;
+        unsigned long long greater = 0, equal = 0, n_pos = 0, n_neg = 0;
+        for (int64_t w0 = 0; w0 < n; w0 += kRocNegTile) {
+            if (threadIdx.x == 0) s_count = 0u;
+            __syncthreads();
+            for (int j = threadIdx.x; j < kRocNegTile; j += kRocSortThreads) {
+                const int64_t i = w0 + j;
+                if (i < n) {
+                    const double v = zp[i];
+                    if (v == v && !lp[i]) s[atomicAdd(&s_count, 1u)] = v;
+                }
+            }
+            __syncthreads();
+            const unsigned m = s_count;
+            for (int j = m + threadIdx.x; j < kRocNegTile; j += kRocSortThreads) s[j] = inf;
+            __syncthreads();
+            for (int k = 2; k <= kRocNegTile; k <<= 1) {
+                for (int j = k >> 1; j > 0; j >>= 1) {
+                    const int t = threadIdx.x;
+                    const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+                    const double a = s[i], b = s[i + j];
+                    if ((a > b) == ((i & k) == 0)) {
+                        s[i] = b;
+                        s[i + j] = a;
+                    }
+                    __syncthreads();
+                }
+            }
+            if (threadIdx.x == 0) n_neg += m;
+            if (m > 0) {
+                for (int64_t i = threadIdx.x; i < n; i += kRocSortThreads) {
+                    const double p = lp[i] ? zp[i] : nan;          // NaN compares false: counts nothing
+                    unsigned lt = 0, le = 0;
+#pragma unroll
+                    for (int step = kRocNegTile / 2; step > 0; step >>= 1) {
+                        if (s[lt + step - 1] < p) lt += step;
+                        if (s[le + step - 1] <= p) le += step;
+                    }
+                    if (s[lt] < p) lt += 1;
+                    if (s[le] <= p) le += 1;
+                    lt = min(lt, m);
+                    le = min(le, m);
+                    greater += lt;
+                    equal += le - lt;
+                }
+            }
+            __syncthreads();
+        }
+        for (int64_t i = threadIdx.x; i < n; i += kRocSortThreads) {
+            const double v = zp[i];
+            if (v == v && lp[i]) n_pos += 1;
+        }
+        for (int d = 16; d > 0; d >>= 1) {
+            greater += __shfl_down_sync(0xffffffffu, greater, d);
+            equal += __shfl_down_sync(0xffffffffu, equal, d);
+            n_pos += __shfl_down_sync(0xffffffffu, n_pos, d);
+        }
+        if ((threadIdx.x & 31) == 0) {
+            red[0][threadIdx.x >> 5] = greater;
+            red[1][threadIdx.x >> 5] = equal;
+            red[2][threadIdx.x >> 5] = n_pos;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned long long G = 0, E = 0, P = 0;
+            for (int w = 0; w < kRocSortThreads / 32; ++w) {
+                G += red[0][w];
+                E += red[1][w];
+                P += red[2][w];
+            }
+            if (out_stats) {
+                out_stats[4 * prob + 0] = G;
+                out_stats[4 * prob + 1] = E;
+                out_stats[4 * prob + 2] = P;
+                out_stats[4 * prob + 3] = n_neg;
+            }
+            out_auc[prob] = (P == 0 || n_neg == 0)
+                                ? nan
+                                : __ddiv_rn(__ull2double_rn(2ull * G + E), __ull2double_rn(2ull * P * n_neg));
+        }
+        __syncthreads();
+    }
+}
+
 }  // namespace
 }  // namespace sbw
 
@@ -213,6 +315,21 @@ extern "C" int sbw_roc_auc(const double *z, const uint8_t *labels, int64_t n, do
     const int64_t cap = 4LL * di.sm_count;
     const unsigned grid = static_cast<unsigned>(max_items < cap ? max_items : cap);
     pairs_kernel<<<grid, kRocThreads, 0, s>>>(pos, neg, c, out_auc, out_stats);
+    SBW_CUDA_TRY(cudaGetLastError());
+    return SBW_OK;
+}
+
+extern "C" int sbw_roc_auc_batched(const double *z, const uint8_t *labels, const int64_t *offsets, int64_t M,
+                                   double *out_auc, uint64_t *out_stats, void *stream) {
+    using namespace sbw;
+    if (M < 0) return SBW_ERR_INVALID_ARG;
+    if (M == 0) return SBW_OK;
+    if (!offsets || !out_auc || !z || !labels) return SBW_ERR_INVALID_ARG;
+    DeviceInfo di;
+    if (int rc = current_device_info(&di)) return rc;
+    const int64_t cap = 2LL * di.sm_count;
+    batched_kernel<<<static_cast<unsigned>(M < cap ? M : cap), kRocSortThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        z, labels, offsets, M, out_auc, out_stats);
     SBW_CUDA_TRY(cudaGetLastError());
     return SBW_OK;
 }

@@ -194,3 +194,28 @@ def test_auc_of_detector_scores():
     want = oracle.roc_auc(z.cpu().numpy(), y.cpu().numpy())[0]
     assert float(auc.cpu()[0]) == want and want > 0.95
     assert abs(want - oracle.roc_auc(oz, y.cpu().numpy())[0]) < 1e-6
+
+
+def test_batched_auc_equals_one_call_per_slice():
+    """Table-4 shape: one AUC per configuration, 500 + 500 scores each, plus ragged and empty slices."""
+    dev = require_gpu()
+    rng = np.random.default_rng(55)
+    sizes = [1000] * 16 + [0, 1, 2, 2047, 2048, 2049, 5000, 12000]
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    n = int(off[-1])
+    y = (rng.random(n) < 0.5).astype(np.uint8)
+    z = rng.normal(size=n) + 1.1 * y
+    z[::11] = np.round(z[::11])
+    z[::501] = np.nan
+    y[off[20]:off[21]] = 1                                     # a slice with one class only
+    M = len(sizes)
+    auc = torch.full((M,), 7.0, dtype=torch.float64, device=dev)
+    stats = torch.full((4 * M,), -1, dtype=torch.int64, device=dev)
+    sbw.sbw_roc_auc_batched(torch.from_numpy(z).to(dev), torch.from_numpy(y).to(dev), torch.from_numpy(off).to(dev),
+                            auc, out_stats=stats)
+    torch.cuda.synchronize()
+    got, gst = auc.cpu().numpy(), stats.cpu().numpy().astype(np.uint64).reshape(M, 4)
+    for i in range(M):
+        want, wst = oracle.roc_auc(z[off[i]:off[i + 1]], y[off[i]:off[i + 1]], threads=4)
+        assert np.array_equal(gst[i], wst), i
+        assert (np.isnan(got[i]) and np.isnan(want)) or got[i] == want, i
