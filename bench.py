@@ -466,7 +466,7 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
     # timed calls, CUDA events, synchronise between calls, p50/p99) on its two full-vocabulary schemes
     # with context width 4 (SBW-4, SBW-ss-V); fp32 logits (the paper does not state its dtype)
     sweep = {}
-    for B in (1, 16, 64, 256, 512):
+    for B in (1, 2, 4, 8, 16, 32, 64, 128, 256, 512):
         x = inputs.logits_normal(B, 151936, 4.0, torch.float32, seed=800 + B, device=dev)
         c = inputs.uniform_tokens((B, 4), 151936, seed=900 + B, device=dev)
         for name, scheme in (("sbw4", sbw.SCHEME_CONTEXT), ("sbw_ss_v", sbw.SCHEME_SELFSALT)):
