@@ -56,6 +56,17 @@ struct FilterArgs {
     BlockKeys gkeys;       // Philox round keys of the Gumbel stream
     int32_t *out_tokens;
     int32_t *out_kept;     // nullable
+    // candidate path (top_k set): the unbiased rows and what the green test needs; raw = nullptr
+    // means `biased` already holds the biased rows
+    const void *raw;
+    int64_t ld_raw;
+    const int32_t *ctx;
+    int W;
+    int scheme;
+    uint64_t key;
+    uint32_t thr_m1;
+    float delta;           // in the logits' precision, widened
+    Weyl weyl;
 };
 
 // Weights go into the histogram as four 11-bit limbs, each its own array of 32-bit counters:
@@ -411,191 +422,342 @@ __device__ __forceinline__ unsigned long long packed_score(const FilterArgs &a, 
     return (static_cast<unsigned long long>(enc) << 32) | (0xFFFFFFFFu - col);
 }
 
-// One CTA per row (CS = 1), or a cluster of CS CTAs per row for small batches.  The usual case --
-// the kept candidates are a few hundred at most -- needs two passes over the row and no
-// histogram: pass A finds every thread's largest code; the r-th largest of those maxima is a
-// floor that at least r candidates reach; pass B gathers everything at or above the floor into
-// the shared-memory list (and adds up the weights of the whole row); the sorted list is then the
-// head of the row's order, complete down to the floor, and if the top-k cut and the top-p
-// crossing both fall inside it, the sample is drawn from the list.  Otherwise (a deep nucleus,
-// flat or tied rows, a large top_k) the radix descent above finds the boundary and one more pass
-// over the row draws the sample.
-// In a cluster every CTA runs the two passes on its own CS-th of the row; the CTAs exchange their
-// maxima and floors (the smallest of the local floors, each reached by r / CS local candidates,
-// is reached by r candidates of the row), then CTA 0 pulls the other lists and weight sums over
-// distributed shared memory and finishes the row alone.  All CTAs pass the same three cluster
-// barriers whatever the data; nothing spins.
+// ---------------------------------------------------------------------------------------------
+// The head of a row's order, in shared memory.  Two passes over the CTA's part of the row: pass A
+// finds every thread's largest code; the r-th largest of those maxima is a floor that at least r
+// columns reach; pass B gathers every column at or above the floor as (key_m - code) << 32 | column
+// (and, when asked, adds up the weights of the part).  In a cluster (CS > 1) every CTA does this on
+// its own CS-th of the row with ceil(r / CS) in place of r -- the smallest of the local floors is
+// reached by r columns of the row -- the maxima and floors travel through distributed shared
+// memory, and CTA 0 pulls the other lists and weight sums.  All CTAs pass the same three cluster
+// barriers whatever the data; the others then leave (`leave`), CTA 0 finishes the row alone.
+// `slack` > 0 lowers the floor by that much (plus rounding room) in the logits' own units: the
+// caller gathers unbiased logits and wants every column that a bias of at most `slack` could lift
+// to the floor.  More than kListCap columns at or above the floor are reported as kListCap + 1.
+// ---------------------------------------------------------------------------------------------
+struct Head {
+    uint32_t key_m;               // largest code of the row
+    unsigned gathered;            // entries in sh.list (unsorted), or kListCap + 1
+    unsigned long long z_all;     // total weight of the row (want_z)
+    bool leave;
+};
+
 template <int DTYPE, int CS>
-__global__ void __launch_bounds__(kFilterThreads)
-filter_sample_kernel(const FilterArgs a) {
-    constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
-    constexpr int kCodeBits = DTYPE == SBW_DTYPE_F32 ? 32 : 16;
-    constexpr int kPer = kListCap / kFilterThreads;
-    __shared__ FilterShared sh;
+__device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &sh, const char *src_row, unsigned part,
+                                            int want, float slack, bool want_z) {
     namespace cg = cooperative_groups;
     const uint32_t V = static_cast<uint32_t>(a.V);
     const uint32_t nvec = vectors_of<DTYPE>(V);
+    const uint32_t vec_lo = static_cast<uint32_t>(static_cast<uint64_t>(nvec) * part / CS);
+    const uint32_t vec_hi = static_cast<uint32_t>(static_cast<uint64_t>(nvec) * (part + 1) / CS);
+    Head h;
+    h.leave = false;
+    // pass A: per-thread maxima, sorted descending (as ~code ascending) in the list area
+    uint32_t my_max = 0;
+    for_each<DTYPE>(src_row, V, vec_lo, vec_hi, [&](uint32_t, uint32_t code) { my_max = max(my_max, code); });
+    __syncthreads();
+    sh.list[threadIdx.x] = static_cast<unsigned long long>(~my_max);
+    if (threadIdx.x == 0) sh.list_n = 0u;
+    __syncthreads();
+    sort_list(sh, kFilterThreads);
+    uint32_t key_m = ~static_cast<uint32_t>(sh.list[0]);
+    uint32_t floor_code = ~static_cast<uint32_t>(sh.list[(want + CS - 1) / CS - 1]);
+    __syncthreads();
+    if constexpr (CS > 1) {
+        if (threadIdx.x == 0) {
+            sh.part_max = key_m;
+            sh.part_floor = floor_code;
+        }
+        cg::this_cluster().sync();
+        for (unsigned r = 0; r < CS; ++r) {
+            const FilterShared *other = cg::this_cluster().map_shared_rank(&sh, r);
+            key_m = max(key_m, other->part_max);
+            floor_code = min(floor_code, other->part_floor);
+        }
+    }
+    h.key_m = key_m;
+    if (slack > 0.0f) {
+        const float fl = value_of_code<DTYPE>(floor_code);
+        if (fl == fl && fabsf(fl) != __int_as_float(0x7f800000)) {
+            // room for the rounding of the biased sum (it may round up to the floor) and of this
+            // subtraction: a few units in the last place of the logits' type
+            const float eps = DTYPE == SBW_DTYPE_F32 ? 0x1p-20f : 0x1p-5f;
+            const float t = __fsub_rn(__fsub_rn(fl, slack), __fmul_rn(__fadd_rn(fabsf(fl), slack), eps));
+            const uint32_t c = code_of_bits<DTYPE>(__float_as_uint(t));
+            floor_code = min(floor_code, c > 0u ? c - 1u : 0u);
+        } else {
+            floor_code = 0u;                          // no arithmetic on such a floor: gather all, overflow
+        }
+    }
+    const float m = value_of_code<DTYPE>(key_m);
+    // columns with a weight lie within 41 / c of the maximum: code_lo is below all of them
+    uint32_t code_lo = key_m;
+    if (m == m && fabsf(m) != __int_as_float(0x7f800000))
+        code_lo = code_of_bits<DTYPE>(__float_as_uint(__fsub_rn(m, __fdiv_rn(42.0f, a.c))));
+
+    // pass B
+    unsigned long long z_local = 0;
+    for_each<DTYPE>(src_row, V, vec_lo, vec_hi, [&](uint32_t col, uint32_t code) {
+        const uint32_t dist = key_m - code;
+        if (want_z && code >= code_lo) z_local += nucleus_weight(value_of_code<DTYPE>(code), m, dist == 0u, a.c);
+        if (code >= floor_code && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= kListCap) {
+            const unsigned idx = atomicAdd(&sh.list_n, 1u);
+            if (idx < kListCap) sh.list[idx] = (static_cast<unsigned long long>(dist) << 32) | col;
+        }
+    });
+    h.z_all = want_z ? block_sum(z_local, sh) : 0ull;
+    __syncthreads();
+    unsigned gathered = sh.list_n;
+    if constexpr (CS > 1) {
+        if (threadIdx.x == 0) sh.part_z = h.z_all;
+        cg::this_cluster().sync();
+        if (part == 0) {
+            for (unsigned r = 1; r < CS; ++r) {
+                const FilterShared *other = cg::this_cluster().map_shared_rank(&sh, r);
+                const unsigned n_r = other->list_n;
+                if (gathered <= kListCap && n_r <= kListCap && gathered + n_r <= kListCap)
+                    for (unsigned i = threadIdx.x; i < n_r; i += kFilterThreads) sh.list[gathered + i] = other->list[i];
+                gathered = (gathered > kListCap || n_r > kListCap) ? kListCap + 1 : gathered + n_r;
+                h.z_all += other->part_z;
+            }
+        }
+        cg::this_cluster().sync();                   // the other CTAs' shared memory has been read
+        h.leave = part != 0;
+        __syncthreads();
+    }
+    h.gathered = gathered > kListCap ? kListCap + 1 : gathered;
+    return h;
+}
+
+// sh.list[0 .. n) holds composites relative to key_m, unsorted.  Sorts them and applies the
+// top-k cut and the top-p crossing; returns the number of kept candidates (a prefix of the sorted
+// list), or 0 when the list does not reach far enough down the order.
+template <int DTYPE>
+__device__ __forceinline__ int cut_list(const FilterArgs &a, FilterShared &sh, int n, uint32_t key_m, bool use_k,
+                                        bool use_p, unsigned long long z_all) {
+    constexpr int kPer = kListCap / kFilterThreads;
+    const float m = value_of_code<DTYPE>(key_m);
+    int len = 2;
+    while (len < n) len <<= 1;
+    __syncthreads();
+    for (int i = n + threadIdx.x; i < len; i += kFilterThreads) sh.list[i] = kAll;
+    __syncthreads();
+    sort_list(sh, len);
+    int n1 = n;
+    if (use_k) {
+        if (a.top_k > n) return 0;
+        n1 = static_cast<int>(a.top_k);
+    }
+    if (!use_p) return n1;
+    unsigned long long w[kPer], mine = 0;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+        const int idx = threadIdx.x * kPer + i;
+        const uint32_t dist = static_cast<uint32_t>(sh.list[idx < len ? idx : 0] >> 32);
+        w[i] = idx < n1 ? nucleus_weight(value_of_code<DTYPE>(key_m - dist), m, dist == 0u, a.c) : 0ull;
+        mine += w[i];
+    }
+    const unsigned long long in_list = block_sum(mine, sh);
+    const unsigned long long Z = use_k ? in_list : z_all;
+    const unsigned long long lo = a.p32 * Z, hi = __umul64hi(a.p32, Z);
+    unsigned long long target = (hi << 32) | (lo >> 32);
+    if (lo & 0xffffffffull) target += 1;
+    if (threadIdx.x == 0) sh.bcast[0] = kAll;
+    unsigned long long at = block_exclusive_scan(mine, sh);
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+        if (at < target && at + w[i] >= target) sh.bcast[0] = threadIdx.x * kPer + i;
+        at += w[i];
+    }
+    __syncthreads();
+    const unsigned long long cross = sh.bcast[0];
+    __syncthreads();
+    return cross == kAll ? 0 : static_cast<int>(cross) + 1;     // 0: the nucleus reaches below the floor
+}
+
+// Arg max of the packed scores over the CTA and the row's outputs.
+__device__ __forceinline__ void finish_row(const FilterArgs &a, FilterShared &sh, int64_t row, unsigned long long best,
+                                           unsigned long long kept) {
+    for (int d = 16; d > 0; d >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xffffffffu, best, d);
+        best = o > best ? o : best;
+    }
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sh.red[threadIdx.x >> 5] = best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long top = 0;
+        for (int w = 0; w < kFilterWarps; ++w) top = sh.red[w] > top ? sh.red[w] : top;
+        a.out_tokens[row] = static_cast<int32_t>(0xFFFFFFFFu - static_cast<uint32_t>(top));
+    }
+    const unsigned long long total = block_sum(kept, sh);
+    if (threadIdx.x == 0 && a.out_kept) a.out_kept[row] = static_cast<int32_t>(total);
+    __syncthreads();
+}
+
+// Draws the sample from the first n2 entries of the sorted list.
+template <int DTYPE>
+__device__ __forceinline__ void sample_list(const FilterArgs &a, FilterShared &sh, int64_t row, uint32_t key_m, int n2) {
+    unsigned long long best = 0;
+    for (int i = threadIdx.x; i < n2; i += kFilterThreads) {
+        const unsigned long long comp = sh.list[i];
+        const unsigned long long cand = packed_score<DTYPE>(a, static_cast<uint32_t>(row), static_cast<uint32_t>(comp),
+                                                            key_m - static_cast<uint32_t>(comp >> 32));
+        best = cand > best ? cand : best;
+    }
+    finish_row(a, sh, row, best, threadIdx.x == 0 ? n2 : 0);
+}
+
+// The general path on a biased row: list if it reaches far enough, else the radix descent and one
+// more pass over the row.
+template <int DTYPE, int CS>
+__device__ __forceinline__ bool full_row(const FilterArgs &a, FilterShared &sh, int64_t row, unsigned part) {
+    constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
+    constexpr int kCodeBits = DTYPE == SBW_DTYPE_F32 ? 32 : 16;
+    const uint32_t V = static_cast<uint32_t>(a.V);
     const bool use_k = a.top_k > 0 && a.top_k < a.V;
     const bool use_p = a.p32 != 0ull;
+    const char *row_ptr = static_cast<const char *>(a.biased) + row * a.ld * ESIZE;
+    const int want = use_k ? static_cast<int>(min(a.top_k, static_cast<int64_t>(kFilterThreads))) : 384;
+    const Head h = gather_head<DTYPE, CS>(a, sh, row_ptr, part, want, 0.0f, use_p && !use_k);
+    if (h.leave) return false;
+    const uint32_t key_m = h.key_m;
+    int n2 = 0;
+    if ((use_k || use_p) && h.gathered <= kListCap)
+        n2 = cut_list<DTYPE>(a, sh, static_cast<int>(h.gathered), key_m, use_k, use_p, h.z_all);
+    if (n2 > 0) {
+        sample_list<DTYPE>(a, sh, row, key_m, n2);
+        return true;
+    }
+    __syncthreads();
+    const float m = value_of_code<DTYPE>(key_m);
+    unsigned long long boundary = kAll;
+    if (use_k)
+        boundary = select_boundary<DTYPE, kModeCount>(row_ptr, V, key_m, m, a.c, kAll,
+                                                      static_cast<unsigned long long>(a.top_k), kCodeBits, sh);
+    if (use_p) {
+        uint32_t code_lo = key_m;
+        if (m == m && fabsf(m) != __int_as_float(0x7f800000))
+            code_lo = code_of_bits<DTYPE>(__float_as_uint(__fsub_rn(m, __fdiv_rn(42.0f, a.c))));
+        const int s0 = 32 - __clz(key_m - code_lo);
+        boundary = select_boundary<DTYPE, kModeMass>(row_ptr, V, key_m, m, a.c, boundary, a.p32, s0, sh);
+    }
+    unsigned long long best = 0, kept = 0;
+    for_each<DTYPE>(row_ptr, V, [&](uint32_t col, uint32_t code) {
+        const uint32_t dist = key_m - code;
+        if (((static_cast<unsigned long long>(dist) << 32) | col) > boundary) return;
+        kept += 1;
+        const unsigned long long cand = packed_score<DTYPE>(a, static_cast<uint32_t>(row), col, code);
+        best = cand > best ? cand : best;
+    });
+    finish_row(a, sh, row, best, kept);
+    return true;
+}
+
+// Eq. 1 + Eq. 2 on one logit given as its code; returns the code of the biased logit.
+template <int DTYPE>
+__device__ __forceinline__ uint32_t biased_code(const FilterArgs &a, uint64_t r_row, uint32_t jmin, uint32_t col,
+                                                uint32_t code) {
+    const uint32_t v = a.vocab_offset + col;
+    const uint64_t r = a.scheme == SBW_SCHEME_CONTEXT ? r_row : seed_selfsalt(a.key, jmin, v);
+    if (a.delta == 0.0f || philox_word0(v, r, a.weyl) > a.thr_m1) return code;
+    const float l = value_of_code<DTYPE>(code);
+    if constexpr (DTYPE == SBW_DTYPE_F32) {
+        return code_of_bits<DTYPE>(__float_as_uint(__fadd_rn(l, a.delta)));
+    } else {
+        // both operands are bf16 values: rounding their fp32 sum once more is the bf16 sum
+        const __nv_bfloat16 s = __float2bfloat16_rn(__fadd_rn(l, a.delta));
+        return code_of_bits<DTYPE>(static_cast<uint32_t>(__bfloat16_as_ushort(s)) << 16);
+    }
+}
+
+// With top_k set, the kept candidates can be found without biasing the row.  Let f be the k-th
+// largest unbiased logit.  At least k biased logits reach f - max(-delta, 0), so the k-th largest
+// biased logit does too, and a column of the biased top-k, whose biased logit is at most
+// l + max(delta, 0), has l >= f - |delta| (less the rounding of the sum).  Those columns -- a few
+// hundred for ordinary rows -- are gathered from the unbiased row, hashed and biased in shared
+// memory, and then cut and sampled like any list.  A row whose candidates do not fit the list is
+// biased into the workspace by this CTA and takes the general path.
+template <int DTYPE, int CS>
+__device__ __forceinline__ bool candidate_row(const FilterArgs &a, FilterShared &sh, int64_t row, unsigned part) {
+    constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
+    constexpr int VEC = DTYPE == SBW_DTYPE_F32 ? 4 : 8;
+    const uint32_t V = static_cast<uint32_t>(a.V);
+    const bool use_p = a.p32 != 0ull;
+    const char *raw_row = static_cast<const char *>(a.raw) + row * a.ld_raw * ESIZE;
+    const int want = static_cast<int>(min(a.top_k, static_cast<int64_t>(kFilterThreads)));
+    const Head h = gather_head<DTYPE, CS>(a, sh, raw_row, part, want, fmaxf(fabsf(a.delta), 0x1p-126f), false);
+    if (h.leave) return false;
+    const int32_t *ctx = a.ctx + row * a.W;
+    const uint64_t r_row = a.scheme == SBW_SCHEME_CONTEXT ? seed_context(a.key, ctx, a.W) : 0ull;
+    const uint32_t jmin = a.scheme == SBW_SCHEME_SELFSALT ? jenkins_min(ctx, a.W) : 0u;
+    if (h.gathered <= kListCap && static_cast<int64_t>(h.gathered) >= a.top_k) {
+        const int n = static_cast<int>(h.gathered);
+        // bias the candidates: entries become (biased code << 32 | column), then composites
+        // relative to the largest biased code
+        uint32_t top = 0;
+        for (int i = threadIdx.x; i < n; i += kFilterThreads) {
+            const unsigned long long e = sh.list[i];
+            const uint32_t col = static_cast<uint32_t>(e);
+            const uint32_t code = biased_code<DTYPE>(a, r_row, jmin, col, h.key_m - static_cast<uint32_t>(e >> 32));
+            sh.list[i] = (static_cast<unsigned long long>(code) << 32) | col;
+            top = max(top, code);
+        }
+        for (int d = 16; d > 0; d >>= 1) top = max(top, __shfl_xor_sync(0xffffffffu, top, d));
+        __syncthreads();
+        if ((threadIdx.x & 31) == 0) sh.red32[threadIdx.x >> 5] = top;
+        __syncthreads();
+        uint32_t key_m = 0;
+        for (int w = 0; w < kFilterWarps; ++w) key_m = max(key_m, sh.red32[w]);
+        for (int i = threadIdx.x; i < n; i += kFilterThreads) {
+            const unsigned long long e = sh.list[i];
+            sh.list[i] = (static_cast<unsigned long long>(key_m - static_cast<uint32_t>(e >> 32)) << 32) |
+                         static_cast<uint32_t>(e);
+        }
+        const int n2 = cut_list<DTYPE>(a, sh, n, key_m, true, use_p, 0ull);
+        if (n2 > 0) {
+            sample_list<DTYPE>(a, sh, row, key_m, n2);
+            return true;
+        }
+    }
+    // the candidates do not fit: bias the whole row into the workspace, then the general path
+    __syncthreads();
+    char *dst_row = static_cast<char *>(const_cast<void *>(a.biased)) + row * a.ld * ESIZE;
+    const uint32_t nvec = vectors_of<DTYPE>(V);
+    for (uint32_t j = threadIdx.x; j < nvec; j += kFilterThreads) {
+        uint4 w = reinterpret_cast<const uint4 *>(raw_row)[j];
+        uint32_t *e = reinterpret_cast<uint32_t *>(&w);
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+            const uint32_t col = j * VEC + i;
+            if (col >= V) continue;
+            if constexpr (DTYPE == SBW_DTYPE_F32) {
+                e[i] = order_decode(biased_code<DTYPE>(a, r_row, jmin, col, code_of_bits<DTYPE>(e[i])));
+            } else {
+                const uint32_t bits = (i & 1) ? (e[i >> 1] & 0xffff0000u) : (e[i >> 1] << 16);
+                const float v = value_of_code<DTYPE>(biased_code<DTYPE>(a, r_row, jmin, col, code_of_bits<DTYPE>(bits)));
+                const uint32_t b16 = __float_as_uint(v) >> 16;
+                e[i >> 1] = (i & 1) ? ((e[i >> 1] & 0x0000ffffu) | (b16 << 16)) : ((e[i >> 1] & 0xffff0000u) | b16);
+            }
+        }
+        reinterpret_cast<uint4 *>(dst_row)[j] = w;
+    }
+    __syncthreads();
+    return full_row<DTYPE, 1>(a, sh, row, 0u);
+}
+
+// One CTA per row (CS = 1, a persistent grid walking the rows), or a cluster of CS CTAs per row
+// for small batches.
+template <int DTYPE, int CS>
+__global__ void __launch_bounds__(kFilterThreads, 2)   // two CTAs per SM: the paths are latency-bound
+filter_sample_kernel(const FilterArgs a) {
+    __shared__ FilterShared sh;
     const unsigned part = CS > 1 ? blockIdx.x % CS : 0u;          // this CTA's part of the row
     const int64_t first_row = CS > 1 ? blockIdx.x / CS : blockIdx.x;
     const int64_t row_step = CS > 1 ? a.B : gridDim.x;            // a cluster handles exactly one row
     for (int64_t row = first_row; row < a.B; row += row_step) {
-        const char *row_ptr = static_cast<const char *>(a.biased) + row * a.ld * ESIZE;
-        const uint32_t rowb = static_cast<uint32_t>(row);
-        const uint32_t vec_lo = static_cast<uint32_t>(static_cast<uint64_t>(nvec) * part / CS);
-        const uint32_t vec_hi = static_cast<uint32_t>(static_cast<uint64_t>(nvec) * (part + 1) / CS);
-        // pass A: per-thread maxima, sorted descending (as ~code ascending) in the list area
-        uint32_t my_max = 0;
-        for_each<DTYPE>(row_ptr, V, vec_lo, vec_hi, [&](uint32_t, uint32_t code) { my_max = max(my_max, code); });
-        sh.list[threadIdx.x] = static_cast<unsigned long long>(~my_max);
-        if (threadIdx.x == 0) sh.list_n = 0u;
-        __syncthreads();
-        sort_list(sh, kFilterThreads);
-        uint32_t key_m = ~static_cast<uint32_t>(sh.list[0]);
-        const int want = use_k ? static_cast<int>(min(a.top_k, static_cast<int64_t>(kFilterThreads))) : 384;
-        uint32_t floor_code = ~static_cast<uint32_t>(sh.list[(want + CS - 1) / CS - 1]);
-        __syncthreads();
-        if constexpr (CS > 1) {
-            if (threadIdx.x == 0) {
-                sh.part_max = key_m;
-                sh.part_floor = floor_code;
-            }
-            cg::this_cluster().sync();
-            for (unsigned r = 0; r < CS; ++r) {
-                const FilterShared *other = cg::this_cluster().map_shared_rank(&sh, r);
-                key_m = max(key_m, other->part_max);
-                floor_code = min(floor_code, other->part_floor);
-            }
-        }
-        const float m = value_of_code<DTYPE>(key_m);
-
-        // candidates with a weight lie within 41 / c of the maximum: code_lo is below all of them
-        uint32_t code_lo = key_m;
-        if (m == m && fabsf(m) != __int_as_float(0x7f800000))
-            code_lo = code_of_bits<DTYPE>(__float_as_uint(__fsub_rn(m, __fdiv_rn(42.0f, a.c))));
-
-        // pass B: gather the head of the order; total weight of the row when top-p works on all of it
-        unsigned long long z_local = 0;
-        if (use_k || use_p) {
-            for_each<DTYPE>(row_ptr, V, vec_lo, vec_hi, [&](uint32_t col, uint32_t code) {
-                const uint32_t dist = key_m - code;
-                if (use_p && !use_k && code >= code_lo)
-                    z_local += nucleus_weight(value_of_code<DTYPE>(code), m, dist == 0u, a.c);
-                if (code >= floor_code && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= kListCap) {
-                    const unsigned idx = atomicAdd(&sh.list_n, 1u);
-                    if (idx < kListCap) sh.list[idx] = (static_cast<unsigned long long>(dist) << 32) | col;
-                }
-            });
-        }
-        unsigned long long z_all = (use_p && !use_k) ? block_sum(z_local, sh) : 0ull;
-        __syncthreads();
-        unsigned gathered = sh.list_n;
-        if constexpr (CS > 1) {
-            if (threadIdx.x == 0) sh.part_z = z_all;
-            cg::this_cluster().sync();
-            if (part == 0) {
-                // pull the other parts: list entries behind the own ones, weight sums added up
-                for (unsigned r = 1; r < CS; ++r) {
-                    const FilterShared *other = cg::this_cluster().map_shared_rank(&sh, r);
-                    const unsigned n_r = other->list_n;
-                    if (gathered <= kListCap && n_r <= kListCap && gathered + n_r <= kListCap)
-                        for (unsigned i = threadIdx.x; i < n_r; i += kFilterThreads) sh.list[gathered + i] = other->list[i];
-                    gathered = (gathered > kListCap || n_r > kListCap) ? kListCap + 1 : gathered + n_r;
-                    z_all += other->part_z;
-                }
-            }
-            cg::this_cluster().sync();               // the other CTAs' shared memory has been read
-            if (part != 0) return;
-            __syncthreads();
-        }
-        bool resolved = (use_k || use_p) && gathered <= kListCap;
-        int n2 = 0;                                   // candidates kept, a prefix of the sorted list
-        if (resolved) {
-            const int n = static_cast<int>(gathered);
-            int len = 2;
-            while (len < n) len <<= 1;
-            __syncthreads();
-            for (int i = n + threadIdx.x; i < len; i += kFilterThreads) sh.list[i] = kAll;
-            __syncthreads();
-            sort_list(sh, len);
-            int n1 = n;
-            if (use_k) {
-                if (a.top_k <= n) n1 = static_cast<int>(a.top_k);
-                else resolved = false;
-            }
-            n2 = n1;
-            if (resolved && use_p) {
-                unsigned long long w[kPer], mine = 0;
-#pragma unroll
-                for (int i = 0; i < kPer; ++i) {
-                    const int idx = threadIdx.x * kPer + i;
-                    const uint32_t dist = static_cast<uint32_t>(sh.list[idx < len ? idx : 0] >> 32);
-                    w[i] = idx < n1 ? nucleus_weight(value_of_code<DTYPE>(key_m - dist), m, dist == 0u, a.c) : 0ull;
-                    mine += w[i];
-                }
-                const unsigned long long in_list = block_sum(mine, sh);
-                const unsigned long long Z = use_k ? in_list : z_all;
-                const unsigned long long lo = a.p32 * Z, hi = __umul64hi(a.p32, Z);
-                unsigned long long target = (hi << 32) | (lo >> 32);
-                if (lo & 0xffffffffull) target += 1;
-                if (threadIdx.x == 0) sh.bcast[0] = kAll;
-                unsigned long long at = block_exclusive_scan(mine, sh);
-#pragma unroll
-                for (int i = 0; i < kPer; ++i) {
-                    if (at < target && at + w[i] >= target) sh.bcast[0] = threadIdx.x * kPer + i;
-                    at += w[i];
-                }
-                __syncthreads();
-                const unsigned long long cross = sh.bcast[0];
-                __syncthreads();
-                if (cross == kAll) resolved = false;      // the nucleus reaches below the floor
-                else n2 = static_cast<int>(cross) + 1;
-            }
-        }
-
-        unsigned long long best = 0, kept = 0;
-        if (resolved) {
-            for (int i = threadIdx.x; i < n2; i += kFilterThreads) {
-                const unsigned long long comp = sh.list[i];
-                const unsigned long long cand = packed_score<DTYPE>(a, rowb, static_cast<uint32_t>(comp),
-                                                                    key_m - static_cast<uint32_t>(comp >> 32));
-                best = cand > best ? cand : best;
-            }
-            kept = threadIdx.x == 0 ? n2 : 0;
-        } else {
-            __syncthreads();
-            unsigned long long boundary = kAll;
-            if (use_k)
-                boundary = select_boundary<DTYPE, kModeCount>(row_ptr, V, key_m, m, a.c, kAll,
-                                                              static_cast<unsigned long long>(a.top_k), kCodeBits, sh);
-            if (use_p) {
-                const int s0 = 32 - __clz(key_m - code_lo);
-                boundary = select_boundary<DTYPE, kModeMass>(row_ptr, V, key_m, m, a.c, boundary, a.p32, s0, sh);
-            }
-            for_each<DTYPE>(row_ptr, V, [&](uint32_t col, uint32_t code) {
-                const uint32_t dist = key_m - code;
-                if (((static_cast<unsigned long long>(dist) << 32) | col) > boundary) return;
-                kept += 1;
-                const unsigned long long cand = packed_score<DTYPE>(a, rowb, col, code);
-                best = cand > best ? cand : best;
-            });
-        }
-        for (int d = 16; d > 0; d >>= 1) {
-            const unsigned long long o = __shfl_xor_sync(0xffffffffu, best, d);
-            best = o > best ? o : best;
-        }
-        __syncthreads();
-        if ((threadIdx.x & 31) == 0) sh.red[threadIdx.x >> 5] = best;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            unsigned long long top = 0;
-            for (int w = 0; w < kFilterWarps; ++w) top = sh.red[w] > top ? sh.red[w] : top;
-            a.out_tokens[row] = static_cast<int32_t>(0xFFFFFFFFu - static_cast<uint32_t>(top));
-        }
-        const unsigned long long total = block_sum(kept, sh);
-        if (threadIdx.x == 0 && a.out_kept) a.out_kept[row] = static_cast<int32_t>(total);
-        __syncthreads();
+        const bool stay = a.raw ? candidate_row<DTYPE, CS>(a, sh, row, part) : full_row<DTYPE, CS>(a, sh, row, part);
+        if (!stay) return;
     }
 }
 
@@ -652,17 +814,24 @@ extern "C" int sbw_bias_sample_filtered(const void *logits, int dtype, int64_t B
     const size_t es = dtype == SBW_DTYPE_F32 ? 4 : 2;
     const int64_t vp = static_cast<int64_t>(align_up(static_cast<size_t>(V), 8));
 
-    // l' of Eq. 2, in the logits' precision, into the workspace: one out-of-place pass of the bias
-    // kernel when the rows are 16-byte aligned, else a row copy and the in-place kernel
-    bool fused = false;
-    if (int rc = bias_copy_impl(logits, ld, workspace, dtype, B, V, vp, vocab_offset, ctx_tokens, ctx_width, key,
-                                gamma, delta, scheme, s, &fused))
-        return rc;
-    if (!fused) {
-        SBW_CUDA_TRY(cudaMemcpy2DAsync(workspace, vp * es, logits, ld * es, V * es, B, cudaMemcpyDeviceToDevice, s));
-        if (int rc = bias_logits_impl(workspace, dtype, B, V, vp, vocab_offset, ctx_tokens, ctx_width, key, gamma,
-                                      delta, scheme, s))
+    // With top_k set and 16-byte aligned rows the kernel works on the unbiased rows (candidate
+    // path) and no bias pass is launched.  Otherwise l' of Eq. 2, in the logits' precision, goes
+    // into the workspace first: one out-of-place pass of the bias kernel when the rows are aligned,
+    // else a row copy and the in-place kernel.
+    const bool candidates = top_k > 0 && top_k < V && reinterpret_cast<uintptr_t>(logits) % 16 == 0 &&
+                            (ld * es) % 16 == 0 && vocab_offset + V <= (int64_t(1) << 32) &&
+                            delta == delta && delta - delta == 0.0f;
+    if (!candidates) {
+        bool fused = false;
+        if (int rc = bias_copy_impl(logits, ld, workspace, dtype, B, V, vp, vocab_offset, ctx_tokens, ctx_width, key,
+                                    gamma, delta, scheme, s, &fused))
             return rc;
+        if (!fused) {
+            SBW_CUDA_TRY(cudaMemcpy2DAsync(workspace, vp * es, logits, ld * es, V * es, B, cudaMemcpyDeviceToDevice, s));
+            if (int rc = bias_logits_impl(workspace, dtype, B, V, vp, vocab_offset, ctx_tokens, ctx_width, key, gamma,
+                                          delta, scheme, s))
+                return rc;
+        }
     }
 
     FilterArgs a;
@@ -684,6 +853,15 @@ extern "C" int sbw_bias_sample_filtered(const void *logits, int dtype, int64_t B
     a.gkeys = make_block_keys(static_cast<uint32_t>(rng_seed), static_cast<uint32_t>(rng_seed >> 32));
     a.out_tokens = out_tokens;
     a.out_kept = out_kept;
+    a.raw = candidates ? logits : nullptr;
+    a.ld_raw = ld;
+    a.ctx = ctx_tokens;
+    a.W = ctx_width;
+    a.scheme = scheme;
+    a.key = key;
+    a.thr_m1 = threshold_minus_one(gamma);
+    a.delta = dtype == SBW_DTYPE_BF16 ? __bfloat162float(__float2bfloat16_rn(delta)) : delta;
+    a.weyl = make_weyl();
     // small batches: a cluster of CTAs per row, as many as keeps every SM busy with two CTAs
     const int64_t cap = 2LL * di.sm_count;
     const int cs = B * 8 <= cap ? 8 : B * 4 <= cap ? 4 : B * 2 <= cap ? 2 : 1;
