@@ -345,6 +345,9 @@ int sbw_roc_auc_batched(const double *z, const uint8_t *labels, const int64_t *o
  *   out_kept    device [B] int32 or NULL: the number of candidates left per row.
  *   workspace   device, 256-byte aligned, at least sbw_sample_filtered_workspace_bytes(dtype, B, V)
  *               bytes (a biased copy of the logits); contents undefined afterwards.
+ * With top_k set and 16-byte aligned rows the full-vocabulary hash is not evaluated: the columns that
+ * can reach the biased top-k are found on the unbiased logits (l >= k-th largest l - |delta|) and only
+ * they are hashed; the result is the same.
  * Rows that contain NaN are not supported (the result is some kept column).  V <= 2^21
  * (SBW_ERR_UNSUPPORTED beyond: the weight histogram's counters hold that many candidates).
  */
