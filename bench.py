@@ -440,10 +440,16 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
         c = inputs.uniform_tokens((B, 1), V2, seed=700 + B, device=dev)
         ids = torch.empty(B, dtype=torch.int32, device=dev)
         wsb = torch.empty(sbw.sbw_sample_workspace_bytes(B, V2), dtype=torch.uint8, device=dev)
+        zsum = torch.empty(B, dtype=torch.float32, device=dev)
         for name, scheme in (("context", sbw.SCHEME_CONTEXT), ("selfsalt", sbw.SCHEME_SELFSALT)):
-            s = _time_calls(lambda i: sbw.sbw_bias_sample(x, c, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, wsb), 20)
+            # with the softmax sum requested every logit is hashed; ids alone let the kernel screen on
+            # the Gumbel words first and hash only the candidates that could win
+            s = _time_calls(lambda i: sbw.sbw_bias_sample(x, c, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, wsb,
+                                                          out_sumexp=zsum), 20)
             out[f"sample_bf16_{name}_B{B}"] = {"gelem_s": B * V2 / s / 1e9, "ms": s * 1e3,
                                                "l2_resident": B * V2 * 2 < 100e6}
+            s = _time_calls(lambda i: sbw.sbw_bias_sample(x, c, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, wsb), 20)
+            out[f"sample_ids_only_bf16_{name}_B{B}"] = {"gelem_s": B * V2 / s / 1e9, "ms": s * 1e3}
     # Appendix F's sampling setting (temperature 0.7, top_p 0.8) and a top-k one, through the truncated sampler
     for B in (64, 1024):
         x = inputs.logits_normal(B, V2, 4.0, torch.bfloat16, seed=600 + B, device=dev)
@@ -496,7 +502,7 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
 
 PROFILE_CASES = ("topk40_fp32_selfsalt", "bias_bf16_context", "bias_bf16_selfsalt", "bias_fp32_context", "bias_fp32_selfsalt",
                  "detect_context", "detect_selfsalt", "sample_bf16_context", "sample_bf16_selfsalt",
-                 "detectunique_context", "filtered_bf16_context")
+                 "detectunique_context", "filtered_bf16_context", "sampleids_bf16_context", "sampleids_bf16_selfsalt")
 
 
 def run_profile_case(name: str, launches: int) -> None:
@@ -541,8 +547,10 @@ def run_profile_case(name: str, launches: int) -> None:
             fn = lambda i: sbw.sbw_bias_logits(x, ctx, KEY, 0.5, 2.0, scheme)  # noqa: E731
         else:
             ids = torch.empty(B, dtype=torch.int32, device=dev)
+            zsum = torch.empty(B, dtype=torch.float32, device=dev) if kind == "sample" else None
             ws = torch.empty(sbw.sbw_sample_workspace_bytes(B, V), dtype=torch.uint8, device=dev)
-            fn = lambda i: sbw.sbw_bias_sample(x, ctx, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, ws)  # noqa: E731
+            fn = lambda i: sbw.sbw_bias_sample(x, ctx, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, ws,  # noqa: E731
+                                               out_sumexp=zsum)
     for i in range(3 + launches):
         fn(i)
     torch.cuda.synchronize()

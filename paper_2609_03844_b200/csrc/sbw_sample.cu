@@ -67,6 +67,7 @@ struct SampleArgs {
     uint32_t thr_m1;
     float delta;          // in the logits' precision, widened
     uint32_t delta_bf16;  // bf16 bits of delta
+    float slack;          // max(delta, 0): the most a bias can add
     float inv_tau;        // 1/tau rounded once to fp32 (feeds the score)
     float c2_hi, c2_lo;   // log2(e)/tau as an fp32 pair (feeds the softmax sum)
     double tau;
@@ -282,6 +283,33 @@ __device__ __forceinline__ void load_biased(const SampleArgs &a, const RowSeedS<
     }
 }
 
+// Unbiased logits of slot j as raw bit patterns (fp32 bits, or bf16 bits in the low half) and
+// widened values; columns at or beyond V give -inf.
+template <int DTYPE, bool VECTOR, int VEC>
+__device__ __forceinline__ void load_raw(const char *row_ptr, uint32_t j, uint32_t cb, uint32_t V, uint32_t (&raw)[VEC],
+                                         float (&lr)[VEC]) {
+    if (VECTOR && cb + VEC <= V) {
+        const uint4 w = __ldg(reinterpret_cast<const uint4 *>(row_ptr) + j);
+        const uint32_t *e = reinterpret_cast<const uint32_t *>(&w);
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+            if constexpr (DTYPE == SBW_DTYPE_F32) raw[i] = e[i];
+            else raw[i] = (i & 1) ? e[i >> 1] >> 16 : e[i >> 1] & 0xffffu;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+            raw[i] = DTYPE == SBW_DTYPE_F32 ? 0xff800000u : 0xff80u;        // -inf
+            if (cb + i < V) {
+                if constexpr (DTYPE == SBW_DTYPE_F32) raw[i] = reinterpret_cast<const uint32_t *>(row_ptr)[cb + i];
+                else raw[i] = reinterpret_cast<const uint16_t *>(row_ptr)[cb + i];
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) lr[i] = __uint_as_float(DTYPE == SBW_DTYPE_F32 ? raw[i] : raw[i] << 16);
+}
+
 // Philox words of the Gumbel stream for the VEC candidates starting at global id vg:
 // candidate v uses word v & 3 of block v >> 2.
 template <int VEC>
@@ -306,7 +334,14 @@ __device__ __forceinline__ void gumbel_words(const SampleArgs &a, uint32_t vg, u
     }
 }
 
-template <int DTYPE, int SCHEME, bool VECTOR>
+// STATS = false serves callers that want the sampled ids only (no maximum, softmax sum,
+// probability or shard summary).  Then a logit's green test is needed only if the logit could
+// win: the Gumbel word of every candidate is drawn first (a quarter of a Philox block each), the
+// screen assumes the largest bias the candidate could get, l + max(delta, 0), and the green hash
+// -- four fifths of the multiplies of the full pass -- runs for the few candidates that survive.
+// The ids are the same: a candidate that fails the screen with the largest possible bias fails it
+// with its true one.
+template <int DTYPE, int SCHEME, bool VECTOR, bool STATS>
 __global__ void __launch_bounds__(kSampleThreads, SBW_SAMPLE_MIN_BLOCKS)
 sample_kernel(const SampleArgs a) {
     constexpr int VEC = VECTOR ? (DTYPE == SBW_DTYPE_F32 ? 4 : 8) : 1;
@@ -339,6 +374,47 @@ sample_kernel(const SampleArgs a) {
             const uint32_t j = jb + lane;
             const bool live = j < j_end;
             const uint32_t cb = j * VEC;
+            if constexpr (!STATS) {
+                uint32_t raw[VEC], y[VEC];
+                float lr[VEC];
+                if (live) {
+                    load_raw<DTYPE, VECTOR, VEC>(row_ptr, j, cb, V, raw, lr);
+                    gumbel_words<VEC>(a, a.vocab_offset + cb, rowb, y);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < VEC; ++i) { raw[i] = 0u; lr[i] = -INFINITY; y[i] = 0u; }
+                }
+                float vmax = lr[0];
+#pragma unroll
+                for (int i = 1; i < VEC; ++i) vmax = fmaxf(vmax, lr[i]);
+                // the largest biased value any of these logits could take, rounding included
+                float upper = vmax + a.slack;
+                upper += fabsf(upper) * (DTYPE == SBW_DTYPE_F32 ? 0x1p-22f : 0x1p-7f);
+                bound = fmaxf(bound, decode_score(shared_bound));
+                const uint32_t floor_word = word_floor(bound, upper, a.inv_tau);
+                bool maybe = false;
+#pragma unroll
+                for (int i = 0; i < VEC; ++i) maybe |= y[i] >= floor_word;
+                maybe &= live;
+                if (__any_sync(0xffffffffu, maybe)) {
+#pragma unroll
+                    for (int i = 0; i < VEC; ++i) {
+                        if (live && cb + i < V && y[i] >= floor_word) {
+                            const bool green = rs.word0(a.vocab_offset + cb + i, a.key, a.weyl) <= a.thr_m1;
+                            const float lp = biased<DTYPE>(raw[i], green, a.delta);
+                            const float s = __fmaf_rn(lp, a.inv_tau, gumbel_of_word(y[i]));
+                            if (s > best.s) { best.s = s; best.id = static_cast<int>(cb + i); best.l = lp; }
+                        }
+                    }
+                    float b = best.s;
+                    for (int d = 16; d > 0; d >>= 1) b = fmaxf(b, __shfl_xor_sync(0xffffffffu, b, d));
+                    if (b > bound) {
+                        bound = b;
+                        if (lane == 0) atomicMax(a.bounds + row, encode_score(b));
+                    }
+                }
+                continue;
+            }
             float lp[VEC];
             uint32_t y[VEC];
             if (live) {
@@ -496,7 +572,7 @@ int choose_split(int64_t B, int64_t nslot, int64_t ctas, int64_t max_parts) {
     return best;
 }
 
-template <int DTYPE, int SCHEME, bool VECTOR>
+template <int DTYPE, int SCHEME, bool VECTOR, bool STATS>
 int launch_one(SampleArgs &a, int64_t nslot, size_t partial_bytes, cudaStream_t s) {
     DeviceInfo di;
     const int rc = current_device_info(&di);
@@ -504,7 +580,7 @@ int launch_one(SampleArgs &a, int64_t nslot, size_t partial_bytes, cudaStream_t 
     static std::atomic<int> blocks_per_sm{0};  // a property of the compiled kernel, equal on every sm_100a device
     if (blocks_per_sm == 0) {
         int n = 0;
-        SBW_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, sample_kernel<DTYPE, SCHEME, VECTOR>,
+        SBW_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, sample_kernel<DTYPE, SCHEME, VECTOR, STATS>,
                                                                    kSampleThreads, 0));
         blocks_per_sm = n > 0 ? n : 1;
     }
@@ -516,15 +592,18 @@ int launch_one(SampleArgs &a, int64_t nslot, size_t partial_bytes, cudaStream_t 
     SBW_CUDA_TRY(cudaMemsetAsync(a.tickets, 0, 2 * static_cast<size_t>(a.B) * sizeof(unsigned), s));
     const int64_t want_ctas = (a.n_items + kSampleWarps - 1) / kSampleWarps;
     const unsigned grid = static_cast<unsigned>(want_ctas < ctas ? want_ctas : ctas);
-    sample_kernel<DTYPE, SCHEME, VECTOR><<<grid, kSampleThreads, 0, s>>>(a);
+    sample_kernel<DTYPE, SCHEME, VECTOR, STATS><<<grid, kSampleThreads, 0, s>>>(a);
     SBW_CUDA_TRY(cudaGetLastError());
     return SBW_OK;
 }
 
 template <int DTYPE, int SCHEME>
 int launch(SampleArgs &a, bool vector, int64_t nslot, size_t partial_bytes, float *out_probs, cudaStream_t s) {
-    const int rc = vector ? launch_one<DTYPE, SCHEME, true>(a, nslot, partial_bytes, s)
-                          : launch_one<DTYPE, SCHEME, false>(a, nslot, partial_bytes, s);
+    const bool stats = a.out_max || a.out_sumexp || a.out_prob || a.out_shard || out_probs;
+    const int rc = stats ? (vector ? launch_one<DTYPE, SCHEME, true, true>(a, nslot, partial_bytes, s)
+                                   : launch_one<DTYPE, SCHEME, false, true>(a, nslot, partial_bytes, s))
+                         : (vector ? launch_one<DTYPE, SCHEME, true, false>(a, nslot, partial_bytes, s)
+                                   : launch_one<DTYPE, SCHEME, false, false>(a, nslot, partial_bytes, s));
     if (rc != SBW_OK) return rc;
     if (out_probs) {
         const unsigned gx = static_cast<unsigned>((a.V + 255) / 256 < 1024 ? (a.V + 255) / 256 : 1024);
@@ -582,6 +661,7 @@ int bias_sample_impl(const void *logits, int dtype, int64_t B, int64_t V, int64_
         a.delta_bf16 = static_cast<uint32_t>(__bfloat16_as_ushort(d));
         a.delta = __bfloat162float(d);
     }
+    a.slack = a.delta > 0.0f ? a.delta : 0.0f;
     a.inv_tau = 1.0f / temperature;
     a.c2_hi = c2_hi;
     a.c2_lo = static_cast<float>(c2 - static_cast<double>(c2_hi));

@@ -151,3 +151,29 @@ def test_sampled_tokens_feed_the_next_step():
         assert np.array_equal(nxt.cpu().numpy(), want["tokens"])
         ctx_dev = nxt.view(B, 1)
         ctx_host = want["tokens"].reshape(B, 1).copy()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("scheme", SCHEMES)
+@pytest.mark.parametrize("delta", [0.5, 4.0, -1.5, 0.0])
+def test_ids_only_calls_skip_the_green_test_where_it_cannot_matter(dtype, scheme, delta):
+    """Without statistics outputs the kernel screens on the Gumbel words first and hashes only the
+    candidates that could win with the largest possible bias: the ids must not change."""
+    dev = require_gpu()
+    for B, V, ld, tau in ((1, 128256, 128256, 0.7), (9, 20011, 20016, 1.3), (130, 5000, 5003, 0.3)):
+        x = inputs.logits_normal(B, ld, 3.0, dtype, seed=7 + B)
+        ctx = inputs.uniform_tokens((B, 2), V, seed=8 + B)
+        xd, cd = x.to(dev), ctx.to(dev)
+        ws = torch.empty(sbw.sbw_sample_workspace_bytes(B, V), dtype=torch.uint8, device=dev)
+        ids = torch.empty(B, dtype=torch.int32, device=dev)
+        ids_stats = torch.empty(B, dtype=torch.int32, device=dev)
+        m = torch.empty(B, dtype=torch.float32, device=dev)
+        for step in range(3):
+            sbw.sbw_bias_sample(xd, cd, KEY, 0.25, delta, scheme, tau, 3, step, ids, ws, V=V, vocab_offset=11)
+            sbw.sbw_bias_sample(xd, cd, KEY, 0.25, delta, scheme, tau, 3, step, ids_stats, ws, out_max=m, V=V,
+                                vocab_offset=11)
+            torch.cuda.synchronize()
+            want = oracle.bias_sample(host_bits(x), V, ctx.numpy(), KEY, 0.25, delta, scheme, tau, 3, step,
+                                      vocab_offset=11, threads=8)
+            assert np.array_equal(ids.cpu().numpy(), want["tokens"])
+            assert np.array_equal(ids_stats.cpu().numpy(), want["tokens"])
