@@ -341,8 +341,11 @@ __device__ __forceinline__ void gumbel_words(const SampleArgs &a, uint32_t vg, u
 // -- four fifths of the multiplies of the full pass -- runs for the few candidates that survive.
 // The ids are the same: a candidate that fails the screen with the largest possible bias fails it
 // with its true one.
+#ifndef SBW_SAMPLE_IDS_MIN_BLOCKS
+#define SBW_SAMPLE_IDS_MIN_BLOCKS 3
+#endif
 template <int DTYPE, int SCHEME, bool VECTOR, bool STATS>
-__global__ void __launch_bounds__(kSampleThreads, SBW_SAMPLE_MIN_BLOCKS)
+__global__ void __launch_bounds__(kSampleThreads, STATS ? SBW_SAMPLE_MIN_BLOCKS : SBW_SAMPLE_IDS_MIN_BLOCKS)
 sample_kernel(const SampleArgs a) {
     constexpr int VEC = VECTOR ? (DTYPE == SBW_DTYPE_F32 ? 4 : 8) : 1;
     constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
@@ -586,7 +589,12 @@ int launch_one(SampleArgs &a, int64_t nslot, size_t partial_bytes, cudaStream_t 
     }
     const int64_t ctas = static_cast<int64_t>(di.sm_count) * blocks_per_sm;
     const int64_t warps = ctas * kSampleWarps;
-    a.split = choose_split(a.B, nslot, warps, static_cast<int64_t>(partial_bytes / sizeof(Partial)));
+    // small batches: no more chunks per row than fill two CTAs per SM, even when more CTAs fit --
+    // beyond that the extra partials cost more in the final merge than the extra warps bring
+    int64_t max_parts = static_cast<int64_t>(partial_bytes / sizeof(Partial));
+    const int64_t two_per_sm = static_cast<int64_t>(di.sm_count) * 2 * kSampleWarps;
+    if (two_per_sm / a.B >= 32 && max_parts > two_per_sm) max_parts = two_per_sm;
+    a.split = choose_split(a.B, nslot, warps, max_parts);
     a.n_items = a.B * a.split;
     a.slots_per_chunk = static_cast<uint32_t>((nslot + a.split - 1) / a.split);
     SBW_CUDA_TRY(cudaMemsetAsync(a.tickets, 0, 2 * static_cast<size_t>(a.B) * sizeof(unsigned), s));
