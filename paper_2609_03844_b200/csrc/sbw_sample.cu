@@ -378,6 +378,9 @@ sample_kernel(const SampleArgs a) {
             const bool live = j < j_end;
             const uint32_t cb = j * VEC;
             if constexpr (!STATS) {
+                // this path waits on its loads: ask for the next trip's logits now
+                if (VECTOR && j + 32 < j_end)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint4 *>(row_ptr) + j + 32));
                 uint32_t raw[VEC], y[VEC];
                 float lr[VEC];
                 if (live) {
