@@ -139,6 +139,9 @@ int sbw_bias_logits_host(void *logits_host, int dtype, int64_t B, int64_t V, int
  *   out_max, out_sumexp, out_prob   device [B] float, each may be NULL: m, Z, p.
  *   out_probs     device [B, V] float or NULL: the full softmax of the biased logits
  *                 (costs a second pass; meant for tests and small batches).
+ *                 With all four NULL only the ids are produced, and the green test is evaluated
+ *                 only for candidates whose Gumbel variate could make them win (same ids, about
+ *                 twice the throughput).
  *   workspace     device scratch, 256-byte aligned, at least
  *                 sbw_sample_workspace_bytes(B, V) bytes; contents undefined afterwards.
  *                 Calls that share a workspace must not overlap on the GPU.
