@@ -147,3 +147,24 @@ def test_every_cluster_size(B):
     _check(x, ctx, sbw.SCHEME_SELFSALT, 0.7, 40, 0.9)
     _check(x, ctx, sbw.SCHEME_CONTEXT, 1.0, 700, 1.0)
     _check(x.float(), ctx, sbw.SCHEME_CONTEXT, 0.7, 0, 0.97)
+
+
+@pytest.mark.parametrize("dtype,base", [(torch.bfloat16, 256.0), (torch.float32, 16777216.0)])
+@pytest.mark.parametrize("delta", [1.0, 2.0, 3.0, -1.0])
+def test_rounding_of_the_biased_sum_at_the_cut(dtype, base, delta):
+    """Logits around a power of two where the spacing of the type doubles: l + delta rounds (ties to
+    even), biased values collapse onto each other, and the k-th largest biased logit is reached by
+    columns whose exact sum lies below it.  The candidate threshold has to keep all of them."""
+    B, V = 6, 9000
+    rng = np.random.default_rng(int(base) % 97 + int(delta * 4) + 20)
+    step = base / 256.0                                        # spacing below `base`
+    grid = base + step * rng.integers(-40, 12, size=(B, V))    # above `base` every other value is not representable
+    x = torch.from_numpy(grid).to(dtype)
+    x[:, ::7] = x[:, ::7] - 50 * step                          # a bulk below the interesting range
+    # rows 3..5: only some 600 columns stay near the top, so that the candidates fit the list
+    sparse = torch.from_numpy(rng.random((3, V)) < 0.93)
+    x[3:][sparse] = x[3:][sparse] - 1000 * step
+    ctx = inputs.uniform_tokens((B, 1), V, seed=3)
+    for top_k in (5, 50, 300):
+        _check(x, ctx, sbw.SCHEME_CONTEXT, 1.0, top_k, 1.0, delta=delta * step, gamma=0.5)
+        _check(x, ctx, sbw.SCHEME_SELFSALT, 1.0, top_k, 0.7, delta=delta * step, gamma=0.5)
