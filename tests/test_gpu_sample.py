@@ -177,3 +177,25 @@ def test_ids_only_calls_skip_the_green_test_where_it_cannot_matter(dtype, scheme
                                       vocab_offset=11, threads=8)
             assert np.array_equal(ids.cpu().numpy(), want["tokens"])
             assert np.array_equal(ids_stats.cpu().numpy(), want["tokens"])
+
+
+@pytest.mark.parametrize("dtype,base", [(torch.bfloat16, 256.0), (torch.float32, 16777216.0)])
+def test_ids_only_screen_allows_for_the_rounding_of_the_biased_sum(dtype, base):
+    """Logits next to a power of two, where l + delta rounds up by half a spacing: the screen's
+    bound on the biased value must cover that."""
+    dev = require_gpu()
+    B, V = 4, 6000
+    rng = np.random.default_rng(5)
+    step = base / 256.0
+    x = torch.from_numpy(base + step * rng.integers(-6, 3, size=(B, V))).to(dtype)
+    ctx = inputs.uniform_tokens((B, 1), V, seed=6)
+    xd, cd = x.to(dev), ctx.to(dev)
+    ws = torch.empty(sbw.sbw_sample_workspace_bytes(B, V), dtype=torch.uint8, device=dev)
+    ids = torch.empty(B, dtype=torch.int32, device=dev)
+    tau = float(step)                                          # scores then differ by O(1) between neighbours
+    for delta in (1.0, 3.0):
+        for step_no in range(12):
+            sbw.sbw_bias_sample(xd, cd, KEY, 0.5, delta * step, 0, tau, 3, step_no, ids, ws)
+            torch.cuda.synchronize()
+            want = oracle.bias_sample(host_bits(x), V, ctx.numpy(), KEY, 0.5, delta * step, 0, tau, 3, step_no)
+            assert np.array_equal(ids.cpu().numpy(), want["tokens"])
