@@ -116,6 +116,23 @@ __device__ __forceinline__ float value_of_code(uint32_t code) {
     return __uint_as_float(b16 << 16);
 }
 
+// The two hot passes work on a cheaper monotone key, a signed integer made from the raw bits in
+// two operations (flip the magnitude bits of negative values); for bf16 the bits are the widened
+// ones, so the key of a negative value carries 0xFFFF in its low half.  key >= key_of_code(c) is
+// code >= c.
+__device__ __forceinline__ int32_t order_key(uint32_t bits32) {
+    return static_cast<int32_t>(bits32 ^ (static_cast<uint32_t>(static_cast<int32_t>(bits32) >> 31) & 0x7fffffffu));
+}
+template <int DTYPE>
+__device__ __forceinline__ uint32_t code_of_key(int32_t key) {
+    const uint32_t c = static_cast<uint32_t>(key) ^ 0x80000000u;
+    return DTYPE == SBW_DTYPE_F32 ? c : c >> 16;
+}
+template <int DTYPE>
+__device__ __forceinline__ int32_t key_of_code(uint32_t code) {
+    return static_cast<int32_t>((DTYPE == SBW_DTYPE_F32 ? code : code << 16) ^ 0x80000000u);
+}
+
 // Integer softmax weight of a candidate at distance `dist` below the maximum code (see the oracle
 // of this library for the same steps): 2^40 at the maximum, trunc(2^(40 + (l' - m) c)) below it.
 __device__ __forceinline__ unsigned long long nucleus_weight(float l, float m, bool is_max, float c) {
@@ -177,6 +194,35 @@ __device__ __forceinline__ void for_each(const char *row_ptr, uint32_t V, uint32
 template <int DTYPE, typename F>
 __device__ __forceinline__ void for_each(const char *row_ptr, uint32_t V, F f) {
     for_each<DTYPE>(row_ptr, V, 0u, vectors_of<DTYPE>(V), f);
+}
+
+// The same walk handing out f(column, widened bits, key).
+template <int DTYPE, typename F>
+__device__ __forceinline__ void for_each_key(const char *row_ptr, uint32_t V, uint32_t vec_begin, uint32_t nvec, F f) {
+    constexpr int VEC = DTYPE == SBW_DTYPE_F32 ? 4 : 8;
+    constexpr int kInFlight = 4;
+    for (uint32_t j0 = vec_begin + threadIdx.x; j0 < nvec; j0 += kInFlight * kFilterThreads) {
+        uint4 w[kInFlight];
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+            const uint32_t j = j0 + u * kFilterThreads;
+            w[u] = j < nvec ? reinterpret_cast<const uint4 *>(row_ptr)[j] : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+            const uint32_t j = j0 + u * kFilterThreads;
+            if (j >= nvec) break;
+            const uint32_t *e = reinterpret_cast<const uint32_t *>(&w[u]);
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                uint32_t bits;
+                if constexpr (DTYPE == SBW_DTYPE_F32) bits = e[i];
+                else bits = (i & 1) ? (e[i >> 1] & 0xffff0000u) : (e[i >> 1] << 16);
+                const uint32_t col = j * VEC + i;
+                if (col < V) f(col, bits, order_key(bits));
+            }
+        }
+    }
 }
 
 __device__ __forceinline__ unsigned long long warp_sum(unsigned long long x) {
@@ -453,8 +499,9 @@ __device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &s
     Head h;
     h.leave = false;
     // pass A: per-thread maxima, sorted descending (as ~code ascending) in the list area
-    uint32_t my_max = 0;
-    for_each<DTYPE>(src_row, V, vec_lo, vec_hi, [&](uint32_t, uint32_t code) { my_max = max(my_max, code); });
+    int32_t my_key = static_cast<int32_t>(0x80000000u);        // decodes to code 0
+    for_each_key<DTYPE>(src_row, V, vec_lo, vec_hi, [&](uint32_t, uint32_t, int32_t key) { my_key = max(my_key, key); });
+    const uint32_t my_max = code_of_key<DTYPE>(my_key);
     __syncthreads();
     sh.list[threadIdx.x] = static_cast<unsigned long long>(~my_max);
     if (threadIdx.x == 0) sh.list_n = 0u;
@@ -497,12 +544,14 @@ __device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &s
 
     // pass B
     unsigned long long z_local = 0;
-    for_each<DTYPE>(src_row, V, vec_lo, vec_hi, [&](uint32_t col, uint32_t code) {
-        const uint32_t dist = key_m - code;
-        if (want_z && code >= code_lo) z_local += nucleus_weight(value_of_code<DTYPE>(code), m, dist == 0u, a.c);
-        if (code >= floor_code && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= kListCap) {
+    const int32_t floor_key = key_of_code<DTYPE>(floor_code), lo_key = key_of_code<DTYPE>(code_lo);
+    for_each_key<DTYPE>(src_row, V, vec_lo, vec_hi, [&](uint32_t col, uint32_t bits, int32_t key) {
+        if (want_z && key >= lo_key)
+            z_local += nucleus_weight(__uint_as_float(bits), m, code_of_key<DTYPE>(key) == key_m, a.c);
+        if (key >= floor_key && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= kListCap) {
             const unsigned idx = atomicAdd(&sh.list_n, 1u);
-            if (idx < kListCap) sh.list[idx] = (static_cast<unsigned long long>(dist) << 32) | col;
+            if (idx < kListCap)
+                sh.list[idx] = (static_cast<unsigned long long>(key_m - code_of_key<DTYPE>(key)) << 32) | col;
         }
     });
     h.z_all = want_z ? block_sum(z_local, sh) : 0ull;
