@@ -196,31 +196,43 @@ __device__ __forceinline__ void for_each(const char *row_ptr, uint32_t V, F f) {
     for_each<DTYPE>(row_ptr, V, 0u, vectors_of<DTYPE>(V), f);
 }
 
-// The same walk handing out f(column, widened bits, key).
+// The same walk handing out f(column, widened bits, key).  Whole vectors need no column check;
+// a ragged last vector is done by one thread afterwards.
 template <int DTYPE, typename F>
 __device__ __forceinline__ void for_each_key(const char *row_ptr, uint32_t V, uint32_t vec_begin, uint32_t nvec, F f) {
     constexpr int VEC = DTYPE == SBW_DTYPE_F32 ? 4 : 8;
     constexpr int kInFlight = 4;
-    for (uint32_t j0 = vec_begin + threadIdx.x; j0 < nvec; j0 += kInFlight * kFilterThreads) {
+    const uint32_t nfull = min(nvec, V / VEC);
+    for (uint32_t j0 = vec_begin + threadIdx.x; j0 < nfull; j0 += kInFlight * kFilterThreads) {
         uint4 w[kInFlight];
 #pragma unroll
         for (int u = 0; u < kInFlight; ++u) {
             const uint32_t j = j0 + u * kFilterThreads;
-            w[u] = j < nvec ? reinterpret_cast<const uint4 *>(row_ptr)[j] : make_uint4(0, 0, 0, 0);
+            w[u] = j < nfull ? reinterpret_cast<const uint4 *>(row_ptr)[j] : make_uint4(0, 0, 0, 0);
         }
 #pragma unroll
         for (int u = 0; u < kInFlight; ++u) {
             const uint32_t j = j0 + u * kFilterThreads;
-            if (j >= nvec) break;
+            if (j >= nfull) break;
             const uint32_t *e = reinterpret_cast<const uint32_t *>(&w[u]);
 #pragma unroll
             for (int i = 0; i < VEC; ++i) {
                 uint32_t bits;
                 if constexpr (DTYPE == SBW_DTYPE_F32) bits = e[i];
                 else bits = (i & 1) ? (e[i >> 1] & 0xffff0000u) : (e[i >> 1] << 16);
-                const uint32_t col = j * VEC + i;
-                if (col < V) f(col, bits, order_key(bits));
+                f(j * VEC + i, bits, order_key(bits));
             }
+        }
+    }
+    if (nfull < nvec && nfull >= vec_begin && threadIdx.x == 0) {
+        const uint4 w = reinterpret_cast<const uint4 *>(row_ptr)[nfull];
+        const uint32_t *e = reinterpret_cast<const uint32_t *>(&w);
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+            uint32_t bits;
+            if constexpr (DTYPE == SBW_DTYPE_F32) bits = e[i];
+            else bits = (i & 1) ? (e[i >> 1] & 0xffff0000u) : (e[i >> 1] << 16);
+            if (nfull * VEC + i < V) f(nfull * VEC + i, bits, order_key(bits));
         }
     }
 }
