@@ -201,6 +201,23 @@ __device__ __forceinline__ float biased(uint32_t raw, bool green, float delta) {
 // L2): the row maximum first, then every partial's sum rescaled to it -- one independent fp32
 // exp2 per partial (the partial that holds the maximum is scaled by exactly 1), accumulated in
 // fp64 in index order per lane.  The sampled probability is one fp64 exp per row.
+// Ids only: one pass, best score and its column.
+__device__ void finish_row_ids(const SampleArgs &a, int64_t row, const Partial *parts, int n) {
+    const int lane = threadIdx.x & 31;
+    float s = -INFINITY;
+    int id = INT_MAX;
+    for (int i = lane; i < n; i += 32) {
+        const float4 q0 = __ldcg(reinterpret_cast<const float4 *>(parts + i));
+        if (better(q0.z, __float_as_int(q0.w), s, id)) { s = q0.z; id = __float_as_int(q0.w); }
+    }
+    for (int d = 16; d > 0; d >>= 1) {
+        const float os = __shfl_down_sync(0xffffffffu, s, d);
+        const int oid = __shfl_down_sync(0xffffffffu, id, d);
+        if (better(os, oid, s, id)) { s = os; id = oid; }
+    }
+    if (lane == 0) a.out_tokens[row] = id == INT_MAX ? 0 : id;   // every score was -inf: lowest id
+}
+
 __device__ void finish_row(const SampleArgs &a, int64_t row, const Partial *parts, int n) {
     const int lane = threadIdx.x & 31;
     float m = -INFINITY;
@@ -499,7 +516,9 @@ sample_kernel(const SampleArgs a) {
         ticket = __shfl_sync(0xffffffffu, ticket, 0);
         if (a.split == 1 || ticket == static_cast<unsigned>(a.split - 1)) {
             __threadfence();                           // the other warps' partials are visible now
-            finish_row(a, row, a.partials + row * a.split, a.split);
+            // ids only and many partials (small batches): the single-pass merge
+            if (!STATS && a.split > 16) finish_row_ids(a, row, a.partials + row * a.split, a.split);
+            else finish_row(a, row, a.partials + row * a.split, a.split);
             if (lane == 0 && a.split > 1) a.tickets[row] = 0;
         }
     }
