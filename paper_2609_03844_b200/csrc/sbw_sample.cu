@@ -358,6 +358,12 @@ __device__ __forceinline__ void gumbel_words(const SampleArgs &a, uint32_t vg, u
 // -- four fifths of the multiplies of the full pass -- runs for the few candidates that survive.
 // The ids are the same: a candidate that fails the screen with the largest possible bias fails it
 // with its true one.
+__global__ void __launch_bounds__(1024) clear_kernel(unsigned *p, unsigned n) {
+    asm volatile("griddepcontrol.launch_dependents;");
+    const unsigned i = blockIdx.x * 1024u + threadIdx.x;
+    if (i < n) p[i] = 0u;
+}
+
 #ifndef SBW_SAMPLE_IDS_MIN_BLOCKS
 #define SBW_SAMPLE_IDS_MIN_BLOCKS 3
 #endif
@@ -370,6 +376,8 @@ sample_kernel(const SampleArgs a) {
     const int64_t warp_id = static_cast<int64_t>(blockIdx.x) * kSampleWarps + (threadIdx.x >> 5);
     const int64_t n_warps = static_cast<int64_t>(gridDim.x) * kSampleWarps;
     const uint32_t V = static_cast<uint32_t>(a.V);
+    // the kernel that clears tickets and bounds may still be running (see launch_one)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     for (int64_t item = warp_id; item < a.n_items; item += n_warps) {
         const int64_t row = item / a.split;
@@ -619,11 +627,25 @@ int launch_one(SampleArgs &a, int64_t nslot, size_t partial_bytes, cudaStream_t 
     a.split = choose_split(a.B, nslot, warps, max_parts);
     a.n_items = a.B * a.split;
     a.slots_per_chunk = static_cast<uint32_t>((nslot + a.split - 1) / a.split);
-    SBW_CUDA_TRY(cudaMemsetAsync(a.tickets, 0, 2 * static_cast<size_t>(a.B) * sizeof(unsigned), s));
     const int64_t want_ctas = (a.n_items + kSampleWarps - 1) / kSampleWarps;
     const unsigned grid = static_cast<unsigned>(want_ctas < ctas ? want_ctas : ctas);
-    sample_kernel<DTYPE, SCHEME, VECTOR, STATS><<<grid, kSampleThreads, 0, s>>>(a);
-    SBW_CUDA_TRY(cudaGetLastError());
+    // Tickets and bounds start at zero.  Inside a stream capture (where the device-side gap between
+    // the two nodes is what counts) they are cleared by a small kernel that releases its dependents
+    // at once, and the sampler is launched with programmatic stream serialisation: its launch
+    // overlaps the clearing, and it waits (griddepcontrol.wait) before it touches the workspace.
+    // Outside a capture the plain memset + launch is cheaper for the host.
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    SBW_CUDA_TRY(cudaStreamIsCapturing(s, &capturing));
+    if (capturing == cudaStreamCaptureStatusActive) {
+        const unsigned words = static_cast<unsigned>(2 * a.B);
+        clear_kernel<<<(words + 1023) / 1024, 1024, 0, s>>>(a.tickets, words);
+        SBW_CUDA_TRY(cudaGetLastError());
+        SBW_CUDA_TRY(launch_pdl(sample_kernel<DTYPE, SCHEME, VECTOR, STATS>, dim3(grid), dim3(kSampleThreads), s, a));
+    } else {
+        SBW_CUDA_TRY(cudaMemsetAsync(a.tickets, 0, 2 * static_cast<size_t>(a.B) * sizeof(unsigned), s));
+        sample_kernel<DTYPE, SCHEME, VECTOR, STATS><<<grid, kSampleThreads, 0, s>>>(a);
+        SBW_CUDA_TRY(cudaGetLastError());
+    }
     return SBW_OK;
 }
 
