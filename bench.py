@@ -373,6 +373,34 @@ def _time_calls(fn, n, warm=3):
     return e0.elapsed_time(e1) * 1e-3 / n
 
 
+def _time_graph(fn, n, reps=10, warm=3):
+    """Device time per call of `n` calls captured into one CUDA graph and replayed `reps` times
+    (what a serving loop that replays its decode step sees; stream launches of calls this short
+    measure the host instead)."""
+    import torch
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for i in range(warm):
+            fn(i)
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(n):
+                fn(warm + i)
+        graph.replay()
+        side.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(side)
+        for _ in range(reps):
+            graph.replay()
+        e1.record(side)
+        e1.synchronize()
+    torch.cuda.current_stream().wait_stream(side)
+    return e0.elapsed_time(e1) * 1e-3 / (n * reps)
+
+
 def run_extra(sbw, inputs, dev, peaks) -> dict:
     """The other workloads of the hot path, each timed on its own (inputs larger than L2 or
     rotating), and the integer-throughput probe."""
@@ -450,6 +478,12 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
                                                "l2_resident": B * V2 * 2 < 100e6}
             s = _time_calls(lambda i: sbw.sbw_bias_sample(x, c, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, wsb), 20)
             out[f"sample_ids_only_bf16_{name}_B{B}"] = {"gelem_s": B * V2 / s / 1e9, "ms": s * 1e3}
+            if B <= 32:   # calls this short are host-bound as stream launches: device time from a graph
+                s = _time_graph(lambda i: sbw.sbw_bias_sample(x, c, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, wsb,
+                                                              out_sumexp=zsum), 16)
+                out[f"sample_bf16_{name}_B{B}"]["graph_ms"] = s * 1e3
+                s = _time_graph(lambda i: sbw.sbw_bias_sample(x, c, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, wsb), 16)
+                out[f"sample_ids_only_bf16_{name}_B{B}"]["graph_ms"] = s * 1e3
     # Appendix F's sampling setting (temperature 0.7, top_p 0.8) and a top-k one, through the truncated sampler
     for B in (64, 1024):
         x = inputs.logits_normal(B, V2, 4.0, torch.bfloat16, seed=600 + B, device=dev)
