@@ -239,8 +239,10 @@ int scan_lengths(const int32_t *lengths, int64_t N, void *workspace, int64_t **o
     int64_t *tile_sums = reinterpret_cast<int64_t *>(
         static_cast<char *>(workspace) + align_up((static_cast<size_t>(N) + 1) * sizeof(int64_t), 256));
     const unsigned tiles = static_cast<unsigned>((N + kScanTile - 1) / kScanTile);
-    scan_tile_sums<<<tiles, kScanThreads, 0, s>>>(lengths, N, tile_sums);
-    SBW_CUDA_TRY(cudaGetLastError());
+    if (tiles > 1) {                                 // a single tile has no earlier tiles to add up
+        scan_tile_sums<<<tiles, kScanThreads, 0, s>>>(lengths, N, tile_sums);
+        SBW_CUDA_TRY(cudaGetLastError());
+    }
     scan_offsets<<<tiles, kScanThreads, 0, s>>>(lengths, N, tile_sums, ws_offsets);
     SBW_CUDA_TRY(cudaGetLastError());
     *out_offsets = ws_offsets;
