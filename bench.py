@@ -521,7 +521,8 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
                 if i >= 20:
                     times.append(e0.elapsed_time(e1))
             times.sort()
-            sweep[f"{name}_B{B}"] = {"p50_ms": times[len(times) // 2], "p99_ms": times[int(len(times) * 0.99)],
+            sweep[f"{name}_B{B}"] = {"p50_ms": times[len(times) // 2], "p95_ms": times[int(len(times) * 0.95)],
+                                     "p99_ms": times[int(len(times) * 0.99)],
                                      "l2_resident": B * 151936 * 4 < 100e6}
     out["paper_protocol_latency_fp32_V151936_W4"] = sweep
     # integer-throughput probe
