@@ -438,6 +438,9 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
     s = _time_calls(lambda i: sbw.sbw_bias_logits(p2[i % 16], c2[i % 16], KEY, 0.5, 2.0, sbw.SCHEME_SELFSALT), 256)
     out["bias_bf16_selfsalt_B64_V128256"] = {"gelem_s": B2 * V2 / s / 1e9, "ms": s * 1e3,
                                              **place(INT_OPS["selfsalt"] * B2 * V2, 4 * B2 * V2, s)}
+    # the headline step on ONE buffer that stays in L2 (16.4 MB): labelled L2-warm, not a roofline input
+    s = _time_graph(lambda i: sbw.sbw_bias_logits(p2[0], c2[0], KEY, 0.5, 2.0, sbw.SCHEME_CONTEXT), 64)
+    out["bias_bf16_context_B64_V128256_l2_warm_single_buffer"] = {"gelem_s": B2 * V2 / s / 1e9, "ms": s * 1e3}
     del p2, c2
     # config 5 (null half shape): 100000 sequences, lengths uniform in [64, 1024], 218 MB of ids
     N = 100000
