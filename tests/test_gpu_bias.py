@@ -112,6 +112,27 @@ def test_config2_shape_one_step_bf16():
     assert_same_bits(host_bits(x), want)
 
 
+def test_config2_all_256_decode_steps():
+    """Config 2 in full: 256 consecutive decode steps, each on its own (64, 128256) bf16 tensor and
+    context column, launched back to back as the benchmark does; every one of the 2.1e9 biased
+    logits is compared with the oracle (16 steps resident at a time)."""
+    import os
+
+    dev = require_gpu()
+    threads = min(32, os.cpu_count() or 8)
+    for first in range(0, 256, 16):
+        xs = [inputs.logits_normal(64, 128256, 4.0, torch.bfloat16, seed=5000 + t, device=dev)
+              for t in range(first, first + 16)]
+        cs = [inputs.uniform_tokens((64, 1), 128256, seed=6000 + t, device=dev) for t in range(first, first + 16)]
+        before = [host_bits(x) for x in xs]
+        for x, c in zip(xs, cs):
+            sbw.sbw_bias_logits(x, c, KEY, 0.5, 2.0, sbw.SCHEME_CONTEXT)
+        torch.cuda.synchronize()
+        for x, c, b in zip(xs, cs, before):
+            want = oracle.bias_logits(b, 128256, c.cpu().numpy(), KEY, 0.5, 2.0, oracle.SCHEME_CONTEXT, threads=threads)
+            assert host_bits(x).tobytes() == want.tobytes()
+
+
 def test_config3_shape_one_step_fp32_selfsalt_with_zipf_spike():
     """B=256, V=151936 fp32 N(0, 4^2) + Zipf(1.1) spike on 50 ids per row, self-salt, gamma .25,
     delta 4 -- every element."""
