@@ -199,3 +199,38 @@ def test_ids_only_screen_allows_for_the_rounding_of_the_biased_sum(dtype, base):
             torch.cuda.synchronize()
             want = oracle.bias_sample(host_bits(x), V, ctx.numpy(), KEY, 0.5, delta * step, 0, tau, 3, step_no)
             assert np.array_equal(ids.cpu().numpy(), want["tokens"])
+
+
+def test_config4_all_96_combinations():
+    """Config 4 in full: B in {1, 8, 32, 128, 512, 1024} x both schemes x gamma in {.25, .5} x delta in
+    {.5, 1, 2, 4}, V = 128256 bf16, tau 0.7.  The batches are the leading rows of one tensor, so one
+    oracle pass per (scheme, gamma, delta) serves all six batch sizes; ids bit-exact from both
+    kernels (with and without statistics), m exact, Z and p within 1e-6."""
+    import os
+
+    dev = require_gpu()
+    threads = min(32, os.cpu_count() or 8)
+    V, Bmax, tau = 128256, 1024, 0.7
+    x = inputs.logits_normal(Bmax, V, 4.0, torch.bfloat16, seed=0xC4, device=dev)
+    ctx = inputs.uniform_tokens((Bmax, 1), V, seed=0xC5, device=dev)
+    xh, ch = host_bits(x), ctx.cpu().numpy()
+    ws = torch.empty(sbw.sbw_sample_workspace_bytes(Bmax, V), dtype=torch.uint8, device=dev)
+    ids, ids_only = (torch.empty(Bmax, dtype=torch.int32, device=dev) for _ in range(2))
+    m, Z, p = (torch.empty(Bmax, dtype=torch.float32, device=dev) for _ in range(3))
+    step = 0
+    for scheme in SCHEMES:
+        for gamma in (0.25, 0.5):
+            for delta in (0.5, 1.0, 2.0, 4.0):
+                step += 1
+                want = oracle.bias_sample(xh, V, ch, KEY, gamma, delta, scheme, tau, 0xC4, step, threads=threads)
+                for B in (1, 8, 32, 128, 512, 1024):
+                    sbw.sbw_bias_sample(x[:B], ctx[:B], KEY, gamma, delta, scheme, tau, 0xC4, step, ids[:B], ws,
+                                        out_max=m[:B], out_sumexp=Z[:B], out_prob=p[:B])
+                    sbw.sbw_bias_sample(x[:B], ctx[:B], KEY, gamma, delta, scheme, tau, 0xC4, step, ids_only[:B], ws)
+                    torch.cuda.synchronize()
+                    tag = (scheme, gamma, delta, B)
+                    assert np.array_equal(ids[:B].cpu().numpy(), want["tokens"][:B]), tag
+                    assert np.array_equal(ids_only[:B].cpu().numpy(), want["tokens"][:B]), tag
+                    assert np.array_equal(m[:B].cpu().numpy().astype(np.float64), want["max"][:B]), tag
+                    assert np.max(np.abs(Z[:B].cpu().numpy() / want["sumexp"][:B] - 1.0)) <= REL, tag
+                    assert np.max(np.abs(p[:B].cpu().numpy() / want["prob"][:B] - 1.0)) <= REL, tag
