@@ -148,6 +148,25 @@ def test_config3_shape_one_step_fp32_selfsalt_with_zipf_spike():
     assert_same_bits(host_bits(x), want)
 
 
+def test_config3_sixteen_of_the_128_decode_steps():
+    """Config 3 over a rotating pool: steps 0, 8, ..., 120 of the 128-step sequence (each its own
+    (256, 151936) fp32 tensor with its Zipf spike and context column), every logit compared."""
+    import os
+
+    dev = require_gpu()
+    threads = min(32, os.cpu_count() or 8)
+    for t in range(0, 128, 8):
+        x = inputs.logits_normal(256, 151936, 4.0, torch.float32, seed=7000 + t, device=dev)
+        inputs.add_zipf_spike_(x, 151936, seed=7500 + t)
+        ctx = inputs.uniform_tokens((256, 1), 151936, seed=8000 + t, device=dev)
+        before = host_bits(x)
+        sbw.sbw_bias_logits(x, ctx, KEY, 0.25, 4.0, sbw.SCHEME_SELFSALT)
+        torch.cuda.synchronize()
+        want = oracle.bias_logits(before, 151936, ctx.cpu().numpy(), KEY, 0.25, 4.0, oracle.SCHEME_SELFSALT,
+                                  threads=threads)
+        assert host_bits(x).tobytes() == want.tobytes(), t
+
+
 def test_consecutive_steps_on_a_side_stream_and_other_keys():
     """Several decode steps enqueued back to back on a non-default stream, 64-bit keys."""
     dev = require_gpu()
