@@ -185,6 +185,19 @@ int sbw_sample_combine(const float *shards, int64_t S, int64_t B, float temperat
                        void *stream);
 
 /*
+ * sbw_bias_sample_shard_ids -- sbw_bias_sample_shard for callers that want the global ids only:
+ * same arguments and summary layout, but the summary carries no statistics (m = -inf, Z = 0), so
+ * the shard takes the ids-only path of sbw_bias_sample (the green test runs only for candidates
+ * that could win).  sbw_sample_combine on such summaries gives the same out_tokens; its m, Z and
+ * p outputs must then be NULL.
+ */
+int sbw_bias_sample_shard_ids(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
+                              int64_t vocab_offset, int64_t row_offset, const int32_t *ctx_tokens,
+                              int ctx_width, uint64_t key, double gamma, float delta, int scheme,
+                              float temperature, uint64_t rng_seed, uint64_t rng_step, float *out_shard,
+                              int32_t *out_tokens, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * sbw_bias_sample_noalloc -- sbw_bias_sample for callers that cannot hand over a workspace.
  * The paper has no counterpart for this call; it exists for deployment.  Some users of this
  * library cannot allocate device memory at all: a logits processor plugged into a serving

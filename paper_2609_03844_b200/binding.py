@@ -32,7 +32,7 @@ EXPORTS = ("sbw_version", "sbw_last_cuda_error", "sbw_bias_logits",
            "sbw_bias_sample_shard", "sbw_sample_combine", "sbw_detect_bits_words", "sbw_detect_bits",
            "sbw_window_z", "sbw_prefix_z", "sbw_detect_unique_workspace_bytes", "sbw_detect_unique",
            "sbw_roc_auc_workspace_bytes", "sbw_roc_auc", "sbw_sample_filtered_workspace_bytes",
-           "sbw_bias_sample_filtered", "sbw_roc_auc_batched")
+           "sbw_bias_sample_filtered", "sbw_roc_auc_batched", "sbw_bias_sample_shard_ids")
 
 _lib = None
 
@@ -90,6 +90,9 @@ def lib() -> ctypes.CDLL:
         L.sbw_bias_sample_shard.restype = i32
         L.sbw_bias_sample_shard.argtypes = [vp, i32, i64, i64, i64, i64, i64, vp, i32, u64, c.c_double,
                                             c.c_float, i32, c.c_float, u64, u64, vp, vp, vp, sz, vp]
+        L.sbw_bias_sample_shard_ids.restype = i32
+        L.sbw_bias_sample_shard_ids.argtypes = [vp, i32, i64, i64, i64, i64, i64, vp, i32, u64, c.c_double,
+                                                c.c_float, i32, c.c_float, u64, u64, vp, vp, vp, sz, vp]
         L.sbw_sample_combine.restype = i32
         L.sbw_sample_combine.argtypes = [vp, i64, i64, c.c_float, vp, vp, vp, vp, vp]
         L.sbw_detect_workspace_bytes.restype = sz
@@ -307,17 +310,19 @@ def sbw_bias_sample_shard(logits: torch.Tensor, ctx_tokens: torch.Tensor, key: i
                           delta: float, scheme: int, temperature: float, rng_seed: int, rng_step: int,
                           out_shard: torch.Tensor, out_tokens: torch.Tensor, workspace: torch.Tensor, *,
                           vocab_offset: int, row_offset: int = 0, V: int | None = None,
-                          stream=None) -> torch.Tensor:
-    """Fused sampling on one vocabulary shard; fills ``out_shard`` ([B, 8] float32) and returns it."""
+                          ids_only: bool = False, stream=None) -> torch.Tensor:
+    """Fused sampling on one vocabulary shard; fills ``out_shard`` ([B, 8] float32) and returns it.
+    ``ids_only`` calls sbw_bias_sample_shard_ids: the summary then serves the ids alone."""
     B, V, ld = _row_layout(logits, V)
     W = _ctx(ctx_tokens, B)
     if out_shard.dtype != torch.float32 or out_shard.numel() != B * 8 or not out_shard.is_contiguous():
         raise TypeError("out_shard must be a contiguous float32 tensor of B * 8 values")
-    rc = lib().sbw_bias_sample_shard(_ptr(logits), _dtype_code(logits), B, V, ld, vocab_offset, row_offset,
-                                     _ptr(ctx_tokens), W, key, gamma, delta, scheme, temperature, rng_seed,
-                                     rng_step, _ptr(out_shard), _ptr(out_tokens), _ptr(workspace),
-                                     workspace.numel() * workspace.element_size(), _stream(stream))
-    _check("sbw_bias_sample_shard", rc)
+    name = "sbw_bias_sample_shard_ids" if ids_only else "sbw_bias_sample_shard"
+    rc = getattr(lib(), name)(_ptr(logits), _dtype_code(logits), B, V, ld, vocab_offset, row_offset,
+                              _ptr(ctx_tokens), W, key, gamma, delta, scheme, temperature, rng_seed,
+                              rng_step, _ptr(out_shard), _ptr(out_tokens), _ptr(workspace),
+                              workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(name, rc)
     return out_shard
 
 

@@ -77,6 +77,7 @@ struct SampleArgs {
     int32_t *out_tokens;
     float *out_max, *out_sumexp, *out_prob;
     float *out_shard;     // [B, 8] or NULL: (m, Z, best score, global id bits, its biased logit, 0, 0, 0)
+    bool shard_ids_only;  // the summary is wanted for the ids alone: m = -inf, Z = 0 in it
     uint32_t row_offset;  // global index of row 0 (enters the Gumbel counter)
     Partial *partials;    // [B * split]
     unsigned *tickets;    // [B], zero before the launch
@@ -215,7 +216,15 @@ __device__ void finish_row_ids(const SampleArgs &a, int64_t row, const Partial *
         const int oid = __shfl_down_sync(0xffffffffu, id, d);
         if (better(os, oid, s, id)) { s = os; id = oid; }
     }
-    if (lane == 0) a.out_tokens[row] = id == INT_MAX ? 0 : id;   // every score was -inf: lowest id
+    if (lane == 0) {
+        if (id == INT_MAX) id = 0;                       // every score was -inf: lowest id
+        a.out_tokens[row] = id;
+        if (a.out_shard) {
+            float4 *o = reinterpret_cast<float4 *>(a.out_shard + row * 8);
+            o[0] = make_float4(-INFINITY, 0.0f, s, __int_as_float(static_cast<int>(a.vocab_offset) + id));
+            o[1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        }
+    }
 }
 
 __device__ void finish_row(const SampleArgs &a, int64_t row, const Partial *parts, int n) {
@@ -651,7 +660,7 @@ int launch_one(SampleArgs &a, int64_t nslot, size_t partial_bytes, cudaStream_t 
 
 template <int DTYPE, int SCHEME>
 int launch(SampleArgs &a, bool vector, int64_t nslot, size_t partial_bytes, float *out_probs, cudaStream_t s) {
-    const bool stats = a.out_max || a.out_sumexp || a.out_prob || a.out_shard || out_probs;
+    const bool stats = a.out_max || a.out_sumexp || a.out_prob || (a.out_shard && !a.shard_ids_only) || out_probs;
     const int rc = stats ? (vector ? launch_one<DTYPE, SCHEME, true, true>(a, nslot, partial_bytes, s)
                                    : launch_one<DTYPE, SCHEME, false, true>(a, nslot, partial_bytes, s))
                          : (vector ? launch_one<DTYPE, SCHEME, true, false>(a, nslot, partial_bytes, s)
@@ -673,7 +682,7 @@ int bias_sample_impl(const void *logits, int dtype, int64_t B, int64_t V, int64_
                      int scheme, float temperature, uint64_t rng_seed, uint64_t rng_step, int32_t *out_tokens,
                      float *out_max, float *out_sumexp, float *out_prob, float *out_probs, void *workspace,
                      size_t workspace_bytes, bool need_full_workspace, cudaStream_t s,
-                     float *out_shard = nullptr, int64_t row_offset = 0) {
+                     float *out_shard = nullptr, int64_t row_offset = 0, bool shard_ids_only = false) {
     if (!valid_common(dtype, ctx_width, gamma, scheme)) return SBW_ERR_INVALID_ARG;
     if (B < 0 || V <= 0 || ld < V || vocab_offset < 0) return SBW_ERR_INVALID_ARG;
     if (!(temperature > 0.0f) || temperature - temperature != 0.0f) return SBW_ERR_INVALID_ARG;
@@ -727,6 +736,7 @@ int bias_sample_impl(const void *logits, int dtype, int64_t B, int64_t V, int64_
     a.out_sumexp = out_sumexp;
     a.out_prob = out_prob;
     a.out_shard = out_shard;
+    a.shard_ids_only = shard_ids_only;
     a.row_offset = static_cast<uint32_t>(row_offset);
     a.partials = ws.partials;
     a.tickets = ws.tickets;
@@ -874,6 +884,19 @@ extern "C" int sbw_bias_sample_shard(const void *logits, int dtype, int64_t B, i
                                  delta, scheme, temperature, rng_seed, rng_step, out_tokens, nullptr, nullptr,
                                  nullptr, nullptr, workspace, workspace_bytes, true,
                                  static_cast<cudaStream_t>(stream), out_shard, row_offset);
+}
+
+extern "C" int sbw_bias_sample_shard_ids(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld,
+                                         int64_t vocab_offset, int64_t row_offset, const int32_t *ctx_tokens,
+                                         int ctx_width, uint64_t key, double gamma, float delta, int scheme,
+                                         float temperature, uint64_t rng_seed, uint64_t rng_step,
+                                         float *out_shard, int32_t *out_tokens, void *workspace,
+                                         size_t workspace_bytes, void *stream) {
+    if (B > 0 && !out_shard) return SBW_ERR_INVALID_ARG;
+    return sbw::bias_sample_impl(logits, dtype, B, V, ld, vocab_offset, ctx_tokens, ctx_width, key, gamma,
+                                 delta, scheme, temperature, rng_seed, rng_step, out_tokens, nullptr, nullptr,
+                                 nullptr, nullptr, workspace, workspace_bytes, true,
+                                 static_cast<cudaStream_t>(stream), out_shard, row_offset, true);
 }
 
 extern "C" int sbw_sample_combine(const float *shards, int64_t S, int64_t B, float temperature,

@@ -35,19 +35,24 @@ def gather_summaries(local: torch.Tensor, group=None) -> torch.Tensor:
 
 def sharded_bias_sample(logits_shard: torch.Tensor, ctx_tokens: torch.Tensor, key: int, gamma: float,
                         delta: float, scheme: int, temperature: float, rng_seed: int, rng_step: int,
-                        vocab_offset: int, workspace: torch.Tensor, group=None, row_offset: int = 0):
+                        vocab_offset: int, workspace: torch.Tensor, group=None, row_offset: int = 0,
+                        ids_only: bool = False):
     """Samples one token per row from logits whose columns are spread over the ranks of ``group``.
     ``logits_shard`` holds this rank's columns, ``vocab_offset`` the global id of its column 0.
-    Returns (global token ids [B] int32, m [B], Z [B], p [B]) -- identical on every rank."""
+    Returns (global token ids [B] int32, m [B], Z [B], p [B]) -- identical on every rank; with
+    ``ids_only`` the shards take the cheaper ids-only path and m, Z, p are returned as None."""
     B = logits_shard.shape[0]
     dev = logits_shard.device
     summary = torch.empty((B, 8), dtype=torch.float32, device=dev)
     local_ids = torch.empty(B, dtype=torch.int32, device=dev)
     binding.sbw_bias_sample_shard(logits_shard, ctx_tokens, key, gamma, delta, scheme, temperature, rng_seed,
                                   rng_step, summary, local_ids, workspace, vocab_offset=vocab_offset,
-                                  row_offset=row_offset)
+                                  row_offset=row_offset, ids_only=ids_only)
     shards = gather_summaries(summary, group)
     tokens = torch.empty(B, dtype=torch.int32, device=dev)
+    if ids_only:
+        binding.sbw_sample_combine(shards, temperature, tokens)
+        return tokens, None, None, None
     m = torch.empty(B, dtype=torch.float32, device=dev)
     Z = torch.empty(B, dtype=torch.float32, device=dev)
     p = torch.empty(B, dtype=torch.float32, device=dev)

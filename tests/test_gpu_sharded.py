@@ -75,3 +75,29 @@ def test_single_rank_helper_and_all_masked_rows():
     torch.cuda.synchronize()
     want = oracle.bias_sample(host_bits(x), V, ctx.cpu().numpy(), KEY, 0.5, 1.0, 0, 0.7, 1, 2)
     assert np.array_equal(tok.cpu().numpy(), want["tokens"]) and tok[1].item() == 0
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("scheme", [sbw.SCHEME_CONTEXT, sbw.SCHEME_SELFSALT])
+@pytest.mark.parametrize("S,B", [(2, 12), (8, 3), (4, 600)])
+def test_ids_only_shards_give_the_same_ids(dtype, scheme, S, B):
+    """Shards that are asked for the ids alone (no statistics in the summary) take the cheaper
+    kernel; the combined ids are those of the unsharded call and of the oracle."""
+    dev = require_gpu()
+    V, tau = 50000, 0.7
+    x = inputs.logits_normal(B, V, 4.0, dtype, seed=1600 + B, device=dev)
+    ctx = inputs.uniform_tokens((B, 1), V, seed=1601, device=dev)
+    ws = torch.empty(sbw.sbw_sample_workspace_bytes(B, V), dtype=torch.uint8, device=dev)
+    summaries = torch.empty((S, B, 8), dtype=torch.float32, device=dev)
+    local = torch.empty(B, dtype=torch.int32, device=dev)
+    for r in range(S):
+        lo, hi = sharded.shard_columns(V, r, S)
+        sbw.sbw_bias_sample_shard(x[:, lo:hi], ctx, KEY, 0.25, 2.0, scheme, tau, 0xC4, 9, summaries[r], local, ws,
+                                  vocab_offset=lo, ids_only=True)
+    tok = torch.empty(B, dtype=torch.int32, device=dev)
+    sbw.sbw_sample_combine(summaries, tau, tok)
+    torch.cuda.synchronize()
+    want = oracle.bias_sample(host_bits(x), V, ctx.cpu().numpy(), KEY, 0.25, 2.0, scheme, tau, 0xC4, 9, threads=8)
+    assert np.array_equal(tok.cpu().numpy(), want["tokens"])
+    s = summaries.cpu().numpy()
+    assert np.isneginf(s[:, :, 0]).all() and (s[:, :, 1] == 0).all()       # no statistics in these summaries
