@@ -30,17 +30,30 @@ def is_stale() -> bool:
 
 
 def build(force: bool = False, verbose: bool = False) -> Path:
-    """Compile every kernel for sm_100a and link libsbw.so.  Needs nvcc, not a GPU."""
+    """Compile every kernel for sm_100a and link libsbw.so.  Needs nvcc, not a GPU.  The sources
+    are compiled to objects side by side (one nvcc per file), then linked."""
     if not force and not is_stale():
         return LIB
-    tmp = LIB.with_suffix(f".{os.getpid()}.tmp")
-    cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared", "-I", str(INCLUDE)]
+    import tempfile
+    from concurrent.futures import ThreadPoolExecutor
+
+    flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+             "-Xcompiler", "-fPIC", "-I", str(INCLUDE)]
     if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += ["-o", str(tmp)] + [str(s) for s in sources()]
-    subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB)
+        flags += ["-Xptxas", "-v"]
+    with tempfile.TemporaryDirectory(prefix="sbw_build_") as tmpdir:
+        def compile_one(src: Path) -> str:
+            obj = str(Path(tmpdir) / (src.stem + ".o"))
+            subprocess.run([_nvcc(), *flags, "-c", str(src), "-o", obj], check=True)
+            return obj
+
+        srcs = sources()
+        with ThreadPoolExecutor(max_workers=min(len(srcs), os.cpu_count() or 4)) as pool:
+            objects = list(pool.map(compile_one, srcs))
+        tmp = LIB.with_suffix(f".{os.getpid()}.tmp")
+        subprocess.run([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-cudart", "shared",
+                        "-o", str(tmp), *objects], check=True)
+        os.replace(tmp, LIB)
     return LIB
 
 
