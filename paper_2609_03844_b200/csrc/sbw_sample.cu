@@ -227,22 +227,46 @@ __device__ void finish_row_ids(const SampleArgs &a, int64_t row, const Partial *
     }
 }
 
+// The loads of a pass are issued eight at a time per lane before any is used.
 __device__ void finish_row(const SampleArgs &a, int64_t row, const Partial *parts, int n) {
+    constexpr int kBatch = 8;
     const int lane = threadIdx.x & 31;
     float m = -INFINITY;
-    for (int i = lane; i < n; i += 32) m = fmaxf(m, __ldcg(&parts[i].m));
+    for (int i0 = lane; i0 < n; i0 += 32 * kBatch) {
+        float pm[kBatch];
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) {
+            const int i = i0 + 32 * k;
+            pm[k] = i < n ? __ldcg(&parts[i].m) : -INFINITY;
+        }
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) m = fmaxf(m, pm[k]);
+    }
     for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
     double Z = 0.0;
     float s = -INFINITY, l = -INFINITY;
     int id = INT_MAX;
-    for (int i = lane; i < n; i += 32) {
+    for (int i0 = lane; i0 < n; i0 += 32 * kBatch) {
         // L2 loads: the partials were written by other SMs during this launch
-        const float4 q0 = __ldcg(reinterpret_cast<const float4 *>(parts + i));
-        const float pl = __ldcg(&parts[i].l);
-        const float pm = q0.x, pz = q0.y, ps = q0.z;
-        const int pid = __float_as_int(q0.w);
-        if (pm > -INFINITY) Z += static_cast<double>(pz * exp2_scaled(pm - m, a.c2_hi, a.c2_lo));
-        if (better(ps, pid, s, id)) { s = ps; id = pid; l = pl; }
+        float4 q[kBatch];
+        float pl[kBatch];
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) {
+            const int i = i0 + 32 * k;
+            q[k] = make_float4(-INFINITY, 0.0f, -INFINITY, __int_as_float(INT_MAX));
+            pl[k] = -INFINITY;
+            if (i < n) {
+                q[k] = __ldcg(reinterpret_cast<const float4 *>(parts + i));
+                pl[k] = __ldcg(&parts[i].l);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) {                  // index order per lane
+            const float pm = q[k].x, pz = q[k].y, ps = q[k].z;
+            const int pid = __float_as_int(q[k].w);
+            if (pm > -INFINITY) Z += static_cast<double>(pz * exp2_scaled(pm - m, a.c2_hi, a.c2_lo));
+            if (better(ps, pid, s, id)) { s = ps; id = pid; l = pl[k]; }
+        }
     }
     for (int d = 16; d > 0; d >>= 1) {
         Z += __shfl_down_sync(0xffffffffu, Z, d);
