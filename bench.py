@@ -540,7 +540,7 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
 
 PROFILE_CASES = ("topk40_fp32_selfsalt", "bias_bf16_context", "bias_bf16_selfsalt", "bias_fp32_context", "bias_fp32_selfsalt",
                  "detect_context", "detect_selfsalt", "sample_bf16_context", "sample_bf16_selfsalt",
-                 "detectunique_context", "filtered_bf16_context", "sampleids_bf16_context", "sampleids_bf16_selfsalt")
+                 "detectunique_context", "filtered_bf16_context", "sampleids_bf16_context", "sampleids_bf16_selfsalt", "filteredtopk_bf16_context")
 
 
 def run_profile_case(name: str, launches: int) -> None:
@@ -568,13 +568,14 @@ def run_profile_case(name: str, launches: int) -> None:
             ws = torch.empty(sbw.sbw_detect_unique_workspace_bytes(N, tokens.numel(), 1024), dtype=torch.uint8,
                              device=dev)
             fn = lambda i: sbw.sbw_detect_unique(tokens, lengths, 1024, KEY, 0.25, scheme, counts, z, ws)  # noqa: E731
-    elif kind == "filtered":
+    elif kind in ("filtered", "filteredtopk"):
         B = 512
         x = inputs.logits_normal(B, V2, 4.0, torch.bfloat16, seed=1, device=dev)
         ctx = inputs.uniform_tokens((B, 1), V2, seed=2, device=dev)
         ids = torch.empty(B, dtype=torch.int32, device=dev)
         ws = torch.empty(sbw.sbw_sample_filtered_workspace_bytes(x.dtype, B, V2), dtype=torch.uint8, device=dev)
-        fn = lambda i: sbw.sbw_bias_sample_filtered(x, ctx, KEY, 0.25, 2.0, scheme, 0.7, 0, 0.8, 0xC4, i, ids, ws)  # noqa: E731
+        top_k, top_p = (50, 0.9) if kind == "filteredtopk" else (0, 0.8)
+        fn = lambda i: sbw.sbw_bias_sample_filtered(x, ctx, KEY, 0.25, 2.0, scheme, 0.7, top_k, top_p, 0xC4, i, ids, ws)  # noqa: E731
     else:
         B, V, dtype = (512, V2, torch.bfloat16) if dt == "bf16" else (256, 151936, torch.float32)
         x = inputs.logits_normal(B, V, 4.0, dtype, seed=1, device=dev)
