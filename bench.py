@@ -505,7 +505,7 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
                     256)
     out["topk40_bf16_selfsalt_B64_V128256"] = {"gelem_s": B2 * V2 / s / 1e9, "ms": s * 1e3}
     del xs, cs
-    # the paper's isolated-benchmark protocol (Appendix B: fresh (B, 151936) logits, 20 warm-up + 200
+    # the paper's isolated-benchmark protocol (Appendix D: fresh (B, 151936) logits, 20 warm-up + 200
     # timed calls, CUDA events, synchronise between calls, p50/p99) on its two full-vocabulary schemes
     # with context width 4 (SBW-4, SBW-ss-V); fp32 logits (the paper does not state its dtype)
     sweep = {}

@@ -312,7 +312,7 @@ int sbw_detect_unique(const int32_t *tokens, const int32_t *lengths, const int64
                       size_t workspace_bytes, void *stream);
 
 /*
- * sbw_roc_auc -- Section 4.4: area under the ROC curve of z-scores as a detector of label 1
+ * sbw_roc_auc -- Section 4.3: area under the ROC curve of z-scores as a detector of label 1
  * (watermarked) against label 0, computed exactly as the pair statistic
  *   AUC = (2 #{z_pos > z_neg} + #{z_pos == z_neg}) / (2 n_pos n_neg),
  * which equals the trapezoid area under the (FPR, TPR) curve swept over every threshold.  NaN

@@ -436,7 +436,7 @@ void sbw_oracle_prefix_z(const uint8_t *green, const int32_t *lengths, const int
     }
 }
 
-/* Section 4.4: area under the ROC curve of the z-score as a detector of label 1 against label 0,
+/* Section 4.3: area under the ROC curve of the z-score as a detector of label 1 against label 0,
  * written as the probability that a watermarked text outscores an unmarked one, ties counting a
  * half (equal to the trapezoid area under the curve swept over all thresholds).  NaN scores are
  * left out of both classes.  stats (nullable) receives {pairs with z_pos > z_neg, pairs with

@@ -114,7 +114,7 @@ void sbw_oracle_detect_unique(const int32_t *tokens, const int32_t *lengths, int
  * per-token array of sbw_oracle_detect_bits. */
 void sbw_oracle_prefix_z(const uint8_t *green, const int32_t *lengths, const int32_t *keep, int64_t N,
                          int ctx_width, double gamma, int32_t *counts, int32_t *T, double *z);
-/* Section 4.4: ROC-AUC of z against binary labels = P(z_pos > z_neg) + P(z_pos == z_neg) / 2 over
+/* Section 4.3: ROC-AUC of z against binary labels = P(z_pos > z_neg) + P(z_pos == z_neg) / 2 over
  * all (positive, negative) pairs.  stats (nullable): {greater, equal, n_pos, n_neg}. */
 double sbw_oracle_roc_auc(const double *z, const uint8_t *labels, int64_t n, uint64_t stats[4], int threads);
 /* Eq. 5 alone. */

@@ -1,4 +1,4 @@
-// sbw_roc_auc: area under the ROC curve of detection scores (Section 4.4 of the paper) as the
+// sbw_roc_auc: area under the ROC curve of detection scores (Section 4.3 of the paper) as the
 // exact pair statistic  AUC = (2 #{z_pos > z_neg} + #{z_pos == z_neg}) / (2 n_pos n_neg).
 //
 // Three kernels.  split_kernel copies the scores of each class into its own dense array (slot

@@ -4,7 +4,7 @@ This module holds input generators only -- no hashing, no thresholds, no bias, n
 so that the CUDA path, the CPU oracle, the tests and the benchmark can all draw the same bytes
 without sharing any of the method's arithmetic.  Everything is a pure function of its seed.
 
-Workload shapes (Appendix B of the paper benchmarks fresh random ``(B, 151936)`` logits; its
+Workload shapes (Appendix D of the paper benchmarks fresh random ``(B, 151936)`` logits; its
 completions are at most 200 tokens long; its batch sweep runs from 1 to 512):
 
 * logits: i.i.d. normal with a given standard deviation, float32 or bfloat16, optionally with

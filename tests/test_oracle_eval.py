@@ -1,5 +1,5 @@
 """Pins for the oracle's evaluation steps around detection: distinct-tuple scoring, truncated
-text, ROC-AUC (Section 4.4).  Each is checked against something that is not the oracle's own
+text, ROC-AUC (Section 4.3).  Each is checked against something that is not the oracle's own
 formula: Python sets, slices fed to the plain detector, scikit-learn, exact rationals, closed forms."""
 from fractions import Fraction
 
