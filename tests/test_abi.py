@@ -101,6 +101,81 @@ def test_argument_validation_happens_on_the_host():
     assert L.sbw_last_cuda_error() == 0
 
 
+def test_argument_validation_of_the_widened_entry_points():
+    """Same for the calls added after the first three: bad arguments come back before any CUDA work."""
+    L = sbw.lib()
+    fake = ctypes.c_void_p(0x1000)
+    INV, UNS, WSP, OK = (binding.SBW_ERR_INVALID_ARG, binding.SBW_ERR_UNSUPPORTED, binding.SBW_ERR_WORKSPACE,
+                         binding.SBW_OK)
+
+    def topk(**kw):
+        a = dict(logits=fake, dtype=0, B=2, V=8, ld=8, off=0, ctx=fake, W=1, gamma=0.25, delta=2.0, scheme=1, k=3)
+        a.update(kw)
+        return L.sbw_bias_logits_topk(a["logits"], a["dtype"], a["B"], a["V"], a["ld"], a["off"], a["ctx"], a["W"], 1,
+                                      a["gamma"], a["delta"], a["scheme"], a["k"], None)
+
+    assert topk(B=0) == OK and topk(delta=0.0) == OK
+    for bad in (dict(k=0), dict(k=-2), dict(gamma=1.0), dict(V=0), dict(ld=4), dict(logits=None), dict(ctx=None),
+                dict(delta=float("nan")), dict(W=9)):
+        assert topk(**bad) == INV, bad
+
+    def filtered(**kw):
+        a = dict(logits=fake, dtype=1, B=2, V=64, ld=64, off=0, ctx=fake, W=1, gamma=0.25, delta=2.0, scheme=0,
+                 tau=0.7, k=0, p=0.8, out=fake, ws=fake, ws_bytes=1 << 20)
+        a.update(kw)
+        return L.sbw_bias_sample_filtered(a["logits"], a["dtype"], a["B"], a["V"], a["ld"], a["off"], a["ctx"],
+                                          a["W"], 1, a["gamma"], a["delta"], a["scheme"], a["tau"], a["k"], a["p"],
+                                          1, 2, a["out"], None, a["ws"], a["ws_bytes"], None)
+
+    assert filtered(B=0) == OK
+    for bad in (dict(p=0.0), dict(p=-1.0), dict(p=float("nan")), dict(k=-1), dict(tau=0.0), dict(gamma=0.0),
+                dict(V=0), dict(ld=8), dict(out=None), dict(logits=None), dict(ctx=None), dict(off=-1)):
+        assert filtered(**bad) == INV, bad
+    assert filtered(V=(1 << 21) + 8, ld=(1 << 21) + 8) == UNS
+    assert filtered(ws=None) == WSP and filtered(ws_bytes=64) == WSP
+    assert L.sbw_sample_filtered_workspace_bytes(1, 2, 64) >= 2 * 64 * 2
+    assert L.sbw_sample_filtered_workspace_bytes(7, 2, 64) == 0
+
+    def unique(**kw):
+        a = dict(tokens=fake, lengths=fake, off=None, N=4, total=40, maxlen=10, W=1, gamma=0.25, scheme=0,
+                 counts=fake, z=fake, ws=fake, ws_bytes=1 << 20)
+        a.update(kw)
+        return L.sbw_detect_unique(a["tokens"], a["lengths"], a["off"], a["N"], a["total"], a["maxlen"], a["W"], 1,
+                                   a["gamma"], a["scheme"], a["counts"], None, a["z"], a["ws"], a["ws_bytes"], None)
+
+    assert unique(N=0) == OK
+    for bad in (dict(gamma=1.0), dict(N=-1), dict(total=-1), dict(maxlen=-1), dict(W=0), dict(scheme=3),
+                dict(lengths=None), dict(counts=None), dict(z=None), dict(tokens=None)):
+        assert unique(**bad) == INV, bad
+    assert unique(ws=None) == WSP and unique(ws_bytes=8) == WSP
+    assert L.sbw_detect_unique_workspace_bytes(4, 40, 5000) >= 16 * 40
+
+    def prefix(**kw):
+        a = dict(bits=fake, lengths=fake, off=fake, keep=fake, N=4, total=40, W=1, gamma=0.25, counts=fake, z=fake)
+        a.update(kw)
+        return L.sbw_prefix_z(a["bits"], a["lengths"], a["off"], a["keep"], a["N"], a["total"], a["W"], a["gamma"],
+                              a["counts"], None, a["z"], None)
+
+    assert prefix(N=0) == OK
+    for bad in (dict(gamma=0.0), dict(W=9), dict(N=-1), dict(bits=None), dict(off=None), dict(keep=None),
+                dict(counts=None), dict(z=None)):
+        assert prefix(**bad) == INV, bad
+
+    def roc(**kw):
+        a = dict(z=fake, labels=fake, n=10, auc=fake, ws=fake, ws_bytes=1 << 20)
+        a.update(kw)
+        return L.sbw_roc_auc(a["z"], a["labels"], a["n"], a["auc"], None, a["ws"], a["ws_bytes"], None)
+
+    for bad in (dict(n=-1), dict(auc=None), dict(z=None), dict(labels=None)):
+        assert roc(**bad) == INV, bad
+    assert roc(n=(1 << 31) + 1, ws_bytes=1 << 40) == UNS
+    assert roc(ws=None) == WSP and roc(ws_bytes=16) == WSP
+    assert L.sbw_roc_auc_batched(fake, fake, fake, 0, fake, None, None) == OK
+    assert L.sbw_roc_auc_batched(fake, fake, None, 3, fake, None, None) == INV
+    assert L.sbw_roc_auc_batched(fake, fake, fake, -1, fake, None, None) == INV
+    assert L.sbw_last_cuda_error() == 0
+
+
 def test_python_binding_type_checks():
     import torch
 
