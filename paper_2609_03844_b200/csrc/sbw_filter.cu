@@ -90,7 +90,7 @@ struct FilterShared {
     unsigned int list_n;
     unsigned int red32[kFilterWarps];
     // what the CTAs of a cluster tell each other about their parts of the row
-    unsigned int part_max, part_floor;
+    unsigned int part_max, part_floor, part_deep;
     unsigned long long part_z;
 };
 
@@ -493,10 +493,13 @@ __device__ __forceinline__ unsigned long long packed_score(const FilterArgs &a, 
 // caller gathers unbiased logits and wants every column that a bias of at most `slack` could lift
 // to the floor.  More than kListCap columns at or above the floor are reported as kListCap + 1.
 // ---------------------------------------------------------------------------------------------
+constexpr int kDeepRank = 480;   // of the kFilterThreads thread maxima: about 1400 columns of an ordinary row
+
 struct Head {
     uint32_t key_m;               // largest code of the row
     unsigned gathered;            // entries in sh.list (unsorted), or kListCap + 1
     unsigned long long z_all;     // total weight of the row (want_z)
+    uint32_t deep_floor;          // a lower floor (the 480th largest thread maximum) for one retry
     bool leave;
 };
 
@@ -521,20 +524,24 @@ __device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &s
     sort_list(sh, kFilterThreads);
     uint32_t key_m = ~static_cast<uint32_t>(sh.list[0]);
     uint32_t floor_code = ~static_cast<uint32_t>(sh.list[(want + CS - 1) / CS - 1]);
+    uint32_t deep_floor = ~static_cast<uint32_t>(sh.list[(kDeepRank + CS - 1) / CS - 1]);
     __syncthreads();
     if constexpr (CS > 1) {
         if (threadIdx.x == 0) {
             sh.part_max = key_m;
             sh.part_floor = floor_code;
+            sh.part_deep = deep_floor;
         }
         cg::this_cluster().sync();
         for (unsigned r = 0; r < CS; ++r) {
             const FilterShared *other = cg::this_cluster().map_shared_rank(&sh, r);
             key_m = max(key_m, other->part_max);
             floor_code = min(floor_code, other->part_floor);
+            deep_floor = min(deep_floor, other->part_deep);
         }
     }
     h.key_m = key_m;
+    h.deep_floor = deep_floor;
     if (slack > 0.0f) {
         const float fl = value_of_code<DTYPE>(floor_code);
         if (fl == fl && fabsf(fl) != __int_as_float(0x7f800000)) {
@@ -686,6 +693,24 @@ __device__ __forceinline__ bool full_row(const FilterArgs &a, FilterShared &sh, 
     int n2 = 0;
     if ((use_k || use_p) && h.gathered <= kListCap)
         n2 = cut_list<DTYPE>(a, sh, static_cast<int>(h.gathered), key_m, use_k, use_p, h.z_all);
+    if (n2 == 0 && use_p && !use_k && h.gathered <= kListCap && h.deep_floor < key_m) {
+        // the nucleus reaches below the floor: one more gather pass with a lower floor (about three
+        // times as many columns) before the radix descent, which costs several passes
+        __syncthreads();
+        if (threadIdx.x == 0) sh.list_n = 0u;
+        __syncthreads();
+        const int32_t deep_key = key_of_code<DTYPE>(h.deep_floor);
+        for_each_key<DTYPE>(row_ptr, V, 0u, vectors_of<DTYPE>(V), [&](uint32_t col, uint32_t, int32_t key) {
+            if (key >= deep_key && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= kListCap) {
+                const unsigned idx = atomicAdd(&sh.list_n, 1u);
+                if (idx < kListCap)
+                    sh.list[idx] = (static_cast<unsigned long long>(key_m - code_of_key<DTYPE>(key)) << 32) | col;
+            }
+        });
+        __syncthreads();
+        const unsigned again = sh.list_n;
+        if (again <= kListCap) n2 = cut_list<DTYPE>(a, sh, static_cast<int>(again), key_m, false, true, h.z_all);
+    }
     if (n2 > 0) {
         sample_list<DTYPE>(a, sh, row, key_m, n2);
         return true;
