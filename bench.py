@@ -157,7 +157,7 @@ def run_reference(args) -> None:
     dt = time.perf_counter() - t0
     value = B2 * V2 * args.steps / dt / 1e9
     line = {"impl": "reference", "metric": "sbw_bias_throughput", "value": value, "unit": "Gelem/s",
-            "n_gpus": 0, "steps": args.steps, "warmup": args.warmup,
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,   # the arm's N; the oracle itself runs on host cores
             "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {**workload_config(), "l2": f"{n_in} host-resident step inputs visited in turn (CPU run)"},
