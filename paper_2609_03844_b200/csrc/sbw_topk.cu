@@ -26,6 +26,9 @@ int bias_logits_impl(void *logits, int dtype, int64_t B, int64_t V, int64_t ld, 
                      const int32_t *ctx_tokens, int ctx_width, uint64_t key, double gamma, float delta,
                      int scheme, cudaStream_t stream);
 
+// Waits of the bulk-copy pipeline that ran out (see topk_stream_kernel); read by sbw_pipeline_timeouts.
+__device__ unsigned long long g_pipeline_timeouts;
+
 namespace {
 
 // CTA size: 1024 threads (one CTA per SM) when there are fewer rows than SMs can take two of,
@@ -249,6 +252,282 @@ topk_kernel(const TopkArgs a) {
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Large batches: the same three steps with the row staged through shared memory by bulk
+// asynchronous copies (cp.async.bulk, completion counted on an mbarrier).  The logits in flight
+// sit in a ring of kStages chunks instead of registers, and one thread keeps the ring full across
+// the steps and across rows: while a row is ranked and biased, the first chunks of the CTA's next
+// row are already on their way.  The order of chunks a CTA consumes is fixed -- per row the
+// prefix, then the whole row -- so producer and consumers only count.
+//
+//   full[s]   completes when the bytes of the chunk in stage s have landed (1 arrival + tx count)
+//   empty[s]  completes when all warps are done with the chunk in stage s (kStreamWarps arrivals)
+//
+// Every wait is bounded (polls and wall time); a wait that runs out marks the CTA dead: it stops
+// issuing copies and waiting, writes nothing more, and the count of such events is readable
+// through sbw_pipeline_timeouts().
+constexpr int kStreamThreads = 512;
+constexpr int kStreamWarps = kStreamThreads / 32;
+constexpr uint32_t kChunkBytes = 16384;
+constexpr int kStages = 4;                              // a power of two
+constexpr uint32_t kWaitPolls = 1u << 24;
+constexpr unsigned long long kWaitNanos = 2000000000ull;
+
+struct StreamShared {
+    alignas(128) unsigned char stage[kStages][kChunkBytes];
+    uint64_t cand[kCap];
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+    uint64_t red[kStreamWarps];
+    uint64_t best;
+    uint32_t max4[kStreamThreads / 4];
+    uint32_t floor_code;
+    unsigned count;
+    unsigned dead;
+};
+
+__device__ __forceinline__ uint32_t shared_address(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t *bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(shared_address(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(shared_address(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(shared_address(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(shared_address(bar)), "r"(parity)
+        : "memory");
+    return ok != 0u;
+}
+__device__ __forceinline__ unsigned long long global_nanos() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Waits for the phase of `bar` with the given parity; false (and the CTA marked dead) when the
+// limits run out.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, StreamShared &sh) {
+    if (mbar_try_wait(bar, parity)) return true;
+    unsigned long long t0 = 0;
+    for (uint32_t n = 1; n < kWaitPolls; ++n) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((n & 1023u) == 0u) {
+            const unsigned long long now = global_nanos();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitNanos) break;
+        }
+    }
+    *reinterpret_cast<volatile unsigned *>(&sh.dead) = 1u;
+    atomicAdd(&g_pipeline_timeouts, 1ull);
+    return false;
+}
+// Source and destination 16-byte aligned, bytes a multiple of 16; this CTA's own shared memory.
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     shared_address(dst)),
+                 "l"(src), "r"(bytes), "r"(shared_address(bar))
+                 : "memory");
+}
+
+// Thread 0's view of the chunk sequence: what to issue next.
+struct Producer {
+    int64_t row;          // row of the next chunk to issue
+    uint32_t w;           // its index within the row's sequence (prefix chunks, then row chunks)
+    uint32_t q;           // its index in the CTA's whole sequence
+};
+
+template <int DTYPE, int SCHEME>
+__global__ void __launch_bounds__(kStreamThreads, 2)
+topk_stream_kernel(const TopkArgs a) {
+    constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
+    constexpr int VEC = 16 / ESIZE;
+    constexpr int kGroups = kStreamThreads / 4;
+    extern __shared__ __align__(128) unsigned char stream_smem[];
+    StreamShared &sh = *reinterpret_cast<StreamShared *>(stream_smem);
+    const uint32_t V = static_cast<uint32_t>(a.V);
+    const uint32_t k = static_cast<uint32_t>(a.k);
+    const uint32_t row_bytes = (V * ESIZE) & ~15u;                       // the part bulk copies can take
+    const uint32_t prefix_bytes = min(row_bytes, static_cast<uint32_t>(kPrefixColumns * ESIZE));
+    const uint32_t chunks_prefix = (prefix_bytes + kChunkBytes - 1) / kChunkBytes;
+    const uint32_t chunks_row = (row_bytes + kChunkBytes - 1) / kChunkBytes;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&sh.full[s], 1u);
+            mbar_init(&sh.empty[s], kStreamWarps);
+        }
+        sh.dead = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    Producer pr{static_cast<int64_t>(blockIdx.x), 0u, 0u};
+    bool dead = false;
+    // thread 0 only: issue the next chunk of the sequence, if there is one
+    auto issue = [&]() {
+        if (pr.row >= a.B) return;
+        const bool in_prefix = pr.w < chunks_prefix;
+        const uint32_t c = in_prefix ? pr.w : pr.w - chunks_prefix;
+        const uint32_t limit = in_prefix ? prefix_bytes : row_bytes;
+        const uint32_t off = c * kChunkBytes;
+        const uint32_t bytes = min(kChunkBytes, limit - off);
+        const uint32_t st = pr.q % kStages;
+        const char *src = static_cast<const char *>(a.logits) + pr.row * a.ld * ESIZE + off;
+        mbar_expect_tx(&sh.full[st], bytes);
+        bulk_load(sh.stage[st], src, bytes, &sh.full[st]);
+        pr.q += 1;
+        pr.w += 1;
+        if (pr.w == chunks_prefix + chunks_row) {
+            pr.w = 0;
+            pr.row += gridDim.x;
+        }
+    };
+    if (threadIdx.x == 0)
+        for (int s = 0; s < kStages; ++s) issue();
+
+    uint32_t q = 0;     // the chunk this thread consumes next
+    // Consumes `nchunks` chunks covering `limit` bytes from the start of the row; f(column, code).
+    auto consume = [&](uint32_t nchunks, uint32_t limit, auto f) {
+        for (uint32_t c = 0; c < nchunks; ++c, ++q) {
+            const uint32_t st = q % kStages;
+            if (threadIdx.x == 0 && q > 0 && !dead && pr.row < a.B) {
+                // the stage of the previous chunk is refilled once every warp has left it
+                const uint32_t qp = q - 1;
+                if (mbar_wait(&sh.empty[qp % kStages], (qp / kStages) & 1u, sh)) issue();
+                else dead = true;
+            }
+            if (!dead && *reinterpret_cast<volatile unsigned *>(&sh.dead)) dead = true;
+            if (!dead && !mbar_wait(&sh.full[st], (q / kStages) & 1u, sh)) dead = true;
+            if (!dead) {
+                const uint32_t off = c * kChunkBytes;
+                const uint32_t nvec = min(kChunkBytes, limit - off) / 16u;
+                const uint4 *src = reinterpret_cast<const uint4 *>(sh.stage[st]);
+                for (uint32_t j = threadIdx.x; j < nvec; j += kStreamThreads) {
+                    const uint4 w = src[j];
+                    const uint32_t *e = reinterpret_cast<const uint32_t *>(&w);
+                    const uint32_t col0 = (off / 16u + j) * VEC;
+#pragma unroll
+                    for (int i = 0; i < VEC; ++i) {
+                        uint32_t bits;
+                        if constexpr (DTYPE == SBW_DTYPE_F32) bits = e[i];
+                        else bits = (i & 1) ? (e[i >> 1] & 0xffff0000u) : (e[i >> 1] << 16);
+                        f(col0 + i, order_code(bits));
+                    }
+                }
+            }
+            __syncwarp();
+            if ((threadIdx.x & 31) == 0) mbar_arrive(&sh.empty[st]);
+        }
+    };
+
+    for (int64_t row = blockIdx.x; row < a.B; row += gridDim.x) {
+        char *row_ptr = static_cast<char *>(a.logits) + row * a.ld * ESIZE;
+
+        // 1. lower bound of the k-th largest code from the prefix
+        uint32_t mx = 0;
+        consume(chunks_prefix, prefix_bytes, [&](uint32_t, uint32_t code) { mx = max(mx, code); });
+        mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        if ((threadIdx.x & 3) == 0) sh.max4[threadIdx.x >> 2] = mx;
+        if (threadIdx.x == 0) {
+            sh.floor_code = 0;
+            sh.count = 0;
+        }
+        __syncthreads();
+        if (threadIdx.x < kGroups) {
+            const uint32_t mine = sh.max4[threadIdx.x];
+            uint32_t rank = 0;
+            for (int u = 0; u < kGroups; ++u) {
+                const uint32_t o = sh.max4[u];
+                rank += (o > mine || (o == mine && u < static_cast<int>(threadIdx.x))) ? 1u : 0u;
+            }
+            if (rank == k - 1) sh.floor_code = mine;       // the launch guarantees k <= kGroups
+        }
+        __syncthreads();
+        const uint32_t floor_code = sh.floor_code;
+
+        // 2. candidates: every column that reaches the bound
+        auto push = [&](uint32_t col, uint32_t code) {
+            if (code >= floor_code) {
+                const unsigned pos = atomicAdd(&sh.count, 1u);
+                if (pos < kCap) sh.cand[pos] = composite(code, col);
+            }
+        };
+        consume(chunks_row, row_bytes, push);
+        for (uint32_t c = row_bytes / ESIZE + threadIdx.x; c < V; c += kStreamThreads) {   // ragged end of the row
+            uint32_t bits;
+            if constexpr (DTYPE == SBW_DTYPE_F32) bits = reinterpret_cast<const uint32_t *>(row_ptr)[c];
+            else bits = static_cast<uint32_t>(reinterpret_cast<const uint16_t *>(row_ptr)[c]) << 16;
+            push(c, order_code(bits));
+        }
+        __syncthreads();
+        const unsigned n = sh.count;
+        const bool row_dead = *reinterpret_cast<volatile unsigned *>(&sh.dead) != 0u;
+
+        if (row_dead) {
+            // a wait ran out somewhere in this CTA: the candidates cannot be trusted, nothing is written
+        } else if (n <= kCap) {
+            // 3. rank by counting, bias ranks below k
+            for (unsigned e = threadIdx.x; e < n; e += kStreamThreads) {
+                const uint64_t mine = sh.cand[e];
+                uint32_t rank = 0;
+                for (unsigned u = 0; u < n; ++u) rank += sh.cand[u] > mine ? 1u : 0u;
+                if (rank < k) bias_column<DTYPE, SCHEME>(a, row, row_ptr, 0xFFFFFFFFu - static_cast<uint32_t>(mine));
+            }
+        } else {
+            // fallback as in topk_kernel, on the row in global memory
+            uint64_t prev = 0;
+            const uint32_t rounds = k < V ? k : V;
+            for (uint32_t r = 0; r < rounds; ++r) {
+                uint64_t best = 0;
+                for_each_code<DTYPE, kStreamThreads>(row_ptr, 0u, V, true, [&](uint32_t col, uint32_t code) {
+                    const uint64_t c = composite(code, col);
+                    if ((r == 0 || c < prev) && c > best) best = c;
+                });
+                prev = block_max_u64<kStreamWarps>(best, sh.red, &sh.best);
+            }
+            const uint64_t kth = prev;
+            for_each_code<DTYPE, kStreamThreads>(row_ptr, 0u, V, true, [&](uint32_t col, uint32_t code) {
+                if (composite(code, col) >= kth) bias_column<DTYPE, SCHEME>(a, row, row_ptr, col);
+            });
+        }
+        __syncthreads();             // shared scratch is reused by the next row
+    }
+
+    // Copies that were issued are all consumed above unless the CTA went dead; then wait, within
+    // the same limits, for the stages that may still be written before the shared memory is given up.
+    if (threadIdx.x == 0 && dead) {
+        for (uint32_t back = 1; back <= static_cast<uint32_t>(kStages) && back <= pr.q; ++back) {
+            const uint32_t qi = pr.q - back;
+            mbar_wait(&sh.full[qi % kStages], (qi / kStages) & 1u, sh);
+        }
+    }
+}
+
+template <int DTYPE, int SCHEME>
+cudaError_t launch_stream(const TopkArgs &a, unsigned grid, cudaStream_t s) {
+    static const cudaError_t configured = cudaFuncSetAttribute(
+        topk_stream_kernel<DTYPE, SCHEME>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        static_cast<int>(sizeof(StreamShared)));
+    if (configured != cudaSuccess) return configured;
+    topk_stream_kernel<DTYPE, SCHEME><<<grid, kStreamThreads, sizeof(StreamShared), s>>>(a);
+    return cudaSuccess;
+}
+
 template <int DTYPE, int SCHEME>
 cudaError_t launch_cluster(const TopkArgs &a, int cs, cudaStream_t s) {
     cudaLaunchConfig_t cfg = {};
@@ -284,7 +563,12 @@ int launch(const TopkArgs &a, cudaStream_t s) {
         SBW_CUDA_TRY((launch_cluster<DTYPE, SCHEME>(a, cs, s)));
     } else if (a.B > di.sm_count && a.k <= 128) {
         const unsigned grid = static_cast<unsigned>(a.B < cap ? a.B : cap);
-        topk_kernel<DTYPE, SCHEME, 512, 1><<<grid, 512, 0, s>>>(a);
+        const int esize = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
+        // aligned rows of ordinary width go through the bulk-copy pipeline
+        if (a.vector && a.V >= 4096 && a.V * esize < (int64_t(1) << 31))
+            SBW_CUDA_TRY((launch_stream<DTYPE, SCHEME>(a, grid, s)));
+        else
+            topk_kernel<DTYPE, SCHEME, 512, 1><<<grid, 512, 0, s>>>(a);
     } else {
         const unsigned grid = static_cast<unsigned>(a.B < di.sm_count ? a.B : di.sm_count);
         topk_kernel<DTYPE, SCHEME, 1024, 1><<<grid, 1024, 0, s>>>(a);
@@ -332,4 +616,11 @@ extern "C" int sbw_bias_logits_topk(void *logits, int dtype, int64_t B, int64_t 
                                             : launch<SBW_DTYPE_F32, SBW_SCHEME_SELFSALT>(a, s);
     return scheme == SBW_SCHEME_CONTEXT ? launch<SBW_DTYPE_BF16, SBW_SCHEME_CONTEXT>(a, s)
                                         : launch<SBW_DTYPE_BF16, SBW_SCHEME_SELFSALT>(a, s);
+}
+
+extern "C" int sbw_pipeline_timeouts(unsigned long long *host_count) {
+    using namespace sbw;
+    if (!host_count) return SBW_ERR_INVALID_ARG;
+    SBW_CUDA_TRY(cudaMemcpyFromSymbol(host_count, g_pipeline_timeouts, sizeof(unsigned long long)));
+    return SBW_OK;
 }
