@@ -14,6 +14,7 @@
 // If the list overflows (rows of equal values, k > 256) the CTA falls back to k rounds of "largest
 // composite below the previous one", a block reduction each, and one pass that biases every
 // column at or above the k-th composite: slow, but it needs no assumption about the data.
+#include <algorithm>
 #include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
@@ -48,6 +49,9 @@ struct TopkArgs {
     Weyl weyl;
     int k;
     bool vector;       // rows start on 16-byte boundaries
+    // bulk-copy kernel only: bytes of a row that bulk copies take (a multiple of 16), bytes of
+    // the prefix pass, and their chunk counts
+    uint32_t row_bytes, prefix_bytes, chunks_row, chunks_prefix;
 };
 
 __device__ __forceinline__ uint32_t order_code(uint32_t bits) {
@@ -268,8 +272,18 @@ topk_kernel(const TopkArgs a) {
 // through sbw_pipeline_timeouts().
 constexpr int kStreamThreads = 512;
 constexpr int kStreamWarps = kStreamThreads / 32;
-constexpr uint32_t kChunkBytes = 16384;
-constexpr int kStages = 4;                              // a power of two
+#ifndef SBW_TOPK_CHUNK
+#define SBW_TOPK_CHUNK 32768
+#endif
+#ifndef SBW_TOPK_STAGES
+#define SBW_TOPK_STAGES 2
+#endif
+constexpr uint32_t kChunkBytes = SBW_TOPK_CHUNK;
+constexpr int kStages = SBW_TOPK_STAGES;                // a power of two
+#ifndef SBW_TOPK_LAG
+#define SBW_TOPK_LAG 1
+#endif
+constexpr uint32_t kRefillLag = SBW_TOPK_LAG;           // 1 <= lag < kStages
 constexpr uint32_t kWaitPolls = 1u << 24;
 constexpr unsigned long long kWaitNanos = 2000000000ull;
 
@@ -284,6 +298,9 @@ struct StreamShared {
     uint32_t floor_code;
     unsigned count;
     unsigned dead;
+    int64_t next_row;      // thread 0: the next chunk to issue is chunk next_w of this row's sequence
+    uint32_t next_w;       //   (prefix chunks, then row chunks),
+    uint32_t next_q;       //   chunk next_q of the CTA's whole sequence
 };
 
 __device__ __forceinline__ uint32_t shared_address(const void *p) {
@@ -342,27 +359,107 @@ __device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t b
                  : "memory");
 }
 
-// Thread 0's view of the chunk sequence: what to issue next.
-struct Producer {
-    int64_t row;          // row of the next chunk to issue
-    uint32_t w;           // its index within the row's sequence (prefix chunks, then row chunks)
-    uint32_t q;           // its index in the CTA's whole sequence
-};
+// Thread 0: issue the next chunk of the CTA's sequence, if there is one.  Its position in the
+// sequence lives in shared memory (sh.next_*): one thread uses it once per chunk.
+template <int ESIZE>
+__device__ __forceinline__ void issue_chunk(const TopkArgs &a, StreamShared &sh) {
+    const int64_t row = sh.next_row;
+    if (row >= a.B) return;
+    const uint32_t w = sh.next_w, q = sh.next_q;
+    const bool in_prefix = w < a.chunks_prefix;
+    const uint32_t c = in_prefix ? w : w - a.chunks_prefix;
+    const uint32_t limit = in_prefix ? a.prefix_bytes : a.row_bytes;
+    const uint32_t off = c * kChunkBytes;
+    const uint32_t bytes = min(kChunkBytes, limit - off);
+    const uint32_t st = q % kStages;
+    const char *src = static_cast<const char *>(a.logits) + row * a.ld * ESIZE + off;
+    mbar_expect_tx(&sh.full[st], bytes);
+    bulk_load(sh.stage[st], src, bytes, &sh.full[st]);
+    sh.next_q = q + 1;
+    if (w + 1 == a.chunks_prefix + a.chunks_row) {
+        sh.next_w = 0;
+        sh.next_row = row + gridDim.x;
+    } else {
+        sh.next_w = w + 1;
+    }
+}
+
+// Order codes of the bulk-copy kernel.  fp32: order_code of the bits.  bf16: the 16-bit analogue,
+// bits ^ 0xffff for negative values and bits ^ 0x8000 otherwise, computed for both halves of a word
+// at once (a byte permute in sign-replication mode gives each half's sign mask).
+__device__ __forceinline__ uint32_t packed_codes(uint32_t w) {
+    uint32_t sign;   // 0xffff in each half whose value is negative (selector bit 3: replicate the byte's msb)
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(sign) : "r"(w), "r"(0u), "r"(0xBB99u));
+    return w ^ (sign | 0x80008000u);
+}
+template <int DTYPE>
+__device__ __forceinline__ uint32_t vector_max_code(const uint4 &w) {
+    if constexpr (DTYPE == SBW_DTYPE_F32) {
+        return max(max(order_code(w.x), order_code(w.y)), max(order_code(w.z), order_code(w.w)));
+    } else {
+        const uint32_t m = __vmaxu2(__vmaxu2(packed_codes(w.x), packed_codes(w.y)),
+                                    __vmaxu2(packed_codes(w.z), packed_codes(w.w)));
+        return max(m >> 16, m & 0xffffu);
+    }
+}
+template <int DTYPE>
+__device__ __forceinline__ uint32_t element_code(const uint4 &w, int i) {
+    const uint32_t *e = reinterpret_cast<const uint32_t *>(&w);
+    if constexpr (DTYPE == SBW_DTYPE_F32) return order_code(e[i]);
+    else return (packed_codes(e[i >> 1]) >> (16 * (i & 1))) & 0xffffu;
+}
+
+// Consumes `nchunks` chunks covering `limit` bytes from the start of the row; f(first column,
+// vector) for every 16-byte vector, each thread taking every kStreamThreads-th.
+template <int DTYPE, typename F>
+__device__ __forceinline__ void consume_chunks(const TopkArgs &a, StreamShared &sh, uint32_t &q_next, bool &dead,
+                                               uint32_t nchunks, uint32_t limit, F f) {
+    constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
+    constexpr int VEC = 16 / ESIZE;
+    constexpr uint32_t kChunkVectors = kChunkBytes / 16u;
+    constexpr int kPer = kChunkVectors / kStreamThreads;
+    for (uint32_t c = 0; c < nchunks; ++c) {
+        const uint32_t q = q_next;
+        const uint32_t st = q % kStages;
+        if (threadIdx.x == 0 && q >= kRefillLag && !dead && sh.next_row < a.B) {
+            // a stage is refilled once every warp has left it
+            const uint32_t qp = q - kRefillLag;
+            if (mbar_wait(&sh.empty[qp % kStages], (qp / kStages) & 1u, sh)) issue_chunk<ESIZE>(a, sh);
+            else dead = true;
+        }
+        if (!dead && !mbar_wait(&sh.full[st], (q / kStages) & 1u, sh)) dead = true;
+        if (!dead) {
+            const uint32_t off = c * kChunkBytes;
+            const uint32_t nvec = min(kChunkBytes, limit - off) / 16u;
+            const uint4 *src = reinterpret_cast<const uint4 *>(sh.stage[st]);
+            const uint32_t vec0 = off / 16u;
+            if (nvec == kChunkVectors) {
+                uint4 w[kPer];
+#pragma unroll
+                for (int u = 0; u < kPer; ++u) w[u] = src[threadIdx.x + u * kStreamThreads];
+#pragma unroll
+                for (int u = 0; u < kPer; ++u) f((vec0 + threadIdx.x + u * kStreamThreads) * VEC, w[u]);
+            } else {
+                for (uint32_t j = threadIdx.x; j < nvec; j += kStreamThreads) f((vec0 + j) * VEC, src[j]);
+            }
+        }
+        __syncwarp();
+        if ((threadIdx.x & 31) == 0) mbar_arrive(&sh.empty[st]);
+        q_next = q + 1;
+    }
+}
 
 template <int DTYPE, int SCHEME>
 __global__ void __launch_bounds__(kStreamThreads, 2)
 topk_stream_kernel(const TopkArgs a) {
     constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
-    constexpr int VEC = 16 / ESIZE;
     constexpr int kGroups = kStreamThreads / 4;
     extern __shared__ __align__(128) unsigned char stream_smem[];
     StreamShared &sh = *reinterpret_cast<StreamShared *>(stream_smem);
     const uint32_t V = static_cast<uint32_t>(a.V);
     const uint32_t k = static_cast<uint32_t>(a.k);
-    const uint32_t row_bytes = (V * ESIZE) & ~15u;                       // the part bulk copies can take
-    const uint32_t prefix_bytes = min(row_bytes, static_cast<uint32_t>(kPrefixColumns * ESIZE));
-    const uint32_t chunks_prefix = (prefix_bytes + kChunkBytes - 1) / kChunkBytes;
-    const uint32_t chunks_row = (row_bytes + kChunkBytes - 1) / kChunkBytes;
+    uint32_t q_next = 0;     // the chunk of the CTA's sequence this thread consumes next
+    bool dead = false;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -370,76 +467,23 @@ topk_stream_kernel(const TopkArgs a) {
             mbar_init(&sh.empty[s], kStreamWarps);
         }
         sh.dead = 0u;
+        sh.next_row = blockIdx.x;
+        sh.next_w = 0u;
+        sh.next_q = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
-
-    Producer pr{static_cast<int64_t>(blockIdx.x), 0u, 0u};
-    bool dead = false;
-    // thread 0 only: issue the next chunk of the sequence, if there is one
-    auto issue = [&]() {
-        if (pr.row >= a.B) return;
-        const bool in_prefix = pr.w < chunks_prefix;
-        const uint32_t c = in_prefix ? pr.w : pr.w - chunks_prefix;
-        const uint32_t limit = in_prefix ? prefix_bytes : row_bytes;
-        const uint32_t off = c * kChunkBytes;
-        const uint32_t bytes = min(kChunkBytes, limit - off);
-        const uint32_t st = pr.q % kStages;
-        const char *src = static_cast<const char *>(a.logits) + pr.row * a.ld * ESIZE + off;
-        mbar_expect_tx(&sh.full[st], bytes);
-        bulk_load(sh.stage[st], src, bytes, &sh.full[st]);
-        pr.q += 1;
-        pr.w += 1;
-        if (pr.w == chunks_prefix + chunks_row) {
-            pr.w = 0;
-            pr.row += gridDim.x;
-        }
-    };
     if (threadIdx.x == 0)
-        for (int s = 0; s < kStages; ++s) issue();
-
-    uint32_t q = 0;     // the chunk this thread consumes next
-    // Consumes `nchunks` chunks covering `limit` bytes from the start of the row; f(column, code).
-    auto consume = [&](uint32_t nchunks, uint32_t limit, auto f) {
-        for (uint32_t c = 0; c < nchunks; ++c, ++q) {
-            const uint32_t st = q % kStages;
-            if (threadIdx.x == 0 && q > 0 && !dead && pr.row < a.B) {
-                // the stage of the previous chunk is refilled once every warp has left it
-                const uint32_t qp = q - 1;
-                if (mbar_wait(&sh.empty[qp % kStages], (qp / kStages) & 1u, sh)) issue();
-                else dead = true;
-            }
-            if (!dead && *reinterpret_cast<volatile unsigned *>(&sh.dead)) dead = true;
-            if (!dead && !mbar_wait(&sh.full[st], (q / kStages) & 1u, sh)) dead = true;
-            if (!dead) {
-                const uint32_t off = c * kChunkBytes;
-                const uint32_t nvec = min(kChunkBytes, limit - off) / 16u;
-                const uint4 *src = reinterpret_cast<const uint4 *>(sh.stage[st]);
-                for (uint32_t j = threadIdx.x; j < nvec; j += kStreamThreads) {
-                    const uint4 w = src[j];
-                    const uint32_t *e = reinterpret_cast<const uint32_t *>(&w);
-                    const uint32_t col0 = (off / 16u + j) * VEC;
-#pragma unroll
-                    for (int i = 0; i < VEC; ++i) {
-                        uint32_t bits;
-                        if constexpr (DTYPE == SBW_DTYPE_F32) bits = e[i];
-                        else bits = (i & 1) ? (e[i >> 1] & 0xffff0000u) : (e[i >> 1] << 16);
-                        f(col0 + i, order_code(bits));
-                    }
-                }
-            }
-            __syncwarp();
-            if ((threadIdx.x & 31) == 0) mbar_arrive(&sh.empty[st]);
-        }
-    };
+        for (int s = 0; s < kStages; ++s) issue_chunk<ESIZE>(a, sh);
 
     for (int64_t row = blockIdx.x; row < a.B; row += gridDim.x) {
         char *row_ptr = static_cast<char *>(a.logits) + row * a.ld * ESIZE;
 
         // 1. lower bound of the k-th largest code from the prefix
         uint32_t mx = 0;
-        consume(chunks_prefix, prefix_bytes, [&](uint32_t, uint32_t code) { mx = max(mx, code); });
+        consume_chunks<DTYPE>(a, sh, q_next, dead, a.chunks_prefix, a.prefix_bytes,
+                              [&](uint32_t, const uint4 &w) { mx = max(mx, vector_max_code<DTYPE>(w)); });
         mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
         mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
         if ((threadIdx.x & 3) == 0) sh.max4[threadIdx.x >> 2] = mx;
@@ -467,12 +511,16 @@ topk_stream_kernel(const TopkArgs a) {
                 if (pos < kCap) sh.cand[pos] = composite(code, col);
             }
         };
-        consume(chunks_row, row_bytes, push);
-        for (uint32_t c = row_bytes / ESIZE + threadIdx.x; c < V; c += kStreamThreads) {   // ragged end of the row
-            uint32_t bits;
-            if constexpr (DTYPE == SBW_DTYPE_F32) bits = reinterpret_cast<const uint32_t *>(row_ptr)[c];
-            else bits = static_cast<uint32_t>(reinterpret_cast<const uint16_t *>(row_ptr)[c]) << 16;
-            push(c, order_code(bits));
+        consume_chunks<DTYPE>(a, sh, q_next, dead, a.chunks_row, a.row_bytes, [&](uint32_t col0, const uint4 &w) {
+            if (vector_max_code<DTYPE>(w) < floor_code) return;       // the common case: one compare per vector
+#pragma unroll
+            for (int i = 0; i < 16 / ESIZE; ++i) push(col0 + i, element_code<DTYPE>(w, i));
+        });
+        for (uint32_t c = a.row_bytes / ESIZE + threadIdx.x; c < V; c += kStreamThreads) {   // ragged end of the row
+            uint32_t code;
+            if constexpr (DTYPE == SBW_DTYPE_F32) code = order_code(reinterpret_cast<const uint32_t *>(row_ptr)[c]);
+            else code = packed_codes(reinterpret_cast<const uint16_t *>(row_ptr)[c]) & 0xffffu;
+            push(c, code);
         }
         __syncthreads();
         const unsigned n = sh.count;
@@ -511,8 +559,9 @@ topk_stream_kernel(const TopkArgs a) {
     // Copies that were issued are all consumed above unless the CTA went dead; then wait, within
     // the same limits, for the stages that may still be written before the shared memory is given up.
     if (threadIdx.x == 0 && dead) {
-        for (uint32_t back = 1; back <= static_cast<uint32_t>(kStages) && back <= pr.q; ++back) {
-            const uint32_t qi = pr.q - back;
+        const uint32_t issued = sh.next_q;
+        for (uint32_t back = 1; back <= static_cast<uint32_t>(kStages) && back <= issued; ++back) {
+            const uint32_t qi = issued - back;
             mbar_wait(&sh.full[qi % kStages], (qi / kStages) & 1u, sh);
         }
     }
@@ -520,9 +569,15 @@ topk_stream_kernel(const TopkArgs a) {
 
 template <int DTYPE, int SCHEME>
 cudaError_t launch_stream(const TopkArgs &a, unsigned grid, cudaStream_t s) {
-    static const cudaError_t configured = cudaFuncSetAttribute(
-        topk_stream_kernel<DTYPE, SCHEME>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-        static_cast<int>(sizeof(StreamShared)));
+    // two CTAs of this size per SM need most of the SM's memory as shared memory
+    static const cudaError_t configured = [] {
+        const cudaError_t e = cudaFuncSetAttribute(topk_stream_kernel<DTYPE, SCHEME>,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   static_cast<int>(sizeof(StreamShared)));
+        if (e != cudaSuccess) return e;
+        return cudaFuncSetAttribute(topk_stream_kernel<DTYPE, SCHEME>,
+                                    cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    }();
     if (configured != cudaSuccess) return configured;
     topk_stream_kernel<DTYPE, SCHEME><<<grid, kStreamThreads, sizeof(StreamShared), s>>>(a);
     return cudaSuccess;
@@ -565,8 +620,14 @@ int launch(const TopkArgs &a, cudaStream_t s) {
         const unsigned grid = static_cast<unsigned>(a.B < cap ? a.B : cap);
         const int esize = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
         // aligned rows of ordinary width go through the bulk-copy pipeline
-        if (a.vector && a.V >= 4096 && a.V * esize < (int64_t(1) << 31))
-            SBW_CUDA_TRY((launch_stream<DTYPE, SCHEME>(a, grid, s)));
+        if (a.vector && a.V >= 4096 && a.V * esize < (int64_t(1) << 31)) {
+            TopkArgs b = a;
+            b.row_bytes = static_cast<uint32_t>(a.V * esize) & ~15u;
+            b.prefix_bytes = std::min<uint32_t>(b.row_bytes, kPrefixColumns * esize);
+            b.chunks_row = (b.row_bytes + kChunkBytes - 1) / kChunkBytes;
+            b.chunks_prefix = (b.prefix_bytes + kChunkBytes - 1) / kChunkBytes;
+            SBW_CUDA_TRY((launch_stream<DTYPE, SCHEME>(b, grid, s)));
+        }
         else
             topk_kernel<DTYPE, SCHEME, 512, 1><<<grid, 512, 0, s>>>(a);
     } else {
@@ -609,6 +670,7 @@ extern "C" int sbw_bias_logits_topk(void *logits, int dtype, int64_t B, int64_t 
     a.k = static_cast<int>(top_k);
     const int esize = dtype == SBW_DTYPE_F32 ? 4 : 2;
     a.vector = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && ((ld * esize) % 16 == 0);
+    a.row_bytes = a.prefix_bytes = a.chunks_row = a.chunks_prefix = 0u;
     if (a.delta == 0.0f) return SBW_OK;   // the paper's delta = 0 control: no bit changes
 
     if (dtype == SBW_DTYPE_F32)
