@@ -9,7 +9,7 @@
 //      largest value L is a lower bound of the row's k-th largest logit (k distinct columns reach
 //      it), and it is known after a fifth of the row.
 //   2. One pass over the whole row: columns with code >= L -- a few hundred for ordinary logits --
-//      go into a shared-memory candidate list.  The common path is one compare per logit.
+//      go into a shared-memory candidate list.  The common path is one compare per 16-byte vector.
 //   3. Candidates are ranked by counting larger composites; ranks below k are hashed and biased.
 // If the list overflows (rows of equal values, k > 256) the CTA falls back to k rounds of "largest
 // composite below the previous one", a block reduction each, and one pass that biases every
@@ -102,6 +102,67 @@ __device__ __forceinline__ void for_each_code(const char *row_ptr, uint32_t begi
     }
 }
 
+// Order codes of the fast paths (steps 1 to 3).  fp32: order_code of the bits.  bf16: the 16-bit analogue,
+// bits ^ 0xffff for negative values and bits ^ 0x8000 otherwise, computed for both halves of a word
+// at once (a byte permute in sign-replication mode gives each half's sign mask).
+__device__ __forceinline__ uint32_t packed_codes(uint32_t w) {
+    uint32_t sign;   // 0xffff in each half whose value is negative (selector bit 3: replicate the byte's msb)
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(sign) : "r"(w), "r"(0u), "r"(0xBB99u));
+    return w ^ (sign | 0x80008000u);
+}
+template <int DTYPE>
+__device__ __forceinline__ uint32_t vector_max_code(const uint4 &w) {
+    if constexpr (DTYPE == SBW_DTYPE_F32) {
+        return max(max(order_code(w.x), order_code(w.y)), max(order_code(w.z), order_code(w.w)));
+    } else {
+        const uint32_t m = __vmaxu2(__vmaxu2(packed_codes(w.x), packed_codes(w.y)),
+                                    __vmaxu2(packed_codes(w.z), packed_codes(w.w)));
+        return max(m >> 16, m & 0xffffu);
+    }
+}
+template <int DTYPE>
+__device__ __forceinline__ uint32_t element_code(const uint4 &w, int i) {
+    const uint32_t *e = reinterpret_cast<const uint32_t *>(&w);
+    if constexpr (DTYPE == SBW_DTYPE_F32) return order_code(e[i]);
+    else return (packed_codes(e[i >> 1]) >> (16 * (i & 1))) & 0xffffu;
+}
+
+template <int DTYPE>
+__device__ __forceinline__ uint32_t scalar_code(const char *row_ptr, uint32_t col) {
+    if constexpr (DTYPE == SBW_DTYPE_F32) return order_code(reinterpret_cast<const uint32_t *>(row_ptr)[col]);
+    else return packed_codes(reinterpret_cast<const uint16_t *>(row_ptr)[col]) & 0xffffu;
+}
+
+// Calls fvec(first column, vector) for the aligned 16-byte vectors of the columns [begin, end) that
+// this thread owns and fone(column, code) for the columns left over (all of them when the rows
+// are not aligned); begin is a multiple of 8 columns.
+template <int DTYPE, int kTopkThreads, typename FV, typename F1>
+__device__ __forceinline__ void for_each_vector(const char *row_ptr, uint32_t begin, uint32_t end, bool vector,
+                                                FV fvec, F1 fone) {
+    constexpr int VEC = DTYPE == SBW_DTYPE_F32 ? 4 : 8;
+    uint32_t done = begin;
+    if (vector) {
+        const uint32_t nfull = end / VEC;
+        constexpr int kInFlight = 4;   // independent 128-bit loads per thread before the first use
+        for (uint32_t j0 = begin / VEC + threadIdx.x; j0 < nfull; j0 += kInFlight * kTopkThreads) {
+            uint4 w[kInFlight];
+#pragma unroll
+            for (int u = 0; u < kInFlight; ++u) {
+                const uint32_t j = j0 + u * kTopkThreads;
+                // plain loads: the row is written later by this kernel
+                w[u] = j < nfull ? reinterpret_cast<const uint4 *>(row_ptr)[j] : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int u = 0; u < kInFlight; ++u) {
+                const uint32_t j = j0 + u * kTopkThreads;
+                if (j < nfull) fvec(j * VEC, w[u]);
+            }
+        }
+        done = max(begin, nfull * VEC);
+    }
+    for (uint32_t c = done + threadIdx.x; c < end; c += kTopkThreads) fone(c, scalar_code<DTYPE>(row_ptr, c));
+}
+
 // Eq. 1 + Eq. 2 on one chosen column.
 template <int DTYPE, int SCHEME>
 __device__ __noinline__ void bias_column(const TopkArgs &a, int64_t row, char *row_ptr, uint32_t col) {
@@ -171,8 +232,10 @@ topk_kernel(const TopkArgs a) {
         // 1. lower bound of the k-th largest code from a prefix of the columns
         const uint32_t prefix_end = min(c_hi, c_lo + static_cast<uint32_t>(kPrefixColumns / CS));
         uint32_t mx = 0;
-        for_each_code<DTYPE, kTopkThreads>(row_ptr, c_lo, prefix_end, a.vector,
-                                           [&](uint32_t, uint32_t code) { mx = max(mx, code); });
+        for_each_vector<DTYPE, kTopkThreads>(
+            row_ptr, c_lo, prefix_end, a.vector,
+            [&](uint32_t, const uint4 &w) { mx = max(mx, vector_max_code<DTYPE>(w)); },
+            [&](uint32_t, uint32_t code) { mx = max(mx, code); });
         mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
         mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
         if ((threadIdx.x & 3) == 0) sh_max[threadIdx.x >> 2] = mx;
@@ -199,12 +262,20 @@ topk_kernel(const TopkArgs a) {
         }
 
         // 2. candidates: every column that reaches the bound
-        for_each_code<DTYPE, kTopkThreads>(row_ptr, c_lo, c_hi, a.vector, [&](uint32_t col, uint32_t code) {
+        auto push = [&](uint32_t col, uint32_t code) {
             if (code >= floor_code) {
                 const unsigned pos = atomicAdd(&sh_count, 1u);
                 if (pos < kCap) sh_cand[pos] = composite(code, col);
             }
-        });
+        };
+        for_each_vector<DTYPE, kTopkThreads>(
+            row_ptr, c_lo, c_hi, a.vector,
+            [&](uint32_t col0, const uint4 &w) {
+                if (vector_max_code<DTYPE>(w) < floor_code) return;   // the common case: one compare per vector
+#pragma unroll
+                for (int i = 0; i < 16 / ESIZE; ++i) push(col0 + i, element_code<DTYPE>(w, i));
+            },
+            push);
         __syncthreads();
         unsigned n = sh_count;
         if constexpr (CS > 1) {
@@ -384,31 +455,6 @@ __device__ __forceinline__ void issue_chunk(const TopkArgs &a, StreamShared &sh)
     }
 }
 
-// Order codes of the bulk-copy kernel.  fp32: order_code of the bits.  bf16: the 16-bit analogue,
-// bits ^ 0xffff for negative values and bits ^ 0x8000 otherwise, computed for both halves of a word
-// at once (a byte permute in sign-replication mode gives each half's sign mask).
-__device__ __forceinline__ uint32_t packed_codes(uint32_t w) {
-    uint32_t sign;   // 0xffff in each half whose value is negative (selector bit 3: replicate the byte's msb)
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(sign) : "r"(w), "r"(0u), "r"(0xBB99u));
-    return w ^ (sign | 0x80008000u);
-}
-template <int DTYPE>
-__device__ __forceinline__ uint32_t vector_max_code(const uint4 &w) {
-    if constexpr (DTYPE == SBW_DTYPE_F32) {
-        return max(max(order_code(w.x), order_code(w.y)), max(order_code(w.z), order_code(w.w)));
-    } else {
-        const uint32_t m = __vmaxu2(__vmaxu2(packed_codes(w.x), packed_codes(w.y)),
-                                    __vmaxu2(packed_codes(w.z), packed_codes(w.w)));
-        return max(m >> 16, m & 0xffffu);
-    }
-}
-template <int DTYPE>
-__device__ __forceinline__ uint32_t element_code(const uint4 &w, int i) {
-    const uint32_t *e = reinterpret_cast<const uint32_t *>(&w);
-    if constexpr (DTYPE == SBW_DTYPE_F32) return order_code(e[i]);
-    else return (packed_codes(e[i >> 1]) >> (16 * (i & 1))) & 0xffffu;
-}
-
 // Consumes `nchunks` chunks covering `limit` bytes from the start of the row; f(first column,
 // vector) for every 16-byte vector, each thread taking every kStreamThreads-th.
 template <int DTYPE, typename F>
@@ -517,10 +563,7 @@ topk_stream_kernel(const TopkArgs a) {
             for (int i = 0; i < 16 / ESIZE; ++i) push(col0 + i, element_code<DTYPE>(w, i));
         });
         for (uint32_t c = a.row_bytes / ESIZE + threadIdx.x; c < V; c += kStreamThreads) {   // ragged end of the row
-            uint32_t code;
-            if constexpr (DTYPE == SBW_DTYPE_F32) code = order_code(reinterpret_cast<const uint32_t *>(row_ptr)[c]);
-            else code = packed_codes(reinterpret_cast<const uint16_t *>(row_ptr)[c]) & 0xffffu;
-            push(c, code);
+            push(c, scalar_code<DTYPE>(row_ptr, c));
         }
         __syncthreads();
         const unsigned n = sh.count;
