@@ -99,18 +99,6 @@ int sbw_bias_logits_topk(void *logits, int dtype, int64_t B, int64_t V, int64_t 
                          float delta, int scheme, int64_t top_k, void *stream);
 
 /*
- * sbw_pipeline_timeouts -- health counter of the kernels that stage rows through shared memory
- * with bulk asynchronous copies (sbw_bias_logits_topk on batches of more rows than SMs).  Their
- * waits on copy completion are bounded; a wait that runs out makes its thread block stop and
- * leave its remaining rows unbiased rather than spin.  *host_count receives the number of such
- * events on the current device since the library was loaded: 0 on a healthy device, so a caller
- * that must know may check it after synchronising.
- *   host_count  host pointer, not NULL.
- * Blocks until earlier work on the device has finished (it is a device-to-host copy).
- */
-int sbw_pipeline_timeouts(unsigned long long *host_count);
-
-/*
  * sbw_bias_logits_host -- the same step for callers whose logits live in HOST memory: copies
  * B*ld elements and the context tokens to the device staging buffer, runs sbw_bias_logits on
  * it, and copies the logits back, all enqueued on `stream` (the copies are asynchronous only if

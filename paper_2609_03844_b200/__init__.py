@@ -11,7 +11,7 @@ from .binding import (DTYPE_BF16, DTYPE_F32, SCHEME_CONTEXT, SCHEME_SELFSALT, Sb
                       sbw_roc_auc, sbw_roc_auc_batched, sbw_roc_auc_workspace_bytes, sbw_bias_sample_filtered,
                       sbw_sample_filtered_workspace_bytes,
                       sbw_detect_workspace_bytes, sbw_int_probe, sbw_sample_workspace_bytes,
-                      sbw_pipeline_timeouts, sbw_version)
+                      sbw_version)
 
 __all__ = ["DTYPE_BF16", "DTYPE_F32", "SCHEME_CONTEXT", "SCHEME_SELFSALT", "SbwError", "lib",
            "library_path", "sbw_bias_logits", "sbw_bias_logits_host", "sbw_bias_logits_topk",
@@ -20,5 +20,4 @@ __all__ = ["DTYPE_BF16", "DTYPE_F32", "SCHEME_CONTEXT", "SCHEME_SELFSALT", "SbwE
            "sbw_prefix_z", "sbw_detect_unique", "sbw_detect_unique_workspace_bytes",
            "sbw_roc_auc", "sbw_roc_auc_batched", "sbw_roc_auc_workspace_bytes", "sbw_bias_sample_filtered",
            "sbw_sample_filtered_workspace_bytes",
-           "sbw_detect_workspace_bytes", "sbw_int_probe", "sbw_sample_workspace_bytes", "sbw_pipeline_timeouts",
-           "sbw_version"]
+           "sbw_detect_workspace_bytes", "sbw_int_probe", "sbw_sample_workspace_bytes", "sbw_version"]

@@ -32,8 +32,7 @@ EXPORTS = ("sbw_version", "sbw_last_cuda_error", "sbw_bias_logits",
            "sbw_bias_sample_shard", "sbw_sample_combine", "sbw_detect_bits_words", "sbw_detect_bits",
            "sbw_window_z", "sbw_prefix_z", "sbw_detect_unique_workspace_bytes", "sbw_detect_unique",
            "sbw_roc_auc_workspace_bytes", "sbw_roc_auc", "sbw_sample_filtered_workspace_bytes",
-           "sbw_bias_sample_filtered", "sbw_roc_auc_batched", "sbw_bias_sample_shard_ids",
-           "sbw_pipeline_timeouts")
+           "sbw_bias_sample_filtered", "sbw_roc_auc_batched", "sbw_bias_sample_shard_ids")
 
 _lib = None
 
@@ -67,8 +66,6 @@ def lib() -> ctypes.CDLL:
         L.sbw_version.argtypes = []
         L.sbw_last_cuda_error.restype = i32
         L.sbw_last_cuda_error.argtypes = []
-        L.sbw_pipeline_timeouts.restype = i32
-        L.sbw_pipeline_timeouts.argtypes = [c.POINTER(c.c_ulonglong)]
         L.sbw_bias_logits.restype = i32
         L.sbw_bias_logits.argtypes = [vp, i32, i64, i64, i64, i64, vp, i32, u64, c.c_double,
                                       c.c_float, i32, vp]
@@ -178,13 +175,6 @@ def _ctx(ctx_tokens: torch.Tensor, B: int) -> int:
 
 def sbw_version() -> str:
     return lib().sbw_version().decode()
-
-
-def sbw_pipeline_timeouts() -> int:
-    """Bounded waits of the bulk-copy kernels that ran out on the current device (0 when healthy)."""
-    count = ctypes.c_ulonglong(0)
-    _check("sbw_pipeline_timeouts", lib().sbw_pipeline_timeouts(ctypes.byref(count)))
-    return int(count.value)
 
 
 def sbw_bias_logits(logits: torch.Tensor, ctx_tokens: torch.Tensor, key: int, gamma: float,

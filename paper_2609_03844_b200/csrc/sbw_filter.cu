@@ -22,6 +22,7 @@
 #include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
+#include "sbw_codes.cuh"
 #include "sbw_common.cuh"
 #include "sbw_gumbel.cuh"
 #include "sbw_hash.cuh"
@@ -93,13 +94,6 @@ struct FilterShared {
     unsigned int part_max, part_floor, part_deep;
     unsigned long long part_z;
 };
-
-__device__ __forceinline__ uint32_t order_code(uint32_t bits) {
-    return (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
-}
-__device__ __forceinline__ uint32_t order_decode(uint32_t code) {
-    return (code & 0x80000000u) ? (code & 0x7fffffffu) : ~code;
-}
 
 // Codes are compared in units of one representable value of the logits' type: 32 significant
 // bits for fp32, the upper 16 for bf16 (whose lower 16 bits are always zero).
@@ -235,6 +229,31 @@ __device__ __forceinline__ void for_each_key(const char *row_ptr, uint32_t V, ui
             if (nfull * VEC + i < V) f(nfull * VEC + i, bits, order_key(bits));
         }
     }
+}
+
+// The walk for passes that only compare: fvec(first column, vector) for whole vectors (each
+// thread every kFilterThreads-th), fone(column, code) for the columns of a ragged last vector.
+template <int DTYPE, typename FV, typename F1>
+__device__ __forceinline__ void for_each_vector(const char *row_ptr, uint32_t V, uint32_t vec_begin, uint32_t nvec,
+                                                FV fvec, F1 fone) {
+    constexpr int VEC = DTYPE == SBW_DTYPE_F32 ? 4 : 8;
+    constexpr int kInFlight = 4;
+    const uint32_t nfull = min(nvec, V / VEC);
+    for (uint32_t j0 = vec_begin + threadIdx.x; j0 < nfull; j0 += kInFlight * kFilterThreads) {
+        uint4 w[kInFlight];
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+            const uint32_t j = j0 + u * kFilterThreads;
+            w[u] = j < nfull ? reinterpret_cast<const uint4 *>(row_ptr)[j] : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+            const uint32_t j = j0 + u * kFilterThreads;
+            if (j < nfull) fvec(j * VEC, w[u]);
+        }
+    }
+    if (nfull < nvec && nfull >= vec_begin && threadIdx.x == 0)
+        for (uint32_t col = nfull * VEC; col < V; ++col) fone(col, scalar_code<DTYPE>(row_ptr, col));
 }
 
 __device__ __forceinline__ unsigned long long warp_sum(unsigned long long x) {
@@ -514,9 +533,11 @@ __device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &s
     Head h;
     h.leave = false;
     // pass A: per-thread maxima, sorted descending (as ~code ascending) in the list area
-    int32_t my_key = static_cast<int32_t>(0x80000000u);        // decodes to code 0
-    for_each_key<DTYPE>(src_row, V, vec_lo, vec_hi, [&](uint32_t, uint32_t, int32_t key) { my_key = max(my_key, key); });
-    const uint32_t my_max = code_of_key<DTYPE>(my_key);
+    uint32_t my_max = 0u;
+    for_each_vector<DTYPE>(
+        src_row, V, vec_lo, vec_hi,
+        [&](uint32_t, const uint4 &w) { my_max = max(my_max, vector_max_code<DTYPE>(w)); },
+        [&](uint32_t, uint32_t code) { my_max = max(my_max, code); });
     __syncthreads();
     sh.list[threadIdx.x] = static_cast<unsigned long long>(~my_max);
     if (threadIdx.x == 0) sh.list_n = 0u;
@@ -564,6 +585,23 @@ __device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &s
     // pass B
     unsigned long long z_local = 0;
     const int32_t floor_key = key_of_code<DTYPE>(floor_code), lo_key = key_of_code<DTYPE>(code_lo);
+    if (!want_z) {
+        // gather only: one compare per vector, the elements only where it reaches the floor
+        auto take = [&](uint32_t col, uint32_t code) {
+            if (code >= floor_code && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= kListCap) {
+                const unsigned idx = atomicAdd(&sh.list_n, 1u);
+                if (idx < kListCap) sh.list[idx] = (static_cast<unsigned long long>(key_m - code) << 32) | col;
+            }
+        };
+        for_each_vector<DTYPE>(
+            src_row, V, vec_lo, vec_hi,
+            [&](uint32_t col0, const uint4 &w) {
+                if (vector_max_code<DTYPE>(w) < floor_code) return;
+#pragma unroll
+                for (int i = 0; i < (DTYPE == SBW_DTYPE_F32 ? 4 : 8); ++i) take(col0 + i, element_code<DTYPE>(w, i));
+            },
+            take);
+    } else
     for_each_key<DTYPE>(src_row, V, vec_lo, vec_hi, [&](uint32_t col, uint32_t bits, int32_t key) {
         if (want_z && key >= lo_key)
             z_local += nucleus_weight(__uint_as_float(bits), m, code_of_key<DTYPE>(key) == key_m, a.c);
