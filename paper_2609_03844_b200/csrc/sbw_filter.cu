@@ -237,7 +237,7 @@ template <int DTYPE, typename FV, typename F1>
 __device__ __forceinline__ void for_each_vector(const char *row_ptr, uint32_t V, uint32_t vec_begin, uint32_t nvec,
                                                 FV fvec, F1 fone) {
     constexpr int VEC = DTYPE == SBW_DTYPE_F32 ? 4 : 8;
-    constexpr int kInFlight = 4;
+    constexpr int kInFlight = 4;   // eight were measured slower here (the kernel is at its register limit)
     const uint32_t nfull = min(nvec, V / VEC);
     for (uint32_t j0 = vec_begin + threadIdx.x; j0 < nfull; j0 += kInFlight * kFilterThreads) {
         uint4 w[kInFlight];

@@ -103,7 +103,7 @@ __device__ __forceinline__ void for_each_vector(const char *row_ptr, uint32_t be
     uint32_t done = begin;
     if (vector) {
         const uint32_t nfull = end / VEC;
-        constexpr int kInFlight = 4;   // independent 128-bit loads per thread before the first use
+        constexpr int kInFlight = 8;   // independent 128-bit loads per thread before the first use
         for (uint32_t j0 = begin / VEC + threadIdx.x; j0 < nfull; j0 += kInFlight * kTopkThreads) {
             uint4 w[kInFlight];
 #pragma unroll
