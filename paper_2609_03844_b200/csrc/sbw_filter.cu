@@ -74,6 +74,7 @@ struct FilterArgs {
 // native 32-bit shared-memory adds instead of 64-bit compare-and-swap loops, which crawl when the
 // candidates crowd into a few bins (bf16 logits have a few hundred distinct values near the top).
 // A limb counter holds up to 2^21 candidates' worth.  The list reuses the histogram's space.
+constexpr int kWeightTab = 1280;   // ten binades of bf16 codes
 constexpr int kLimbs = 4;
 constexpr int kLimbBits = 11;
 constexpr int64_t kMaxFilterV = int64_t(1) << 21;
@@ -85,6 +86,12 @@ struct FilterShared {
             unsigned int hist_l[kLimbs][kBins];
         };
         unsigned long long list[kListCap];
+        struct {
+            unsigned long long list_view[kListCap];
+            // bf16 rows, top-p total: the weights of the kWeightTab codes from the row maximum down
+            // and of the kWeightTab lowest codes that can have a weight, filled once per row
+            unsigned long long wtab[2 * kWeightTab + 1];   // the last entry is 0
+        };
     };
     unsigned long long red[kFilterWarps];
     unsigned long long bcast[4];
@@ -585,7 +592,41 @@ __device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &s
     // pass B
     unsigned long long z_local = 0;
     const int32_t floor_key = key_of_code<DTYPE>(floor_code), lo_key = key_of_code<DTYPE>(code_lo);
-    if (!want_z) {
+    if (want_z && DTYPE == SBW_DTYPE_BF16) {
+        // A bf16 logit is one of 65536 codes and its weight is a function of the code alone: the
+        // weights of the codes that occur in numbers -- the ten binades below the maximum and the
+        // ten above the lowest code with a weight -- are computed once per row, the pass looks them
+        // up, and only a logit outside both windows (tiny magnitudes) is evaluated on the spot.
+        for (int i = threadIdx.x; i < 2 * kWeightTab; i += kFilterThreads) {
+            const bool upper = i < kWeightTab;
+            const uint32_t code = upper ? key_m - static_cast<uint32_t>(i) : code_lo + static_cast<uint32_t>(i - kWeightTab);
+            const bool valid = (upper ? static_cast<uint32_t>(i) <= key_m : code <= key_m) && code >= code_lo;
+            sh.wtab[i] = valid ? nucleus_weight(value_of_code<DTYPE>(code), m, code == key_m, a.c) : 0ull;
+        }
+        if (threadIdx.x == 0) sh.wtab[2 * kWeightTab] = 0ull;
+        __syncthreads();
+        auto take = [&](uint32_t col, uint32_t code) {
+            // one lookup without branches: the upper window, else the lower one, else the zero entry
+            const uint32_t down = key_m - code, up = code - code_lo;
+            const bool in_upper = down < static_cast<uint32_t>(kWeightTab);
+            const bool in_lower = up < static_cast<uint32_t>(kWeightTab);
+            const uint32_t slot = in_upper ? down : in_lower ? kWeightTab + up : 2u * kWeightTab;
+            z_local += sh.wtab[slot];
+            if (!in_upper && !in_lower && code >= code_lo)       // rare: between the windows
+                z_local += nucleus_weight(value_of_code<DTYPE>(code), m, false, a.c);
+            if (code >= floor_code && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= kListCap) {
+                const unsigned idx = atomicAdd(&sh.list_n, 1u);
+                if (idx < kListCap) sh.list[idx] = (static_cast<unsigned long long>(key_m - code) << 32) | col;
+            }
+        };
+        for_each_vector<DTYPE>(
+            src_row, V, vec_lo, vec_hi,
+            [&](uint32_t col0, const uint4 &w) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) take(col0 + i, element_code<DTYPE>(w, i));
+            },
+            take);
+    } else if (!want_z) {
         // gather only: one compare per vector, the elements only where it reaches the floor
         auto take = [&](uint32_t col, uint32_t code) {
             if (code >= floor_code && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= kListCap) {
