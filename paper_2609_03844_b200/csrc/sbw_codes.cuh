@@ -19,6 +19,11 @@ __device__ __forceinline__ uint32_t order_decode(uint32_t code) {
     return (code & 0x80000000u) ? (code & 0x7fffffffu) : ~code;
 }
 
+// A signed integer with the order of order_code: signed_key(b) ^ 0x80000000 == order_code(b).
+__device__ __forceinline__ int32_t signed_key(uint32_t bits) {
+    return static_cast<int32_t>(bits ^ (static_cast<uint32_t>(static_cast<int32_t>(bits) >> 31) & 0x7fffffffu));
+}
+
 // The codes of both bf16 halves of a word at once.
 __device__ __forceinline__ uint32_t packed_codes(uint32_t w) {
     uint32_t sign;   // 0xffff in each half whose value is negative (selector bit 3: replicate the byte's msb)
@@ -30,7 +35,10 @@ __device__ __forceinline__ uint32_t packed_codes(uint32_t w) {
 template <int DTYPE>
 __device__ __forceinline__ uint32_t vector_max_code(const uint4 &w) {
     if constexpr (DTYPE == SBW_DTYPE_F32) {
-        return max(max(order_code(w.x), order_code(w.y)), max(order_code(w.z), order_code(w.w)));
+        // signed keys (the magnitude bits of negative values flipped) cost two operations each; the
+        // largest key with its sign bit flipped is the largest code
+        const int32_t k = max(max(signed_key(w.x), signed_key(w.y)), max(signed_key(w.z), signed_key(w.w)));
+        return static_cast<uint32_t>(k) ^ 0x80000000u;
     } else {
         const uint32_t m = __vmaxu2(__vmaxu2(packed_codes(w.x), packed_codes(w.y)),
                                     __vmaxu2(packed_codes(w.z), packed_codes(w.w)));

@@ -158,6 +158,11 @@ __device__ __forceinline__ unsigned long long nucleus_weight(float l, float m, b
 }
 
 // The row is padded to whole 16-byte vectors; loads are 16 bytes wide, several in flight.
+// The same, out of line, for call sites that are reached rarely inside unrolled loops.
+__device__ __noinline__ unsigned long long nucleus_weight_rare(float l, float m, float c) {
+    return nucleus_weight(l, m, false, c);
+}
+
 template <int DTYPE>
 __device__ __forceinline__ uint32_t vectors_of(uint32_t V) {
     return (V + (DTYPE == SBW_DTYPE_F32 ? 4 : 8) - 1) / (DTYPE == SBW_DTYPE_F32 ? 4 : 8);
@@ -613,7 +618,7 @@ __device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &s
             const uint32_t slot = in_upper ? down : in_lower ? kWeightTab + up : 2u * kWeightTab;
             z_local += sh.wtab[slot];
             if (!in_upper && !in_lower && code >= code_lo)       // rare: between the windows
-                z_local += nucleus_weight(value_of_code<DTYPE>(code), m, false, a.c);
+                z_local += nucleus_weight_rare(value_of_code<DTYPE>(code), m, a.c);
             if (code >= floor_code && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= kListCap) {
                 const unsigned idx = atomicAdd(&sh.list_n, 1u);
                 if (idx < kListCap) sh.list[idx] = (static_cast<unsigned long long>(key_m - code) << 32) | col;
