@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 SCHEMES = [sbw.SCHEME_CONTEXT, sbw.SCHEME_SELFSALT]
 
 
-def _check(x, V, ctx, key, gamma, delta, scheme, k, off=0, view=None):
+def _check(x, V, ctx, key, gamma, delta, scheme, k, off=0, view=None, nan_payload=False):
     dev = require_gpu()
     x_dev = x.to(dev)
     target = x_dev if view is None else view(x_dev)
@@ -23,7 +23,7 @@ def _check(x, V, ctx, key, gamma, delta, scheme, k, off=0, view=None):
     want, sel = oracle.bias_logits_topk(host_bits(src), V, ctx.numpy(), key, gamma, delta, scheme, k,
                                         vocab_offset=off)
     got = host_bits(target.contiguous()) if view is not None else host_bits(x_dev)
-    assert_same_bits(got, want)
+    assert_same_bits(got, want, allow_nan_payload=nan_payload)
     return got, sel
 
 
@@ -141,3 +141,22 @@ def test_large_batches_of_full_vocabulary_rows():
         inputs.add_zipf_spike_(x, V, seed=98)
         ctx = inputs.uniform_tokens((B, 1), V, seed=99)
         _check(x, V, ctx, KEY, 0.25, 4.0, sbw.SCHEME_SELFSALT, 40)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("B", [9, 150])
+def test_special_values_in_the_vector_passes(dtype, B):
+    """NaNs of both signs, infinities, zeros of both signs, subnormals and huge values scattered over aligned
+    rows (a cluster per row at B = 9, one CTA per row at B = 150): the order codes of whole vectors must
+    rank them like the oracle's total order on bit patterns."""
+    V = 8192
+    x = inputs.logits_normal(B, V, 4.0, dtype, seed=120 + B)
+    specials = torch.tensor([float("nan"), -float("nan"), float("inf"), float("-inf"), 0.0, -0.0, 1e-40, -1e-40,
+                             3e38, -3e38], dtype=torch.float32).to(dtype)
+    g = torch.Generator().manual_seed(121)
+    rows = torch.randint(0, B, (400,), generator=g)
+    cols = torch.randint(0, V, (400,), generator=g)
+    x[rows, cols] = specials[torch.randint(0, len(specials), (400,), generator=g)]
+    ctx = inputs.uniform_tokens((B, 1), V, seed=122)
+    for k, delta in ((40, 2.0), (128, -1.0), (3, 8.0)):
+        _check(x, V, ctx, KEY, 0.5, delta, sbw.SCHEME_SELFSALT, k, nan_payload=True)
