@@ -432,6 +432,15 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
         "achieved_gbs": 4 * B3 * V3 / s / 1e9, "frac": 4 * B3 * V3 / s / 1e9 / hbm,
         "note": "one read of the row from HBM (4 B/logit), second read from L2, 40 columns written"}
     del p3, c3
+    # the same scheme on large batches (1024 rows): fp32 at V = 151936 and bf16 at V = 128256
+    for tag, dt, Vk, es in (("fp32", torch.float32, V3, 4), ("bf16", torch.bfloat16, V2, 2)):
+        pk = [inputs.logits_normal(1024, Vk, 4.0, dt, seed=440 + i, device=dev) for i in range(2)]
+        ck = [inputs.uniform_tokens((1024, 1), Vk, seed=450 + i, device=dev) for i in range(2)]
+        s = _time_calls(lambda i: sbw.sbw_bias_logits_topk(pk[i % 2], ck[i % 2], KEY, 0.25, 4.0, sbw.SCHEME_SELFSALT, 40), 32)
+        out[f"bias_top40_{tag}_selfsalt_B1024_V{Vk}"] = {
+            "gelem_s": 1024 * Vk / s / 1e9, "ms": s * 1e3, "bound": "hbm",
+            "achieved_gbs": es * 1024 * Vk / s / 1e9, "frac": es * 1024 * Vk / s / 1e9 / hbm}
+        del pk, ck
     # config 2 shape under the self-salt scheme
     p2 = [inputs.logits_normal(B2, V2, 4.0, torch.bfloat16, seed=400 + i, device=dev) for i in range(16)]
     c2 = [inputs.uniform_tokens((B2, 1), V2, seed=420 + i, device=dev) for i in range(16)]
