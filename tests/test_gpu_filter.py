@@ -168,3 +168,22 @@ def test_rounding_of_the_biased_sum_at_the_cut(dtype, base, delta):
     for top_k in (5, 50, 300):
         _check(x, ctx, sbw.SCHEME_CONTEXT, 1.0, top_k, 1.0, delta=delta * step, gamma=0.5)
         _check(x, ctx, sbw.SCHEME_SELFSALT, 1.0, top_k, 0.7, delta=delta * step, gamma=0.5)
+
+
+@pytest.mark.parametrize("B", [6, 300])
+def test_bf16_weight_table_windows(B):
+    """bf16 top-p totals come from a per-row table over two windows of codes (below the maximum, above the
+    lowest weighted code) with everything else evaluated directly: rows whose logits are all negative, all tiny,
+    spread over many binades, subnormal, or concentrated on a few codes must still give the oracle's kept sets."""
+    V = 12000
+    x = inputs.logits_normal(B, V, 4.0, torch.bfloat16, seed=130 + B)
+    x[0] = x[0] - 40.0                                   # every logit negative: the maximum is a negative code
+    x[1] = x[1] * 1e-20                                  # tiny magnitudes of both signs
+    x[2] = torch.exp2(torch.linspace(-120.0, 4.0, V)).to(torch.bfloat16) * torch.sign(x[2].float()).to(torch.bfloat16)
+    x[3] = x[3] * 1e-39                                  # subnormals and zeros of both signs
+    x[4] = torch.round(x[4] / 4) * 4                     # a handful of distinct codes
+    x[5, :] = -3.0
+    x[5, ::7] = 2.5
+    ctx = inputs.uniform_tokens((B, 1), V, seed=131)
+    for tau, top_p, delta in ((0.7, 0.8, 2.0), (0.05, 0.99, 2.0), (3.0, 0.5, -1.0), (1.0, 0.9999, 0.25)):
+        _check(x, ctx, sbw.SCHEME_CONTEXT, tau, 0, top_p, delta=delta)
