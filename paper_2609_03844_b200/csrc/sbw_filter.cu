@@ -43,6 +43,8 @@ constexpr int kFilterWarps = kFilterThreads / 32;
 constexpr int kBins = 2048;
 constexpr int kBinBits = 11;
 constexpr int kListCap = 2048;
+constexpr int kBigCap = 4096;
+constexpr int kLastColumns = 2600;   // what the last retry aims to gather: below kBigCap with room for ties
 constexpr uint64_t kAll = ~0ull;
 
 struct FilterArgs {
@@ -86,6 +88,7 @@ struct FilterShared {
             unsigned int hist_l[kLimbs][kBins];
         };
         unsigned long long list[kListCap];
+        unsigned long long list_big[kBigCap];   // the last retry before the radix descent
         struct {
             unsigned long long list_view[kListCap];
             // bf16 rows, top-p total: the weights of the kWeightTab codes from the row maximum down
@@ -98,7 +101,7 @@ struct FilterShared {
     unsigned int list_n;
     unsigned int red32[kFilterWarps];
     // what the CTAs of a cluster tell each other about their parts of the row
-    unsigned int part_max, part_floor, part_deep;
+    unsigned int part_max, part_floor, part_deep, part_last;
     unsigned long long part_z;
 };
 
@@ -308,15 +311,15 @@ __device__ __forceinline__ unsigned long long block_exclusive_scan(unsigned long
 enum { kModeCount = 0, kModeMass = 1 };
 
 // Bitonic sort of sh.list[0 .. len), len a power of two >= 2, ascending.
-__device__ __forceinline__ void sort_list(FilterShared &sh, int len) {
+__device__ __forceinline__ void sort_list(unsigned long long *list, int len) {
     for (int k = 2; k <= len; k <<= 1) {
         for (int j = k >> 1; j > 0; j >>= 1) {
             for (int t = threadIdx.x; t < len / 2; t += kFilterThreads) {
                 const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
-                const unsigned long long a = sh.list[i], b = sh.list[i + j];
+                const unsigned long long a = list[i], b = list[i + j];
                 if ((a > b) == ((i & k) == 0)) {
-                    sh.list[i] = b;
-                    sh.list[i + j] = a;
+                    list[i] = b;
+                    list[i + j] = a;
                 }
             }
             __syncthreads();
@@ -428,7 +431,7 @@ __device__ unsigned long long select_boundary(const char *row_ptr, uint32_t V, u
             while (len < n) len <<= 1;
             for (int i = n + threadIdx.x; i < len; i += kFilterThreads) sh.list[i] = kAll;
             __syncthreads();
-            sort_list(sh, len);
+            sort_list(sh.list, len);
             constexpr int kPer = kListCap / kFilterThreads;
             unsigned long long w[kPer], mine = 0;
 #pragma unroll
@@ -531,6 +534,7 @@ struct Head {
     unsigned gathered;            // entries in sh.list (unsorted), or kListCap + 1
     unsigned long long z_all;     // total weight of the row (want_z)
     uint32_t deep_floor;          // a lower floor (the 480th largest thread maximum) for one retry
+    uint32_t last_floor;          // a still lower floor (about kLastColumns columns) for the last retry
     bool leave;
 };
 
@@ -554,16 +558,24 @@ __device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &s
     sh.list[threadIdx.x] = static_cast<unsigned long long>(~my_max);
     if (threadIdx.x == 0) sh.list_n = 0u;
     __syncthreads();
-    sort_list(sh, kFilterThreads);
+    sort_list(sh.list, kFilterThreads);
     uint32_t key_m = ~static_cast<uint32_t>(sh.list[0]);
     uint32_t floor_code = ~static_cast<uint32_t>(sh.list[(want + CS - 1) / CS - 1]);
     uint32_t deep_floor = ~static_cast<uint32_t>(sh.list[(kDeepRank + CS - 1) / CS - 1]);
+    // the floor of the last retry: the thread maximum of the rank that about kLastColumns columns of
+    // an ordinary row reach (a thread of this CTA sees V / (CS kFilterThreads) columns)
+    const float per_thread = fmaxf(static_cast<float>(V) / static_cast<float>(CS * kFilterThreads), 1.0f);
+    const float reach = fminf(static_cast<float>(kLastColumns) / static_cast<float>(V), 0.5f);
+    const int last_rank = min(max(static_cast<int>(kFilterThreads * (1.0f - __powf(1.0f - reach, per_thread))), 1),
+                              static_cast<int>(kFilterThreads));
+    uint32_t last_floor = ~static_cast<uint32_t>(sh.list[last_rank - 1]);
     __syncthreads();
     if constexpr (CS > 1) {
         if (threadIdx.x == 0) {
             sh.part_max = key_m;
             sh.part_floor = floor_code;
             sh.part_deep = deep_floor;
+            sh.part_last = last_floor;
         }
         cg::this_cluster().sync();
         for (unsigned r = 0; r < CS; ++r) {
@@ -571,10 +583,12 @@ __device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &s
             key_m = max(key_m, other->part_max);
             floor_code = min(floor_code, other->part_floor);
             deep_floor = min(deep_floor, other->part_deep);
+            last_floor = min(last_floor, other->part_last);
         }
     }
     h.key_m = key_m;
     h.deep_floor = deep_floor;
+    h.last_floor = last_floor;
     if (slack > 0.0f) {
         const float fl = value_of_code<DTYPE>(floor_code);
         if (fl == fl && fabsf(fl) != __int_as_float(0x7f800000)) {
@@ -684,17 +698,17 @@ __device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &s
 // sh.list[0 .. n) holds composites relative to key_m, unsorted.  Sorts them and applies the
 // top-k cut and the top-p crossing; returns the number of kept candidates (a prefix of the sorted
 // list), or 0 when the list does not reach far enough down the order.
-template <int DTYPE>
-__device__ __forceinline__ int cut_list(const FilterArgs &a, FilterShared &sh, int n, uint32_t key_m, bool use_k,
+template <int DTYPE, int CAP = kListCap>
+__device__ __forceinline__ int cut_list(const FilterArgs &a, FilterShared &sh, unsigned long long *list, int n, uint32_t key_m, bool use_k,
                                         bool use_p, unsigned long long z_all) {
-    constexpr int kPer = kListCap / kFilterThreads;
+    constexpr int kPer = CAP / kFilterThreads;
     const float m = value_of_code<DTYPE>(key_m);
     int len = 2;
     while (len < n) len <<= 1;
     __syncthreads();
-    for (int i = n + threadIdx.x; i < len; i += kFilterThreads) sh.list[i] = kAll;
+    for (int i = n + threadIdx.x; i < len; i += kFilterThreads) list[i] = kAll;
     __syncthreads();
-    sort_list(sh, len);
+    sort_list(list, len);
     int n1 = n;
     if (use_k) {
         if (a.top_k > n) return 0;
@@ -705,7 +719,7 @@ __device__ __forceinline__ int cut_list(const FilterArgs &a, FilterShared &sh, i
 #pragma unroll
     for (int i = 0; i < kPer; ++i) {
         const int idx = threadIdx.x * kPer + i;
-        const uint32_t dist = static_cast<uint32_t>(sh.list[idx < len ? idx : 0] >> 32);
+        const uint32_t dist = static_cast<uint32_t>(list[idx < len ? idx : 0] >> 32);
         w[i] = idx < n1 ? nucleus_weight(value_of_code<DTYPE>(key_m - dist), m, dist == 0u, a.c) : 0ull;
         mine += w[i];
     }
@@ -749,10 +763,10 @@ __device__ __forceinline__ void finish_row(const FilterArgs &a, FilterShared &sh
 
 // Draws the sample from the first n2 entries of the sorted list.
 template <int DTYPE>
-__device__ __forceinline__ void sample_list(const FilterArgs &a, FilterShared &sh, int64_t row, uint32_t key_m, int n2) {
+__device__ __forceinline__ void sample_list(const FilterArgs &a, FilterShared &sh, const unsigned long long *list, int64_t row, uint32_t key_m, int n2) {
     unsigned long long best = 0;
     for (int i = threadIdx.x; i < n2; i += kFilterThreads) {
-        const unsigned long long comp = sh.list[i];
+        const unsigned long long comp = list[i];
         const unsigned long long cand = packed_score<DTYPE>(a, static_cast<uint32_t>(row), static_cast<uint32_t>(comp),
                                                             key_m - static_cast<uint32_t>(comp >> 32));
         best = cand > best ? cand : best;
@@ -776,27 +790,50 @@ __device__ __forceinline__ bool full_row(const FilterArgs &a, FilterShared &sh, 
     const uint32_t key_m = h.key_m;
     int n2 = 0;
     if ((use_k || use_p) && h.gathered <= kListCap)
-        n2 = cut_list<DTYPE>(a, sh, static_cast<int>(h.gathered), key_m, use_k, use_p, h.z_all);
-    if (n2 == 0 && use_p && !use_k && h.gathered <= kListCap && h.deep_floor < key_m) {
-        // the nucleus reaches below the floor: one more gather pass with a lower floor (about three
-        // times as many columns) before the radix descent, which costs several passes
-        __syncthreads();
-        if (threadIdx.x == 0) sh.list_n = 0u;
-        __syncthreads();
-        const int32_t deep_key = key_of_code<DTYPE>(h.deep_floor);
-        for_each_key<DTYPE>(row_ptr, V, 0u, vectors_of<DTYPE>(V), [&](uint32_t col, uint32_t, int32_t key) {
-            if (key >= deep_key && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= kListCap) {
-                const unsigned idx = atomicAdd(&sh.list_n, 1u);
-                if (idx < kListCap)
-                    sh.list[idx] = (static_cast<unsigned long long>(key_m - code_of_key<DTYPE>(key)) << 32) | col;
+        n2 = cut_list<DTYPE>(a, sh, sh.list, static_cast<int>(h.gathered), key_m, use_k, use_p, h.z_all);
+    const unsigned long long *kept_list = sh.list;
+    if (n2 == 0 && use_p && !use_k && h.gathered <= kListCap) {
+        // The nucleus reaches below the floor.  Before the radix descent, which costs several passes
+        // on one CTA, gather again with a lower floor: the 480th largest thread maximum (about
+        // three times as many columns), then one that about kLastColumns columns reach, with a
+        // list of twice the size.
+        auto regather = [&](uint32_t floor_code, unsigned long long *list, unsigned cap) -> unsigned {
+            __syncthreads();
+            if (threadIdx.x == 0) sh.list_n = 0u;
+            __syncthreads();
+            auto take = [&](uint32_t col, uint32_t code) {
+                if (code >= floor_code && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= cap) {
+                    const unsigned idx = atomicAdd(&sh.list_n, 1u);
+                    if (idx < cap) list[idx] = (static_cast<unsigned long long>(key_m - code) << 32) | col;
+                }
+            };
+            for_each_vector<DTYPE>(
+                row_ptr, V, 0u, vectors_of<DTYPE>(V),
+                [&](uint32_t col0, const uint4 &w) {
+                    if (vector_max_code<DTYPE>(w) < floor_code) return;
+#pragma unroll
+                    for (int i = 0; i < (DTYPE == SBW_DTYPE_F32 ? 4 : 8); ++i) take(col0 + i, element_code<DTYPE>(w, i));
+                },
+                take);
+            __syncthreads();
+            return sh.list_n;
+        };
+        unsigned again = kListCap + 1u;
+        if (h.deep_floor < key_m) {
+            again = regather(h.deep_floor, sh.list, kListCap);
+            if (again <= kListCap)
+                n2 = cut_list<DTYPE>(a, sh, sh.list, static_cast<int>(again), key_m, false, true, h.z_all);
+        }
+        if (n2 == 0 && h.last_floor < h.deep_floor) {
+            again = regather(h.last_floor, sh.list_big, kBigCap);
+            if (again <= kBigCap) {
+                n2 = cut_list<DTYPE, kBigCap>(a, sh, sh.list_big, static_cast<int>(again), key_m, false, true, h.z_all);
+                kept_list = sh.list_big;
             }
-        });
-        __syncthreads();
-        const unsigned again = sh.list_n;
-        if (again <= kListCap) n2 = cut_list<DTYPE>(a, sh, static_cast<int>(again), key_m, false, true, h.z_all);
+        }
     }
     if (n2 > 0) {
-        sample_list<DTYPE>(a, sh, row, key_m, n2);
+        sample_list<DTYPE>(a, sh, kept_list, row, key_m, n2);
         return true;
     }
     __syncthreads();
@@ -884,9 +921,9 @@ __device__ __forceinline__ bool candidate_row(const FilterArgs &a, FilterShared 
             sh.list[i] = (static_cast<unsigned long long>(key_m - static_cast<uint32_t>(e >> 32)) << 32) |
                          static_cast<uint32_t>(e);
         }
-        const int n2 = cut_list<DTYPE>(a, sh, n, key_m, true, use_p, 0ull);
+        const int n2 = cut_list<DTYPE>(a, sh, sh.list, n, key_m, true, use_p, 0ull);
         if (n2 > 0) {
-            sample_list<DTYPE>(a, sh, row, key_m, n2);
+            sample_list<DTYPE>(a, sh, sh.list, row, key_m, n2);
             return true;
         }
     }
