@@ -525,7 +525,8 @@ __device__ __forceinline__ unsigned long long packed_score(const FilterArgs &a, 
 // barriers whatever the data; the others then leave (`leave`), CTA 0 finishes the row alone.
 // `slack` > 0 lowers the floor by that much (plus rounding room) in the logits' own units: the
 // caller gathers unbiased logits and wants every column that a bias of at most `slack` could lift
-// to the floor.  More than kListCap columns at or above the floor are reported as kListCap + 1.
+// to the floor.  More than `cap` columns (at most kBigCap; kListCap when the weight table shares the
+// space) at or above the floor are reported as cap + 1.
 // ---------------------------------------------------------------------------------------------
 constexpr int kDeepRank = 480;   // of the kFilterThreads thread maxima: about 1400 columns of an ordinary row
 
@@ -540,7 +541,7 @@ struct Head {
 
 template <int DTYPE, int CS>
 __device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &sh, const char *src_row, unsigned part,
-                                            int want, float slack, bool want_z) {
+                                            int want, float slack, bool want_z, unsigned cap) {
     namespace cg = cooperative_groups;
     const uint32_t V = static_cast<uint32_t>(a.V);
     const uint32_t nvec = vectors_of<DTYPE>(V);
@@ -633,9 +634,9 @@ __device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &s
             z_local += sh.wtab[slot];
             if (!in_upper && !in_lower && code >= code_lo)       // rare: between the windows
                 z_local += nucleus_weight_rare(value_of_code<DTYPE>(code), m, a.c);
-            if (code >= floor_code && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= kListCap) {
+            if (code >= floor_code && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= cap) {
                 const unsigned idx = atomicAdd(&sh.list_n, 1u);
-                if (idx < kListCap) sh.list[idx] = (static_cast<unsigned long long>(key_m - code) << 32) | col;
+                if (idx < cap) sh.list_big[idx] = (static_cast<unsigned long long>(key_m - code) << 32) | col;
             }
         };
         for_each_vector<DTYPE>(
@@ -648,9 +649,9 @@ __device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &s
     } else if (!want_z) {
         // gather only: one compare per vector, the elements only where it reaches the floor
         auto take = [&](uint32_t col, uint32_t code) {
-            if (code >= floor_code && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= kListCap) {
+            if (code >= floor_code && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= cap) {
                 const unsigned idx = atomicAdd(&sh.list_n, 1u);
-                if (idx < kListCap) sh.list[idx] = (static_cast<unsigned long long>(key_m - code) << 32) | col;
+                if (idx < cap) sh.list_big[idx] = (static_cast<unsigned long long>(key_m - code) << 32) | col;
             }
         };
         for_each_vector<DTYPE>(
@@ -665,10 +666,10 @@ __device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &s
     for_each_key<DTYPE>(src_row, V, vec_lo, vec_hi, [&](uint32_t col, uint32_t bits, int32_t key) {
         if (want_z && key >= lo_key)
             z_local += nucleus_weight(__uint_as_float(bits), m, code_of_key<DTYPE>(key) == key_m, a.c);
-        if (key >= floor_key && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= kListCap) {
+        if (key >= floor_key && *reinterpret_cast<volatile unsigned int *>(&sh.list_n) <= cap) {
             const unsigned idx = atomicAdd(&sh.list_n, 1u);
-            if (idx < kListCap)
-                sh.list[idx] = (static_cast<unsigned long long>(key_m - code_of_key<DTYPE>(key)) << 32) | col;
+            if (idx < cap)
+                sh.list_big[idx] = (static_cast<unsigned long long>(key_m - code_of_key<DTYPE>(key)) << 32) | col;
         }
     });
     h.z_all = want_z ? block_sum(z_local, sh) : 0ull;
@@ -681,9 +682,9 @@ __device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &s
             for (unsigned r = 1; r < CS; ++r) {
                 const FilterShared *other = cg::this_cluster().map_shared_rank(&sh, r);
                 const unsigned n_r = other->list_n;
-                if (gathered <= kListCap && n_r <= kListCap && gathered + n_r <= kListCap)
-                    for (unsigned i = threadIdx.x; i < n_r; i += kFilterThreads) sh.list[gathered + i] = other->list[i];
-                gathered = (gathered > kListCap || n_r > kListCap) ? kListCap + 1 : gathered + n_r;
+                if (gathered <= cap && n_r <= cap && gathered + n_r <= cap)
+                    for (unsigned i = threadIdx.x; i < n_r; i += kFilterThreads) sh.list_big[gathered + i] = other->list_big[i];
+                gathered = (gathered > cap || n_r > cap) ? cap + 1 : gathered + n_r;
                 h.z_all += other->part_z;
             }
         }
@@ -691,7 +692,7 @@ __device__ __forceinline__ Head gather_head(const FilterArgs &a, FilterShared &s
         h.leave = part != 0;
         __syncthreads();
     }
-    h.gathered = gathered > kListCap ? kListCap + 1 : gathered;
+    h.gathered = gathered > cap ? cap + 1 : gathered;
     return h;
 }
 
@@ -785,7 +786,7 @@ __device__ __forceinline__ bool full_row(const FilterArgs &a, FilterShared &sh, 
     const bool use_p = a.p32 != 0ull;
     const char *row_ptr = static_cast<const char *>(a.biased) + row * a.ld * ESIZE;
     const int want = use_k ? static_cast<int>(min(a.top_k, static_cast<int64_t>(kFilterThreads))) : 384;
-    const Head h = gather_head<DTYPE, CS>(a, sh, row_ptr, part, want, 0.0f, use_p && !use_k);
+    const Head h = gather_head<DTYPE, CS>(a, sh, row_ptr, part, want, 0.0f, use_p && !use_k, kListCap);
     if (h.leave) return false;
     const uint32_t key_m = h.key_m;
     int n2 = 0;
@@ -893,21 +894,23 @@ __device__ __forceinline__ bool candidate_row(const FilterArgs &a, FilterShared 
     const bool use_p = a.p32 != 0ull;
     const char *raw_row = static_cast<const char *>(a.raw) + row * a.ld_raw * ESIZE;
     const int want = static_cast<int>(min(a.top_k, static_cast<int64_t>(kFilterThreads)));
-    const Head h = gather_head<DTYPE, CS>(a, sh, raw_row, part, want, fmaxf(fabsf(a.delta), 0x1p-126f), false);
+    // the unbiased candidates may be many when |delta| is large: the list of twice the size
+    const Head h = gather_head<DTYPE, CS>(a, sh, raw_row, part, want, fmaxf(fabsf(a.delta), 0x1p-126f), false, kBigCap);
     if (h.leave) return false;
     const int32_t *ctx = a.ctx + row * a.W;
     const uint64_t r_row = a.scheme == SBW_SCHEME_CONTEXT ? seed_context(a.key, ctx, a.W) : 0ull;
     const uint32_t jmin = a.scheme == SBW_SCHEME_SELFSALT ? jenkins_min(ctx, a.W) : 0u;
-    if (h.gathered <= kListCap && static_cast<int64_t>(h.gathered) >= a.top_k) {
+    if (h.gathered <= kBigCap && static_cast<int64_t>(h.gathered) >= a.top_k) {
         const int n = static_cast<int>(h.gathered);
+        unsigned long long *list = sh.list_big;
         // bias the candidates: entries become (biased code << 32 | column), then composites
         // relative to the largest biased code
         uint32_t top = 0;
         for (int i = threadIdx.x; i < n; i += kFilterThreads) {
-            const unsigned long long e = sh.list[i];
+            const unsigned long long e = list[i];
             const uint32_t col = static_cast<uint32_t>(e);
             const uint32_t code = biased_code<DTYPE>(a, r_row, jmin, col, h.key_m - static_cast<uint32_t>(e >> 32));
-            sh.list[i] = (static_cast<unsigned long long>(code) << 32) | col;
+            list[i] = (static_cast<unsigned long long>(code) << 32) | col;
             top = max(top, code);
         }
         for (int d = 16; d > 0; d >>= 1) top = max(top, __shfl_xor_sync(0xffffffffu, top, d));
@@ -917,13 +920,13 @@ __device__ __forceinline__ bool candidate_row(const FilterArgs &a, FilterShared 
         uint32_t key_m = 0;
         for (int w = 0; w < kFilterWarps; ++w) key_m = max(key_m, sh.red32[w]);
         for (int i = threadIdx.x; i < n; i += kFilterThreads) {
-            const unsigned long long e = sh.list[i];
-            sh.list[i] = (static_cast<unsigned long long>(key_m - static_cast<uint32_t>(e >> 32)) << 32) |
+            const unsigned long long e = list[i];
+            list[i] = (static_cast<unsigned long long>(key_m - static_cast<uint32_t>(e >> 32)) << 32) |
                          static_cast<uint32_t>(e);
         }
-        const int n2 = cut_list<DTYPE>(a, sh, sh.list, n, key_m, true, use_p, 0ull);
+        const int n2 = cut_list<DTYPE, kBigCap>(a, sh, list, n, key_m, true, use_p, 0ull);
         if (n2 > 0) {
-            sample_list<DTYPE>(a, sh, sh.list, row, key_m, n2);
+            sample_list<DTYPE>(a, sh, list, row, key_m, n2);
             return true;
         }
     }
