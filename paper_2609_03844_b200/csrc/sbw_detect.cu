@@ -211,8 +211,76 @@ detect_kernel(const DetectArgs a) {
     }
 }
 
+// Few sequences: one CTA per sequence, its warps taking the trips in turn, so that a handful of
+// long texts still spreads over the GPU (a warp per sequence would walk each text alone).
+template <int SCHEME, int WIDTH>
+__global__ void __launch_bounds__(1024)
+detect_wide_kernel(const DetectArgs a) {
+    __shared__ int sh_count[32];
+    __shared__ long long sh_part[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int64_t seq = blockIdx.x;
+    int64_t off;
+    if (a.offsets) {
+        off = a.offsets[seq];
+    } else {
+        // no offsets given and few sequences: the CTA adds up the lengths before its own
+        long long part = 0;
+        for (int64_t i = threadIdx.x; i < seq; i += blockDim.x) part += clamp_len(a.lengths[i]);
+        for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
+        if (lane == 0) sh_part[warp] = part;
+        __syncthreads();
+        off = 0;
+        for (int w = 0; w < nwarps; ++w) off += sh_part[w];
+    }
+    int64_t L = clamp_len(a.lengths[seq]);
+    if (off < 0 || off >= a.total_tokens) L = 0;
+    else if (off + L > a.total_tokens) L = a.total_tokens - off;
+    const int width = WIDTH > 0 ? WIDTH : a.W;
+    const int32_t *tok = a.tokens + off;
+    const int len = static_cast<int>(L);
+    constexpr int kTrip = 32 * kDetectIlp;
+    uint32_t *bits = a.out_bits ? a.out_bits + (off >> 5) + 2 * seq : nullptr;
+
+    int count = 0;
+    const int full = len > width ? (len - width) / kTrip : 0;         // unmasked trips
+    for (int i = warp; i < full; i += nwarps)
+        count += score_trip<SCHEME, WIDTH, false>(a, tok, width + i * kTrip, len, lane, bits);
+    const int tail_base = width + full * kTrip;
+    if (tail_base < len && warp == full % nwarps)
+        count += score_trip<SCHEME, WIDTH, true>(a, tok, tail_base, len, lane, bits);
+    if (lane == 0) sh_count[warp] = count;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int total = 0;
+        for (int w = 0; w < nwarps; ++w) total += sh_count[w];
+        const int T = len > width ? len - width : 0;
+        a.out_counts[seq] = total;
+        if (a.out_T) a.out_T[seq] = T;
+        a.out_z[seq] = zscore(total, T, a.gamma);
+    }
+}
+
+// One warp per sequence fills the GPU from a few thousand sequences on; below that a CTA per
+// sequence, the wider the fewer there are.  Returns the CTA size, or 0 for a warp per sequence.
+inline int wide_threads(int64_t N, int sm_count) {
+    const int64_t resident_warps = static_cast<int64_t>(sm_count) * 64;
+    return N * 32 <= resident_warps ? 1024 : N * 16 <= resident_warps ? 512 : N * 8 <= resident_warps ? 256 : 0;
+}
+
 template <int SCHEME>
-cudaError_t launch_detect(const DetectArgs &a, unsigned grid, cudaStream_t s) {
+cudaError_t launch_detect(const DetectArgs &a, int sm_count, cudaStream_t s) {
+    const int wide = wide_threads(a.N, sm_count);
+    if (wide) {
+        const unsigned grid = static_cast<unsigned>(a.N);
+        switch (a.W) {
+            case 1: detect_wide_kernel<SCHEME, 1><<<grid, wide, 0, s>>>(a); break;
+            case 4: detect_wide_kernel<SCHEME, 4><<<grid, wide, 0, s>>>(a); break;
+            default: detect_wide_kernel<SCHEME, 0><<<grid, wide, 0, s>>>(a); break;
+        }
+        return cudaGetLastError();
+    }
+    const unsigned grid = static_cast<unsigned>((a.N + kDetectThreads / 32 - 1) / (kDetectThreads / 32));
     switch (a.W) {
         case 1: detect_kernel<SCHEME, 1><<<grid, kDetectThreads, 0, s>>>(a); break;
         case 4: detect_kernel<SCHEME, 4><<<grid, kDetectThreads, 0, s>>>(a); break;
@@ -277,18 +345,23 @@ int detect_impl(const int32_t *tokens, const int32_t *lengths, const int64_t *of
     a.out_bits = out_bits;
     a.weyl = make_weyl();
 
+    DeviceInfo di;
+    if (int rc = current_device_info(&di)) return rc;
     if (!offsets) {
         const size_t need = sbw_detect_workspace_bytes(N);
         if (!workspace || workspace_bytes < need || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
             return SBW_ERR_WORKSPACE;
-        int64_t *ws_offsets = nullptr;
-        const int rc = scan_lengths(lengths, N, workspace, &ws_offsets, s);
-        if (rc != SBW_OK) return rc;
-        a.offsets = ws_offsets;
+        // the plain detector on few sequences finds its offsets itself (one launch instead of two);
+        // with stored bits the offsets stay in the workspace for the calls that read the bits
+        if (out_bits || wide_threads(N, di.sm_count) == 0) {
+            int64_t *ws_offsets = nullptr;
+            const int rc = scan_lengths(lengths, N, workspace, &ws_offsets, s);
+            if (rc != SBW_OK) return rc;
+            a.offsets = ws_offsets;
+        }
     }
-    const unsigned grid = static_cast<unsigned>((N + kDetectThreads / 32 - 1) / (kDetectThreads / 32));
-    SBW_CUDA_TRY(scheme == SBW_SCHEME_CONTEXT ? launch_detect<SBW_SCHEME_CONTEXT>(a, grid, s)
-                                              : launch_detect<SBW_SCHEME_SELFSALT>(a, grid, s));
+    SBW_CUDA_TRY(scheme == SBW_SCHEME_CONTEXT ? launch_detect<SBW_SCHEME_CONTEXT>(a, di.sm_count, s)
+                                              : launch_detect<SBW_SCHEME_SELFSALT>(a, di.sm_count, s));
     return SBW_OK;
 }
 

@@ -89,3 +89,15 @@ def test_config5_null_half_full_size(scheme):
     tokens, lengths = inputs.null_token_streams(100000, 64, 1024, 128256, seed=75, device=dev)
     c, T, z = _compare(tokens.cpu(), lengths.cpu(), KEY, 0.25, scheme)
     assert abs(z.mean()) < 0.02 and abs(z.var() - 1.0) < 0.03          # null law of Eq. 5
+
+
+@pytest.mark.parametrize("N", [1, 3, 64, 296, 297, 592, 593, 1184, 1185])
+def test_few_sequences_take_a_cta_each(N):
+    """Below a few thousand sequences a CTA (32, 16 or 8 warps) scores each sequence, its warps taking the
+    128-token trips in turn; the batch sizes sit on both sides of every switch.  Lengths from 0 to beyond
+    many trips, ragged tails, both schemes, widths 1 and 3."""
+    tokens, lengths = inputs.null_token_streams(N, 0, 9000 if N <= 64 else 1500, 128256, seed=75 + N)
+    lengths[0] = 0 if N > 1 else 7777
+    tokens = inputs.uniform_tokens((int(lengths.sum()),), 128256, seed=76)
+    for scheme, W in ((sbw.SCHEME_CONTEXT, 1), (sbw.SCHEME_SELFSALT, 3)):
+        _compare(tokens, lengths, KEY, 0.25, scheme, W=W)
