@@ -345,12 +345,14 @@ int detect_impl(const int32_t *tokens, const int32_t *lengths, const int64_t *of
     a.out_bits = out_bits;
     a.weyl = make_weyl();
 
-    DeviceInfo di;
-    if (int rc = current_device_info(&di)) return rc;
-    if (!offsets) {
+    if (!offsets) {       // host-side validation first: it must not depend on a device being present
         const size_t need = sbw_detect_workspace_bytes(N);
         if (!workspace || workspace_bytes < need || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
             return SBW_ERR_WORKSPACE;
+    }
+    DeviceInfo di;
+    if (int rc = current_device_info(&di)) return rc;
+    if (!offsets) {
         // the plain detector on few sequences finds its offsets itself (one launch instead of two);
         // with stored bits the offsets stay in the workspace for the calls that read the bits
         if (out_bits || wide_threads(N, di.sm_count) == 0) {
