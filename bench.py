@@ -5,12 +5,32 @@
     python bench.py --impl reference --steps K --warmup W    # the CPU oracle, as it stands
 
 One "step" is one decode step of the headline workload: `sbw_bias_logits` (context-hash seeding,
-gamma 0.5, delta 2.0, key 0x5EED) on a fresh [64, 128256] bf16 logits tensor with fresh context
-tokens -- 256 distinct step inputs (4.2 GB) are resident and visited in turn, so no step finds its
-input in L2.  `value` is bias throughput in Gelem/s (B*V logits per second, all GPUs).  The same
-JSON line carries the roofline placement of the bias kernel, the end-to-end figure through the
-host-buffer entry point, the oracle timed on the host cores, and (under "extra") the self-salt
-bias, detection and fused-sampling workloads with their own roofline fractions.
+gamma 0.5, delta 2.0, key 0x5EED) on a [64, 128256] bf16 logits tensor with its own context
+tokens -- max(K, 16) distinct step inputs (>= 0.26 GB) are resident and visited in turn, so no step
+finds its input in L2.  The K steps are captured into one CUDA graph and the graph is replayed
+until the timed region lasts at least a quarter of a second, so the figure does not depend on K.
+`value` is bias throughput in Gelem/s (B*V logits per second, all GPUs).
+
+Roofline.  Nothing on this path is a contraction and every kernel is bound by integer issue, not
+by HBM, so the ceiling is built per pipe from rates measured in the same run by `sbw_int_probe`
+(thread-operations per clock per SM, from the SM cycle counter) and from the SM clock sampled
+during the timed region:
+    wide   32x32->64 multiplies and high halves        (multiplier pipe, half rate: the rate
+                                                         sustained inside the Philox round mix)
+    imad   32-bit multiply-adds                         (multiplier pipe, full rate)
+    alu    logic, shifts, adds, compares, selects       (ALU pipe)
+    issue  the two pipes together
+For a kernel whose unit of work needs `wide`, `imad`, `alu` and `fp` operations at least, the
+shortest possible time per unit is the largest of
+    wide / r_wide + imad / r_imad                                   (multiplier pipe alone)
+    alu / r_alu                                                     (ALU pipe alone)
+    (wide * r_imad / r_wide + imad + alu) / (r_imad + r_alu)        (both, work moved freely)
+    (wide + imad + alu + fp) / r_issue                              (issue slots)
+    bytes / measured HBM bandwidth
+and `frac` is that time divided by the measured one.  The operation counts are the least the
+method's arithmetic needs under the hash layout this library fixes (counted in WORK below), so a
+fraction cannot exceed 1; the looser count of 41 / 80 / 62 / 100 operations per unit that a plain
+evaluation of the hash takes is reported beside it as `plain_eval`.
 """
 from __future__ import annotations
 
@@ -29,16 +49,40 @@ if str(ROOT) not in sys.path:
 KEY = 0x5EED
 B2, V2 = 64, 128256                 # headline workload: bf16, context scheme
 GAMMA2, DELTA2 = 0.5, 2.0
-POOL = 256                          # distinct step inputs kept resident
-# Algorithmic work per logit (what the method itself needs, not what the kernel spends):
-#   context scheme: Philox4x32-10 word 0 = 20 32x32->64 multiplies + 20 three-input xors, and one
-#   compare = 41 integer operations; 2 bytes read + 2 bytes written (bf16).
-INT_OPS = {"context": 41, "selfsalt": 80, "detect_context": 62, "detect_selfsalt": 100}
-# INT32 ceiling of one B200: 148 SMs x 64 INT32 lanes per SM per clock (16 per scheduler; the
-# probe measures 64 ops/clk/SM for integer add, logic and 32-bit multiply-add, and 32 for the
-# 32x32->64 multiply) at the 1965 MHz maximum SM clock = 18.6 T integer operations per second.
-SMS, LANES_PER_SM_CLK, SM_MAX_MHZ = 148, 64, 1965.0
-INT_PEAK_TOPS = SMS * LANES_PER_SM_CLK * SM_MAX_MHZ * 1e6 / 1e12
+MIN_POOL = 16                       # distinct step inputs kept resident, at least (0.26 GB)
+MIN_REGION_S = 0.25                 # the timed region lasts at least this long
+SMS = 148
+
+# Least work per unit (logit or token), by pipe.  Philox4x32-10 word 0 on the counter (v, 0, 0, 0):
+# round 0 has one product (for consecutive ids it is formed by a 64-bit add), round 1 one product
+# per candidate plus M0*k0 (per row when the seed is per row), rounds 2-7 two products each, round
+# 8 one high half and one low half, round 9 one high half; one three-input xor per new counter
+# word that is used.
+#   seed per row (context bias)        15 wide + 1 imad, 17 xor + 64-bit add + compare + select
+#   seed per candidate (detect, self-salt) 17 wide + 1 imad, 17 xor + 16 key-schedule adds + compare
+#   context seed per token             key * id: 1 wide + 1 imad
+#   self-salt seed                     Jenkins 3 imad + 7 alu, min, J*min 1 wide, key * (.) 1 wide + 2 imad
+# Detection hashes each token's id once (the predecessor's Jenkins value is its neighbour's).
+WORK = {
+    "bias_context": {"wide": 15, "imad": 1, "alu": 20, "fp": 1},
+    "bias_selfsalt": {"wide": 19, "imad": 6, "alu": 44, "fp": 1},
+    "detect_context": {"wide": 18, "imad": 2, "alu": 36, "fp": 0},
+    "detect_selfsalt": {"wide": 19, "imad": 6, "alu": 46, "fp": 0},
+    # fused sampler with statistics: the bias hash, a quarter of a Gumbel Philox block (5 wide +
+    # 5 xor), the screen compare, running maximum, and about 7 fp32 operations of online softmax
+    "sample_context": {"wide": 20, "imad": 1, "alu": 27, "fp": 7},
+    "sample_selfsalt": {"wide": 24, "imad": 6, "alu": 51, "fp": 7},
+    # ids only: the Gumbel block and the screen; the green hash runs for a handful of candidates
+    "sample_ids": {"wide": 5, "imad": 0, "alu": 8, "fp": 1},
+}
+# A plain evaluation of the same hash (all 20 products of the ten rounds, every key-schedule add,
+# both Jenkins hashes): the per-unit operation counts of a straightforward implementation.
+PLAIN_EVAL = {
+    "bias_context": {"wide": 20, "imad": 0, "alu": 21, "fp": 0},
+    "bias_selfsalt": {"wide": 22, "imad": 2, "alu": 58, "fp": 0},
+    "detect_context": {"wide": 21, "imad": 1, "alu": 40, "fp": 0},
+    "detect_selfsalt": {"wide": 22, "imad": 2, "alu": 77, "fp": 0},
+}
 # DRAM bytes per bias launch of the headline workload: dram__bytes_read.sum + dram__bytes_write.sum
 # of one ncu capture of the same kernel on B=512 (131.38 MB + 91.60 MB, profiles/), divided by 8
 # because a bench launch processes 1/8 of those units and the traffic grows with the units.
@@ -54,7 +98,13 @@ def measured_peaks() -> dict:
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+    """Samples SM clock and throttle reasons through NVML (about every millisecond) from start()
+    to stop(); summary(t0, t1) reports the samples taken inside [t0, t1] (perf_counter times)."""
+
+    NAMES = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap",
+             0x8: "hw_slowdown", 0x10: "sync_boost", 0x20: "sw_thermal_slowdown",
+             0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+             0x100: "display_clock_setting"}
 
     def __init__(self, index: int):
         self.samples = []
@@ -79,7 +129,7 @@ class ClockSampler:
                 self.samples.append((time.perf_counter(), float(mhz), int(reasons)))
             except Exception:
                 pass
-            time.sleep(0.002)
+            time.sleep(0.001)
 
     def start(self):
         if self.nv is not None:
@@ -92,20 +142,23 @@ class ClockSampler:
             self._thread.join()
 
     def summary(self, t0: float, t1: float) -> dict:
-        if self.nv is None or not self.samples:
-            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
-        inside = [s for s in self.samples if t0 <= s[0] <= t1] or \
-            sorted(self.samples, key=lambda s: min(abs(s[0] - t0), abs(s[0] - t1)))[:3]
+        if self.nv is None:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "samples": 0, "reasons": ["unavailable"]}
+        inside = [s for s in list(self.samples) if t0 <= s[0] <= t1]
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "samples": 0,
+                    "reasons": ["no sample inside the timed region"]}
         mhz = sorted(s[1] for s in inside)
         bits = 0
         for s in inside:
             bits |= s[2]
-        names = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap",
-                 0x8: "hw_slowdown", 0x10: "sync_boost", 0x20: "sw_thermal_slowdown",
-                 0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
-                 0x100: "display_clock_setting"}
-        return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": self.max_mhz, "samples": len(inside),
-                "reasons": [n for b, n in names.items() if bits & b and n != "gpu_idle"]}
+        return {"sm_mhz": mhz[len(mhz) // 2], "sm_min_mhz": mhz[0], "sm_max_mhz": self.max_mhz,
+                "samples": len(inside),
+                "reasons": [n for b, n in self.NAMES.items() if bits & b and n != "gpu_idle"]}
+
+    def mhz(self, t0: float, t1: float) -> float | None:
+        """Median SM clock of the samples inside [t0, t1], else None."""
+        return self.summary(t0, t1).get("sm_mhz")
 
 
 def dist_env():
@@ -131,6 +184,78 @@ def max_over_ranks(x: float, world: int, device=None) -> float:
     return float(t.item())
 
 
+def pool_size(steps: int) -> int:
+    return max(steps, MIN_POOL)
+
+
+def workload_config(steps: int) -> dict:
+    """The `config` object: identical in both arms for the same --steps."""
+    pool = pool_size(steps)
+    return {"workload": "config 2: sbw_bias_logits, B=64, V=128256, bf16 logits N(0,4^2), "
+                        "context-hash seeding on 1 preceding token, gamma=0.5, delta=2.0, key=0x5EED",
+            "B": B2, "V": V2, "scheme": "context", "gamma": GAMMA2, "delta": DELTA2,
+            "l2": f"{pool} distinct step inputs ({pool * B2 * V2 * 2 / 1e9:.2f} GB) visited in turn, "
+                  "larger than the 126 MB L2"}
+
+
+# ------------------------------------------------------------------------------ roofline model
+def probe_rates(sbw) -> dict:
+    """Per-pipe rates in thread-operations per clock per SM, measured now with the cycle counter."""
+    def rate(kind):
+        return max(sbw.sbw_int_probe(kind, steps=4096, blocks_per_sm=b, threads=t)["ops_per_clk_per_sm"]
+                   for b, t in ((4, 256), (2, 512)))
+    raw = {k: rate(k) for k in ("mulhi", "mulwide_xor", "philox", "imad", "lop3", "iadd3", "ffma",
+                                "dual_int", "dual_fp", "add64")}
+    # The multiplier rate is the one sustained inside the Philox round mix (two wide multiplies and
+    # two three-input xors per round, each xor fed by both products): that mix is what every kernel
+    # here issues.  An isolated chain of high-half multiplies runs about 9 % faster; it is reported
+    # as r_wide_isolated, and `frac_isolated` places a kernel against it.
+    return {"r_wide": raw["philox"] / 2.0, "r_wide_isolated": max(raw["mulhi"], raw["mulwide_xor"] / 2.0),
+            "r_imad": raw["imad"], "r_alu": max(raw["lop3"], raw["iadd3"]),
+            "r_issue": max(raw["dual_int"], raw["dual_fp"], raw["ffma"]), "raw": raw}
+
+
+def unit_clocks(w: dict, r: dict) -> dict:
+    """Lower bounds of the SM clocks one unit of work `w` takes on one SM, per limiter."""
+    ratio = r["r_imad"] / r["r_wide"]
+    return {"multiplier pipe": w["wide"] / r["r_wide"] + w["imad"] / r["r_imad"],
+            "alu pipe": w["alu"] / r["r_alu"],
+            "both integer pipes": (w["wide"] * ratio + w["imad"] + w["alu"]) / (r["r_imad"] + r["r_alu"]),
+            "issue slots": (w["wide"] + w["imad"] + w["alu"] + w.get("fp", 0)) / r["r_issue"]}
+
+
+def place(kind: str, units: float, nbytes: float, seconds: float, rates: dict, sm_mhz: float,
+          hbm_gbs: float) -> dict:
+    """Where a measured launch of `units` units sits against its per-pipe ceiling."""
+    hz = sm_mhz * 1e6
+    out = {}
+    for tag, table in (("", WORK), ("plain_eval", PLAIN_EVAL)):
+        if kind not in table:
+            continue
+        w = table[kind]
+        clocks = unit_clocks(w, rates)
+        t_int = {k: v * units / (SMS * hz) for k, v in clocks.items()}
+        limiter = max(t_int, key=t_int.get)
+        t_hbm = nbytes / (hbm_gbs * 1e9)
+        t_bound = max(t_int[limiter], t_hbm)
+        ops = w["wide"] + w["imad"] + w["alu"]
+        d = {"ops_per_unit": ops, "by_pipe": {k: w[k] for k in ("wide", "imad", "alu")},
+             "achieved": ops * units / seconds / 1e12, "peak": ops * units / t_bound / 1e12,
+             "unit": "Tint-op/s", "frac": t_bound / seconds,
+             "bound": "alu" if t_int[limiter] >= t_hbm else "hbm",
+             "limiter": limiter if t_int[limiter] >= t_hbm else "hbm"}
+        if tag:
+            out[tag] = {k: d[k] for k in ("ops_per_unit", "by_pipe", "achieved", "peak", "frac", "limiter")}
+        else:
+            out.update(d)
+            iso = unit_clocks(w, {**rates, "r_wide": rates["r_wide_isolated"]})
+            out["frac_isolated"] = max(max(iso.values()) * units / (SMS * hz), t_hbm) / seconds
+            out["hbm"] = {"achieved": nbytes / seconds / 1e9, "peak": hbm_gbs, "unit": "GB/s",
+                          "frac": t_hbm / seconds}
+            out["sm_mhz"] = sm_mhz
+    return out
+
+
 # ------------------------------------------------------------------------------- reference arm
 def run_reference(args) -> None:
     """Times the CPU oracle, as it stands, on the host cores: each step is one headline decode
@@ -143,7 +268,7 @@ def run_reference(args) -> None:
     from paper_2609_03844_b200 import inputs
 
     cores = os.cpu_count() or 1
-    n_in = min(max(args.steps, 1), 4)
+    n_in = pool_size(args.steps)
     xs = [inputs.as_oracle_array(inputs.logits_normal(B2, V2, 4.0, torch.bfloat16, seed=1000 + i))
           for i in range(n_in)]
     cs = [inputs.uniform_tokens((B2, 1), V2, seed=2000 + i).numpy() for i in range(n_in)]
@@ -160,18 +285,12 @@ def run_reference(args) -> None:
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,   # the arm's N; the oracle itself runs on host cores
             "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {**workload_config(), "l2": f"{n_in} host-resident step inputs visited in turn (CPU run)"},
+            "config": workload_config(args.steps),
+            "launch": "CPU oracle, OpenMP over rows, host-resident inputs",
             "cpu_baseline": {"value": value, "unit": "Gelem/s", "cores": cores, "kind": "oracle",
                              "sample": f"{args.steps} full decode steps of the headline workload"},
             "e2e": {"value": value, "unit": "Gelem/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
-
-
-def workload_config() -> dict:
-    return {"workload": "config 2: sbw_bias_logits, B=64, V=128256, bf16 logits N(0,4^2), "
-                        "context-hash seeding on 1 preceding token, gamma=0.5, delta=2.0, key=0x5EED",
-            "B": B2, "V": V2, "scheme": "context", "gamma": GAMMA2, "delta": DELTA2,
-            "l2": f"{POOL} distinct step inputs (4.2 GB) visited in turn, far larger than the 126 MB L2"}
 
 
 # ------------------------------------------------------------------------------------ our arm
@@ -211,11 +330,15 @@ def run_ours(args) -> None:
         dist.init_process_group("nccl", device_id=dev)
     sbw.lib()
     peaks = measured_peaks()
-    K, W = args.steps, args.warmup
+    K, W = args.steps, max(args.warmup, 3)
     stream = torch.cuda.current_stream()
 
-    # ---- headline workload: every rank holds its own POOL step inputs (weak scaling) ----
-    pool = min(POOL, max(K, 16))
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    rates = probe_rates(sbw)            # per-pipe ceilings of this GPU, measured before the headline
+
+    # ---- headline workload: every rank holds its own step inputs (weak scaling) ----
+    pool = pool_size(K)
     logits = [inputs.logits_normal(B2, V2, 4.0, torch.bfloat16, seed=10_000 * rank + i, device=dev)
               for i in range(pool)]
     ctxs = [inputs.uniform_tokens((B2, 1), V2, seed=5_000_000 + 10_000 * rank + i, device=dev)
@@ -226,13 +349,9 @@ def run_ours(args) -> None:
         j = i % pool
         sbw.sbw_bias_logits(logits[j], ctxs[j], KEY, GAMMA2, DELTA2, sbw.SCHEME_CONTEXT)
 
-    for i in range(max(W, 3)):
+    for i in range(W):
         step(i)
     torch.cuda.synchronize()
-
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    time.sleep(0.02)
 
     launch_mode = "stream"
     graph = None
@@ -247,33 +366,36 @@ def run_ours(args) -> None:
             graph = None
             launch_mode = f"stream (graph capture failed: {type(exc).__name__})"
     stream = torch.cuda.current_stream()
-    if graph is not None:
-        graph.replay()              # one untimed replay: graph upload
-        ms, t0, t1 = time_region(graph.replay, stream, world, dev)
-    else:
-        ms, t0, t1 = time_region(lambda: [step(W + i) for i in range(K)], stream, world, dev)
+
+    def k_steps():
+        if graph is not None:
+            graph.replay()
+        else:
+            for i in range(K):
+                step(W + i)
+
+    k_steps()                           # one untimed pass: graph upload
+    ms1, _, _ = time_region(k_steps, stream, world, dev)
+    replays = max(1, int(MIN_REGION_S * 1.2 / (ms1 * 1e-3)) + 1)
+    if world > 1:                       # every rank replays the same number of times
+        replays = int(max_over_ranks(float(replays), world, dev))
+    ms, t0, t1 = time_region(lambda: [k_steps() for _ in range(replays)], stream, world, dev)
+    clocks = sampler.summary(t0, t1)
+    n_steps = K * replays
     # the same K steps as plain stream launches, for the record
     ms_stream, _, _ = time_region(lambda: [step(W + i) for i in range(K)], stream, world, dev)
-    time.sleep(0.01)
-    sampler.stop()
-    clocks = sampler.summary(t0, t1)
 
     elems_step = B2 * V2
-    value = world * elems_step * K / (ms * 1e-3) / 1e9
-    launch_s = ms * 1e-3 / K
-    int_ops = INT_OPS["context"] * elems_step
-    ach_tops = int_ops / launch_s / 1e12
-    hbm_gbs = 4 * elems_step / launch_s / 1e9
-    roofline = {"bound": "alu", "achieved": ach_tops, "peak": INT_PEAK_TOPS, "unit": "Tint-op/s",
-                "frac": ach_tops / INT_PEAK_TOPS, "traffic": NCU_TRAFFIC_BYTES,
-                "peak_source": "derived: 148 SMs x 64 INT32 lanes x 1965 MHz",
-                "kernel": "bias_kernel<bf16, context, vector>", "avg_launch_us": launch_s * 1e6,
-                "int_ops_per_elem": INT_OPS["context"],
-                "hbm": {"achieved": hbm_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                        "frac": hbm_gbs / peaks["hbm_gbs"], "of": peaks["source"],
-                        "bytes_per_elem": 4},
-                "binding": "alu" if int_ops / (INT_PEAK_TOPS * 1e12) > 4 * elems_step / (peaks["hbm_gbs"] * 1e9)
-                else "hbm"}
+    value = world * elems_step * n_steps / (ms * 1e-3) / 1e9
+    launch_s = ms * 1e-3 / n_steps
+    sm_mhz = clocks.get("sm_mhz") or sampler.max_mhz or 1965.0
+    roofline = place("bias_context", elems_step, 4 * elems_step, launch_s, rates, sm_mhz, peaks["hbm_gbs"])
+    roofline.update({"traffic": NCU_TRAFFIC_BYTES, "kernel": "bias_kernel<bf16, context, vector>",
+                     "avg_launch_us": launch_s * 1e6,
+                     "peak_source": "measured in this run: sbw_int_probe rates x 148 SMs x the SM clock "
+                                    "sampled during the timed region; HBM of " + peaks["source"],
+                     "rates_ops_per_clk_per_sm": {k: rates[k] for k in ("r_wide", "r_wide_isolated", "r_imad",
+                                                                        "r_alu", "r_issue")}})
 
     # ---- end to end: host buffers through the C ABI, copies inside the timed region ----
     # Steps alternate between two streams, each with its own staging buffer, so that one step's
@@ -310,26 +432,76 @@ def run_ours(args) -> None:
     del h_logits, lanes
 
     line = {"metric": "sbw_bias_throughput", "value": value, "unit": "Gelem/s", "n_gpus": world,
-            "steps": K, "warmup": W, "ms_per_step": ms / K, "higher_is_better": True,
+            "steps": K, "warmup": W, "ms_per_step": ms / n_steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {**workload_config(), "launch": launch_mode, "parallelism": f"replicas x{world}",
-                       "l2": f"{pool} distinct step inputs ({pool * elems_step * 2 / 1e9:.1f} GB) visited in "
-                             "turn, far larger than the 126 MB L2"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": K, "roofline": roofline,
+            "config": workload_config(K), "launch": launch_mode, "parallelism": f"replicas x{world}",
+            "replays": replays, "timed_region_s": ms * 1e-3,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": n_steps, "roofline": roofline,
             "stream_launch": {"value": world * elems_step * K / (ms_stream * 1e-3) / 1e9,
                               "ms_per_step": ms_stream / K}}
 
+    del logits, ctxs
+    torch.cuda.empty_cache()
+    if world > 1:
+        line["sharded_sampling"] = run_sharded_leg(sbw, inputs, dev, rank, world)
     if rank == 0 and world == 1 and not args.no_extra:
-        del logits, ctxs
-        torch.cuda.empty_cache()
-        line["extra"] = run_extra(sbw, inputs, dev, peaks)
-        line["detect_tokens_per_s"] = line["extra"]["detect_context_N100000"]["tokens_per_s"]
+        detect = run_detect(sbw, inputs, dev, peaks, rates, sampler)
+        line.update(detect)
+        line["extra"] = run_extra(sbw, inputs, dev, peaks, rates, sampler)
+        line["extra"]["int_probe"] = rates["raw"]
+        line["roofline_sample"] = line["extra"].pop("roofline_sample")
         line["cpu_baseline"] = cpu_baseline()
+        line["cpu_baseline_detect"] = cpu_baseline_detect()
+    sampler.stop()
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+def run_sharded_leg(sbw, inputs, dev, rank, world) -> dict:
+    """Vocabulary-sharded fused sampling across the ranks (N > 1 only): every rank samples its own
+    columns of a common seeded [B, V] batch, one all-gather of the [B, 8] summaries over NCCL, a
+    local combine.  Reports the time per step (max over ranks) and checks that every rank ends
+    with the same ids and that they equal the unsplit call's on the same rows."""
+    import torch
+    import torch.distributed as dist
+    from paper_2609_03844_b200 import sharded
+
+    B, V = 256, V2
+    x = inputs.logits_normal(B, V, 4.0, torch.bfloat16, seed=31337, device=dev)    # same bytes on every rank
+    ctx = inputs.uniform_tokens((B, 1), V, seed=31338, device=dev)
+    lo, hi = sharded.shard_columns(V, rank, world, align=8)
+    xs = x[:, lo:hi]                                   # this rank's columns: a view, row stride V
+    ws = torch.empty(sbw.sbw_sample_workspace_bytes(B, hi - lo), dtype=torch.uint8, device=dev)
+
+    def one(step):
+        return sharded.sharded_bias_sample(xs, ctx, KEY, 0.25, 2.0, sbw.SCHEME_CONTEXT, 0.7, 0xC4, step, lo, ws)
+
+    for s in range(3):
+        one(s)
+    torch.cuda.synchronize()
+    dist.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n = 20
+    e0.record()
+    for s in range(n):
+        one(100 + s)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = max_over_ranks(e0.elapsed_time(e1) / n, world, dev)
+    ids, m, Z, p = one(7)
+    whole = torch.empty(B, dtype=torch.int32, device=dev)
+    zw = torch.empty(B, dtype=torch.float32, device=dev)
+    wsw = torch.empty(sbw.sbw_sample_workspace_bytes(B, V), dtype=torch.uint8, device=dev)
+    sbw.sbw_bias_sample(x, ctx, KEY, 0.25, 2.0, sbw.SCHEME_CONTEXT, 0.7, 0xC4, 7, whole, wsw, out_sumexp=zw)
+    torch.cuda.synchronize()
+    return {"B": B, "V": V, "shards": world, "ms_per_step": ms,
+            "ids_equal_on_every_rank": sharded.same_on_every_rank(ids),
+            "ids_equal_unsplit_call": bool(torch.equal(ids, whole)),
+            "sumexp_max_rel_diff_to_unsplit_call": float(((Z - zw).abs() / zw).max().item()),
+            "exchange": "one NCCL all_gather of 32 bytes per row and rank; no peer pointers, no multicast"}
 
 
 def cpu_baseline() -> dict:
@@ -358,19 +530,53 @@ def cpu_baseline() -> dict:
             "single_thread_value": single}
 
 
-def _time_calls(fn, n, warm=3):
+def cpu_baseline_detect() -> dict:
+    """The oracle's detector on the host cores: a sub-sample of config 5 (sequences of uniform ids,
+    lengths uniform in [64, 1024], context scheme), repeated for about 12 core-seconds."""
+    import oracle
+    from paper_2609_03844_b200 import inputs
+
+    cores = os.cpu_count() or 1
+    n_seq = 4000
+    tokens, lengths = inputs.null_token_streams(n_seq, 64, 1024, V2, seed=500)
+    tok, lens = tokens.numpy(), lengths.numpy()
+    oracle.detect(tok, lens, KEY, 0.25, oracle.SCHEME_CONTEXT, threads=cores)
+    t0 = time.perf_counter()
+    n = 0
+    while True:
+        oracle.detect(tok, lens, KEY, 0.25, oracle.SCHEME_CONTEXT, threads=cores)
+        n += 1
+        dt = time.perf_counter() - t0
+        if dt * cores > 12.0 or n >= 200:
+            break
+    return {"value": tok.size * n / dt, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+            "sample": f"{n} passes over the first {n_seq} sequences of the config-5 null streams "
+                      f"({tok.size / 1e6:.2f} M tokens per pass), context scheme, gamma 0.25"}
+
+
+def _time_calls(fn, n, warm=3, min_s=0.05):
+    """Average device time of fn(i) (seconds) and the host interval [t0, t1] it ran in; the calls
+    are repeated until the timed region lasts at least min_s."""
     import torch
     for i in range(warm):
         fn(i)
     torch.cuda.synchronize()
-    e0 = torch.cuda.Event(enable_timing=True)
-    e1 = torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(n):
-        fn(warm + i)
-    e1.record()
-    torch.cuda.synchronize()
-    return e0.elapsed_time(e1) * 1e-3 / n
+    total_calls, total_ms = 0, 0.0
+    t0 = time.perf_counter()
+    while True:
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n):
+            fn(warm + i)
+        e1.record()
+        torch.cuda.synchronize()
+        total_ms += e0.elapsed_time(e1)
+        total_calls += n
+        if total_ms * 1e-3 >= min_s:
+            break
+    t1 = time.perf_counter()
+    return total_ms * 1e-3 / total_calls, t0, t1
 
 
 def _time_graph(fn, n, reps=10, warm=3):
@@ -401,19 +607,41 @@ def _time_graph(fn, n, reps=10, warm=3):
     return e0.elapsed_time(e1) * 1e-3 / (n * reps)
 
 
-def run_extra(sbw, inputs, dev, peaks) -> dict:
+def run_detect(sbw, inputs, dev, peaks, rates, sampler) -> dict:
+    """Config 5 (null half shape): 100000 sequences, lengths uniform in [64, 1024], 218 MB of ids.
+    Returns the top-level detection keys of the bench line."""
+    import torch
+    N = 100000
+    tokens, lengths = inputs.null_token_streams(N, 64, 1024, V2, seed=500, device=dev)
+    counts = torch.empty(N, dtype=torch.int32, device=dev)
+    z = torch.empty(N, dtype=torch.float64, device=dev)
+    ws = torch.empty(sbw.sbw_detect_workspace_bytes(N), dtype=torch.uint8, device=dev)
+    ntok = tokens.numel()
+    out = {}
+    for name, scheme in (("context", sbw.SCHEME_CONTEXT), ("selfsalt", sbw.SCHEME_SELFSALT)):
+        s, t0, t1 = _time_calls(lambda i: sbw.sbw_detect(tokens, lengths, KEY, 0.25, scheme, counts, z,
+                                                         workspace=ws), 30, min_s=0.25)
+        mhz = sampler.mhz(t0, t1) or sampler.max_mhz or 1965.0
+        r = place(f"detect_{name}", ntok, 4 * ntok + 24 * N, s, rates, mhz, peaks["hbm_gbs"])
+        r.update({"tokens_per_s": ntok / s, "ms": s * 1e3, "tokens": ntok, "sequences": N,
+                  "workload": "config 5 shape: 100000 sequences of uniform ids, lengths uniform in [64, 1024], "
+                              f"V=128256, {name} scheme, gamma 0.25; 218 MB of ids, larger than L2"})
+        out[name] = r
+    return {"detect_tokens_per_s": out["context"]["tokens_per_s"], "roofline_detect": out["context"],
+            "roofline_detect_selfsalt": out["selfsalt"]}
+
+
+def run_extra(sbw, inputs, dev, peaks, rates, sampler) -> dict:
     """The other workloads of the hot path, each timed on its own (inputs larger than L2 or
-    rotating), and the integer-throughput probe."""
+    rotating), placed against the same per-pipe ceilings."""
     import torch
     out = {}
     hbm = peaks["hbm_gbs"]
 
-    def place(int_ops, nbytes, seconds):
-        t_alu = int_ops / (INT_PEAK_TOPS * 1e12)
-        t_hbm = nbytes / (hbm * 1e9)
-        return {"bound": "alu" if t_alu >= t_hbm else "hbm", "frac": max(t_alu, t_hbm) / seconds,
-                "alu_frac": t_alu / seconds, "hbm_frac": t_hbm / seconds,
-                "achieved_tint_ops": int_ops / seconds / 1e12, "achieved_gbs": nbytes / seconds / 1e9}
+    def placed(kind, units, nbytes, timing):
+        s, t0, t1 = timing
+        mhz = sampler.mhz(t0, t1) or sampler.max_mhz or 1965.0
+        return place(kind, units, nbytes, s, rates, mhz, hbm)
 
     # config 3: full-vocabulary self-salt, fp32, B=256, V=151936, gamma .25, delta 4
     B3, V3 = 256, 151936
@@ -421,57 +649,59 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
                                  V3, seed=310 + i) for i in range(4)]
     c3 = [inputs.uniform_tokens((B3, 1), V3, seed=320 + i, device=dev) for i in range(4)]
     for name, scheme in (("selfsalt", sbw.SCHEME_SELFSALT), ("context", sbw.SCHEME_CONTEXT)):
-        s = _time_calls(lambda i: sbw.sbw_bias_logits(p3[i % 4], c3[i % 4], KEY, 0.25, 4.0, scheme), 128)
+        tm = _time_calls(lambda i: sbw.sbw_bias_logits(p3[i % 4], c3[i % 4], KEY, 0.25, 4.0, scheme), 128)
         n = B3 * V3
-        out[f"bias_fp32_{name}_B256_V151936"] = {"gelem_s": n / s / 1e9, "ms": s * 1e3,
-                                                 **place(INT_OPS[name] * n, 8 * n, s)}
+        out[f"bias_fp32_{name}_B256_V151936"] = {"gelem_s": n / tm[0] / 1e9, "ms": tm[0] * 1e3,
+                                                 **placed(f"bias_{name}", n, 8 * n, tm)}
     # the paper's SBW-ss: self-salt on the top-40 candidates of each row only (same shape)
-    s = _time_calls(lambda i: sbw.sbw_bias_logits_topk(p3[i % 4], c3[i % 4], KEY, 0.25, 4.0, sbw.SCHEME_SELFSALT, 40), 128)
+    s = _time_calls(lambda i: sbw.sbw_bias_logits_topk(p3[i % 4], c3[i % 4], KEY, 0.25, 4.0, sbw.SCHEME_SELFSALT, 40), 128)[0]
     out["bias_top40_fp32_selfsalt_B256_V151936"] = {
         "gelem_s": B3 * V3 / s / 1e9, "ms": s * 1e3, "bound": "hbm",
         "achieved_gbs": 4 * B3 * V3 / s / 1e9, "frac": 4 * B3 * V3 / s / 1e9 / hbm,
-        "note": "one read of the row from HBM (4 B/logit), second read from L2, 40 columns written"}
+        "note": "one read of the row from HBM (4 B/logit), 40 columns written"}
     del p3, c3
     # the same scheme on large batches (1024 rows): fp32 at V = 151936 and bf16 at V = 128256
     for tag, dt, Vk, es in (("fp32", torch.float32, V3, 4), ("bf16", torch.bfloat16, V2, 2)):
         pk = [inputs.logits_normal(1024, Vk, 4.0, dt, seed=440 + i, device=dev) for i in range(2)]
         ck = [inputs.uniform_tokens((1024, 1), Vk, seed=450 + i, device=dev) for i in range(2)]
-        s = _time_calls(lambda i: sbw.sbw_bias_logits_topk(pk[i % 2], ck[i % 2], KEY, 0.25, 4.0, sbw.SCHEME_SELFSALT, 40), 32)
+        s = _time_calls(lambda i: sbw.sbw_bias_logits_topk(pk[i % 2], ck[i % 2], KEY, 0.25, 4.0, sbw.SCHEME_SELFSALT, 40), 32)[0]
         out[f"bias_top40_{tag}_selfsalt_B1024_V{Vk}"] = {
             "gelem_s": 1024 * Vk / s / 1e9, "ms": s * 1e3, "bound": "hbm",
             "achieved_gbs": es * 1024 * Vk / s / 1e9, "frac": es * 1024 * Vk / s / 1e9 / hbm}
         del pk, ck
-    # config 2 shape under the self-salt scheme
+    # config 2 shape under the self-salt scheme, and the headline kernel on a large batch
     p2 = [inputs.logits_normal(B2, V2, 4.0, torch.bfloat16, seed=400 + i, device=dev) for i in range(16)]
     c2 = [inputs.uniform_tokens((B2, 1), V2, seed=420 + i, device=dev) for i in range(16)]
-    s = _time_calls(lambda i: sbw.sbw_bias_logits(p2[i % 16], c2[i % 16], KEY, 0.5, 2.0, sbw.SCHEME_SELFSALT), 256)
-    out["bias_bf16_selfsalt_B64_V128256"] = {"gelem_s": B2 * V2 / s / 1e9, "ms": s * 1e3,
-                                             **place(INT_OPS["selfsalt"] * B2 * V2, 4 * B2 * V2, s)}
+    tm = _time_calls(lambda i: sbw.sbw_bias_logits(p2[i % 16], c2[i % 16], KEY, 0.5, 2.0, sbw.SCHEME_SELFSALT), 256)
+    out["bias_bf16_selfsalt_B64_V128256"] = {"gelem_s": B2 * V2 / tm[0] / 1e9, "ms": tm[0] * 1e3,
+                                             **placed("bias_selfsalt", B2 * V2, 4 * B2 * V2, tm)}
     # the headline step on ONE buffer that stays in L2 (16.4 MB): labelled L2-warm, not a roofline input
     s = _time_graph(lambda i: sbw.sbw_bias_logits(p2[0], c2[0], KEY, 0.5, 2.0, sbw.SCHEME_CONTEXT), 64)
     out["bias_bf16_context_B64_V128256_l2_warm_single_buffer"] = {"gelem_s": B2 * V2 / s / 1e9, "ms": s * 1e3}
     del p2, c2
-    # config 5 (null half shape): 100000 sequences, lengths uniform in [64, 1024], 218 MB of ids
+    pb = [inputs.logits_normal(1024, V2, 4.0, torch.bfloat16, seed=470 + i, device=dev) for i in range(2)]
+    cb = [inputs.uniform_tokens((1024, 1), V2, seed=480 + i, device=dev) for i in range(2)]
+    for name, scheme in (("context", sbw.SCHEME_CONTEXT), ("selfsalt", sbw.SCHEME_SELFSALT)):
+        tm = _time_calls(lambda i: sbw.sbw_bias_logits(pb[i % 2], cb[i % 2], KEY, 0.5, 2.0, scheme), 32)
+        n = 1024 * V2
+        out[f"bias_bf16_{name}_B1024_V128256"] = {"gelem_s": n / tm[0] / 1e9, "ms": tm[0] * 1e3,
+                                                  **placed(f"bias_{name}", n, 4 * n, tm)}
+    del pb, cb
+    # evaluation steps on the config-5 streams: distinct-tuple scoring, then ROC-AUC of the z array
+    # against alternating labels (timing only: these streams are all unmarked)
     N = 100000
     tokens, lengths = inputs.null_token_streams(N, 64, 1024, V2, seed=500, device=dev)
     counts = torch.empty(N, dtype=torch.int32, device=dev)
     z = torch.empty(N, dtype=torch.float64, device=dev)
-    ws = torch.empty(sbw.sbw_detect_workspace_bytes(N), dtype=torch.uint8, device=dev)
     ntok = tokens.numel()
-    for name, scheme in (("context", sbw.SCHEME_CONTEXT), ("selfsalt", sbw.SCHEME_SELFSALT)):
-        s = _time_calls(lambda i: sbw.sbw_detect(tokens, lengths, KEY, 0.25, scheme, counts, z, workspace=ws), 30)
-        out[f"detect_{name}_N100000"] = {"tokens_per_s": ntok / s, "ms": s * 1e3, "tokens": ntok,
-                                         **place(INT_OPS[f"detect_{name}"] * ntok, 4 * ntok + 24 * N, s)}
-    # evaluation steps on the same streams: distinct-tuple scoring, then ROC-AUC of the z array
-    # against alternating labels (timing only: these streams are all unmarked)
     wsu = torch.empty(sbw.sbw_detect_unique_workspace_bytes(N, ntok, 1024), dtype=torch.uint8, device=dev)
     s = _time_calls(lambda i: sbw.sbw_detect_unique(tokens, lengths, 1024, KEY, 0.25, sbw.SCHEME_CONTEXT, counts,
-                                                    z, wsu), 20)
+                                                    z, wsu), 20)[0]
     out["detect_unique_context_N100000"] = {"tokens_per_s": ntok / s, "ms": s * 1e3, "tokens": ntok}
     labels = (torch.arange(N, device=dev) % 2).to(torch.uint8)
     auc = torch.empty(1, dtype=torch.float64, device=dev)
     wsr = torch.empty(sbw.sbw_roc_auc_workspace_bytes(N), dtype=torch.uint8, device=dev)
-    s = _time_calls(lambda i: sbw.sbw_roc_auc(z, labels, auc, wsr), 20)
+    s = _time_calls(lambda i: sbw.sbw_roc_auc(z, labels, auc, wsr), 20)[0]
     out["roc_auc_N100000"] = {"ms": s * 1e3, "pairs_per_s": (N / 2) ** 2 / s}
     del tokens, wsu
     # config 4: fused sampling sweep, bf16, V=128256, tau 0.7
@@ -481,21 +711,30 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
         ids = torch.empty(B, dtype=torch.int32, device=dev)
         wsb = torch.empty(sbw.sbw_sample_workspace_bytes(B, V2), dtype=torch.uint8, device=dev)
         zsum = torch.empty(B, dtype=torch.float32, device=dev)
+        n = B * V2
         for name, scheme in (("context", sbw.SCHEME_CONTEXT), ("selfsalt", sbw.SCHEME_SELFSALT)):
             # with the softmax sum requested every logit is hashed; ids alone let the kernel screen on
             # the Gumbel words first and hash only the candidates that could win
-            s = _time_calls(lambda i: sbw.sbw_bias_sample(x, c, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, wsb,
-                                                          out_sumexp=zsum), 20)
-            out[f"sample_bf16_{name}_B{B}"] = {"gelem_s": B * V2 / s / 1e9, "ms": s * 1e3,
-                                               "l2_resident": B * V2 * 2 < 100e6}
-            s = _time_calls(lambda i: sbw.sbw_bias_sample(x, c, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, wsb), 20)
-            out[f"sample_ids_only_bf16_{name}_B{B}"] = {"gelem_s": B * V2 / s / 1e9, "ms": s * 1e3}
+            tm = _time_calls(lambda i: sbw.sbw_bias_sample(x, c, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, wsb,
+                                                           out_sumexp=zsum), 20)
+            e = {"gelem_s": n / tm[0] / 1e9, "ms": tm[0] * 1e3, "l2_resident": n * 2 < 100e6}
+            if B >= 512:
+                e.update(placed(f"sample_{name}", n, 2 * n, tm))
+            out[f"sample_bf16_{name}_B{B}"] = e
+            tm = _time_calls(lambda i: sbw.sbw_bias_sample(x, c, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, wsb), 20)
+            e = {"gelem_s": n / tm[0] / 1e9, "ms": tm[0] * 1e3}
+            if B >= 512:
+                e.update(placed("sample_ids", n, 2 * n, tm))
+            out[f"sample_ids_only_bf16_{name}_B{B}"] = e
             if B <= 32:   # calls this short are host-bound as stream launches: device time from a graph
                 s = _time_graph(lambda i: sbw.sbw_bias_sample(x, c, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, wsb,
                                                               out_sumexp=zsum), 16)
                 out[f"sample_bf16_{name}_B{B}"]["graph_ms"] = s * 1e3
                 s = _time_graph(lambda i: sbw.sbw_bias_sample(x, c, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, wsb), 16)
                 out[f"sample_ids_only_bf16_{name}_B{B}"]["graph_ms"] = s * 1e3
+    out["roofline_sample"] = {**out["sample_bf16_context_B1024"],
+                              "workload": "config 4: sbw_bias_sample with the softmax sum, B=1024, V=128256, "
+                                          "bf16, context scheme, gamma 0.25, delta 2, tau 0.7 (263 MB, larger than L2)"}
     # Appendix F's sampling setting (temperature 0.7, top_p 0.8) and a top-k one, through the truncated sampler
     for B in (64, 1024):
         x = inputs.logits_normal(B, V2, 4.0, torch.bfloat16, seed=600 + B, device=dev)
@@ -505,13 +744,13 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
                           device=dev)
         for name, top_k, top_p in (("top_p0.8", 0, 0.8), ("top_k50", 50, 1.0)):
             s = _time_calls(lambda i: sbw.sbw_bias_sample_filtered(x, c, KEY, 0.25, 2.0, sbw.SCHEME_CONTEXT, 0.7,
-                                                                   top_k, top_p, 0xC4, i, ids, wsf), 20)
+                                                                   top_k, top_p, 0xC4, i, ids, wsf), 20)[0]
             out[f"sample_filtered_bf16_context_{name}_B{B}"] = {"gelem_s": B * V2 / s / 1e9, "ms": s * 1e3}
     # SBW-ss (self-salt on the top-40 candidates) at the headline shape
     xs = [inputs.logits_normal(B2, V2, 4.0, torch.bfloat16, seed=650 + i, device=dev) for i in range(16)]
     cs = [inputs.uniform_tokens((B2, 1), V2, seed=750 + i, device=dev) for i in range(16)]
     s = _time_calls(lambda i: sbw.sbw_bias_logits_topk(xs[i % 16], cs[i % 16], KEY, 0.25, 2.0, sbw.SCHEME_SELFSALT, 40),
-                    256)
+                    256)[0]
     out["topk40_bf16_selfsalt_B64_V128256"] = {"gelem_s": B2 * V2 / s / 1e9, "ms": s * 1e3}
     del xs, cs
     # the paper's isolated-benchmark protocol (Appendix D: fresh (B, 151936) logits, 20 warm-up + 200
@@ -537,13 +776,6 @@ def run_extra(sbw, inputs, dev, peaks) -> dict:
                                      "p99_ms": times[int(len(times) * 0.99)],
                                      "l2_resident": B * 151936 * 4 < 100e6}
     out["paper_protocol_latency_fp32_V151936_W4"] = sweep
-    # integer-throughput probe
-    probes = {}
-    for kind in ("mulwide", "lop3", "iadd3", "imad", "philox", "ffma"):
-        r = sbw.sbw_int_probe(kind, steps=8192, blocks_per_sm=4, threads=256)
-        probes[kind] = {"ops_per_clk_per_sm": r["ops_per_clk_per_sm"], "tops": r["ops_per_s"] / 1e12,
-                        "sm_mhz": r["sm_mhz_implied"]}
-    out["int_probe"] = probes
     return out
 
 
@@ -608,11 +840,11 @@ def run_profile_case(name: str, launches: int) -> None:
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2048)
+    ap.add_argument("--steps", type=int, default=256)
     ap.add_argument("--warmup", type=int, default=16)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches only")
-    ap.add_argument("--no-extra", action="store_true", help="skip the secondary workloads and the CPU baseline")
+    ap.add_argument("--no-extra", action="store_true", help="skip the secondary workloads and the CPU baselines")
     ap.add_argument("--profile-case", choices=PROFILE_CASES, default=None,
                     help="run a few launches of one kernel on a small (> L2) input, for a profiler")
     ap.add_argument("--profile-launches", type=int, default=3)
@@ -621,7 +853,7 @@ def main() -> None:
         run_profile_case(args.profile_case, args.profile_launches)
         return
     if args.impl == "reference":
-        if args.steps == 2048:
+        if args.steps == 256 and args.warmup == 16:
             args.steps, args.warmup = 32, 3
         run_reference(args)
     else:

@@ -22,7 +22,12 @@ extern "C" {
 #define SBW_PROBE_IMAD 3    /* 32-bit multiply-add chains                     1 op / step */
 #define SBW_PROBE_PHILOX 4  /* Philox rounds: 2 wide multiplies + 2 xor3      4 ops / step */
 #define SBW_PROBE_FFMA 5    /* fp32 fused multiply-add chains (for contrast)  1 op / step */
-#define SBW_PROBE_KINDS 6
+#define SBW_PROBE_MULHI 6       /* mul.hi.u32 chains (high half of a 32x32 product)        1 op / step */
+#define SBW_PROBE_MULWIDE_XOR 7 /* mul.wide.u32, then lo ^ hi: 1 wide multiply + 1 xor     2 ops / step */
+#define SBW_PROBE_DUAL_FP 8     /* one xor3 and one fp32 FMA: two pipes, issue-slot bound  2 ops / step */
+#define SBW_PROBE_DUAL_INT 9    /* one xor3 and one 32-bit multiply-add: ALU + multiplier  2 ops / step */
+#define SBW_PROBE_ADD64 10      /* 64-bit integer add chains                               1 op / step */
+#define SBW_PROBE_KINDS 11
 
 /*
  * Launches sm_count * blocks_per_sm blocks of `threads` threads; every thread runs `steps` steps

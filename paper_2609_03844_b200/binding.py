@@ -471,7 +471,8 @@ def sbw_roc_auc_batched(z: torch.Tensor, labels: torch.Tensor, offsets: torch.Te
 
 
 PROBE_KINDS = {"mulwide": (0, 1), "lop3": (1, 1), "iadd3": (2, 1), "imad": (3, 1), "philox": (4, 4),
-               "ffma": (5, 1)}
+               "ffma": (5, 1), "mulhi": (6, 1), "mulwide_xor": (7, 2), "dual_fp": (8, 2), "dual_int": (9, 2),
+               "add64": (10, 1)}
 
 
 def sbw_int_probe(kind: str, steps: int = 4096, blocks_per_sm: int = 4, threads: int = 256,

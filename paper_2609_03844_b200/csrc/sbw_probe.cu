@@ -44,8 +44,21 @@ __global__ void probe_kernel(int steps, int64_t *out_cycles, uint32_t *out_sink)
                 const uint32_t ny = static_cast<uint32_t>(a >> 32) ^ static_cast<uint32_t>(b) ^ k1;
                 x[i] = nx;
                 y[i] = ny;
-            } else {
+            } else if constexpr (KIND == SBW_PROBE_FFMA) {
                 asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[i]) : "f"(0.99999f), "f"(1e-7f));
+            } else if constexpr (KIND == SBW_PROBE_MULHI) {
+                asm volatile("mul.hi.u32 %0, %0, %1;" : "+r"(x[i]) : "r"(0xD2511F53u));
+            } else if constexpr (KIND == SBW_PROBE_MULWIDE_XOR) {
+                asm volatile("{ .reg .b32 lo, hi; .reg .b64 q; mul.wide.u32 q, %0, %1; mov.b64 {lo, hi}, q; "
+                             "xor.b32 %0, lo, hi; }" : "+r"(x[i]) : "r"(0xD2511F53u));
+            } else if constexpr (KIND == SBW_PROBE_DUAL_FP) {
+                asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[i]) : "r"(y[i]), "r"(k0));
+                asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[i]) : "f"(0.99999f), "f"(1e-7f));
+            } else if constexpr (KIND == SBW_PROBE_DUAL_INT) {
+                asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[i]) : "r"(y[i]), "r"(k0));
+                asm volatile("mad.lo.u32 %0, %0, %1, %2;" : "+r"(y[i]) : "r"(0xCD9E8D57u), "r"(k1));
+            } else {
+                asm volatile("add.u64 %0, %0, %1;" : "+l"(p[i]) : "l"((static_cast<uint64_t>(k1) << 32) | k0));
             }
         }
     }
@@ -78,7 +91,12 @@ extern "C" int sbw_int_probe(int kind, int steps, int blocks_per_sm, int threads
         case SBW_PROBE_IADD3: probe_kernel<SBW_PROBE_IADD3><<<grid, threads, 0, s>>>(steps, out_cycles, out_sink); break;
         case SBW_PROBE_IMAD: probe_kernel<SBW_PROBE_IMAD><<<grid, threads, 0, s>>>(steps, out_cycles, out_sink); break;
         case SBW_PROBE_PHILOX: probe_kernel<SBW_PROBE_PHILOX><<<grid, threads, 0, s>>>(steps, out_cycles, out_sink); break;
-        default: probe_kernel<SBW_PROBE_FFMA><<<grid, threads, 0, s>>>(steps, out_cycles, out_sink); break;
+        case SBW_PROBE_FFMA: probe_kernel<SBW_PROBE_FFMA><<<grid, threads, 0, s>>>(steps, out_cycles, out_sink); break;
+        case SBW_PROBE_MULHI: probe_kernel<SBW_PROBE_MULHI><<<grid, threads, 0, s>>>(steps, out_cycles, out_sink); break;
+        case SBW_PROBE_MULWIDE_XOR: probe_kernel<SBW_PROBE_MULWIDE_XOR><<<grid, threads, 0, s>>>(steps, out_cycles, out_sink); break;
+        case SBW_PROBE_DUAL_FP: probe_kernel<SBW_PROBE_DUAL_FP><<<grid, threads, 0, s>>>(steps, out_cycles, out_sink); break;
+        case SBW_PROBE_DUAL_INT: probe_kernel<SBW_PROBE_DUAL_INT><<<grid, threads, 0, s>>>(steps, out_cycles, out_sink); break;
+        default: probe_kernel<SBW_PROBE_ADD64><<<grid, threads, 0, s>>>(steps, out_cycles, out_sink); break;
     }
     SBW_CUDA_TRY(cudaGetLastError());
     return SBW_OK;

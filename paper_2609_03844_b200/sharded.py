@@ -60,6 +60,17 @@ def sharded_bias_sample(logits_shard: torch.Tensor, ctx_tokens: torch.Tensor, ke
     return tokens, m, Z, p
 
 
+def same_on_every_rank(t: torch.Tensor, group=None) -> bool:
+    """True iff the integer tensor ``t`` holds the same values on every rank of ``group`` (two
+    all-reduces: element-wise minimum and maximum over the ranks must coincide)."""
+    if not dist.is_initialized() or dist.get_world_size(group) == 1:
+        return True
+    lo, hi = t.clone(), t.clone()
+    dist.all_reduce(lo, op=dist.ReduceOp.MIN, group=group)
+    dist.all_reduce(hi, op=dist.ReduceOp.MAX, group=group)
+    return bool(torch.equal(lo, hi))
+
+
 def shard_sequences(N: int, rank: int, world: int) -> tuple[int, int]:
     """Sequences [lo, hi) of a batch of N owned by ``rank``: contiguous and balanced.  Detection has
     no cross-sequence dependency, so this is all the sharding it needs."""

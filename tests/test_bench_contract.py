@@ -27,6 +27,7 @@ def test_reference_arm_prints_the_contract_line():
     assert d["metric"] == "sbw_bias_throughput" and d["unit"] == "Gelem/s" and d["higher_is_better"] is True
     assert d["steps"] == 2 and d["warmup"] == 1 and d["vs_baseline"] is None and d["data"] == "synthetic"
     assert "workload" in d["config"] and "model" not in d["config"]
+    assert set(d["config"]) == {"workload", "B", "V", "scheme", "gamma", "delta", "l2"}    # same keys as the GPU arm
     assert d["value"] > 0 and abs(d["value"] - 64 * 128256 / (d["ms_per_step"] * 1e-3) / 1e9) < 1e-6 * d["value"]
     cb = d["cpu_baseline"]
     assert cb["kind"] == "oracle" and cb["cores"] >= 1 and cb["sample"] and cb["value"] == d["value"]
@@ -40,14 +41,27 @@ def test_gpu_arm_prints_the_contract_line():
     if not torch.cuda.is_available():
         pytest.skip("needs a CUDA device")
     d = _run("--steps", "64", "--warmup", "3")
-    assert BASE_KEYS | {"clocks", "gpu_launches", "roofline", "cpu_baseline"} <= set(d) and "impl" not in d
-    assert d["n_gpus"] == 1 and d["steps"] == 64 and d["warmup"] == 3 and d["gpu_launches"] == 64
+    assert BASE_KEYS | {"clocks", "gpu_launches", "roofline", "cpu_baseline", "roofline_detect", "cpu_baseline_detect",
+                        "roofline_sample", "replays", "detect_tokens_per_s"} <= set(d) and "impl" not in d
+    assert d["n_gpus"] == 1 and d["steps"] == 64 and d["warmup"] == 3 and d["gpu_launches"] == 64 * d["replays"]
+    assert d["timed_region_s"] >= 0.25 and d["clocks"]["samples"] >= 50      # clocks sampled inside the region
+    assert set(d["config"]) == {"workload", "B", "V", "scheme", "gamma", "delta", "l2"}
     assert d["dtype"] == "bf16" and d["scaling"] == "weak" and d["vs_baseline"] is None
     elems = 64 * 128256
     assert abs(d["value"] - elems / (d["ms_per_step"] * 1e-3) / 1e9) < 1e-6 * d["value"]
     r = d["roofline"]
     assert r["bound"] in ("alu", "hbm", "tensor") and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
-    assert 0.3 < r["frac"] < 1.3 and r["traffic"] is None or r["traffic"] > 0
+    assert 0.3 < r["frac"] <= 1.05 and (r["traffic"] is None or r["traffic"] > 0)
+    assert "measured in this run" in r["peak_source"]
+    for key in ("roofline_detect", "roofline_detect_selfsalt", "roofline_sample"):      # per-pipe placement of
+        q = d[key]                                                                     # the other kernels
+        assert q["bound"] in ("alu", "hbm") and 0.2 < q["frac"] <= 1.05 and abs(q["frac"] - q["achieved"] / q["peak"]) < 1e-9
+    assert abs(d["detect_tokens_per_s"] - d["roofline_detect"]["tokens_per_s"]) < 1
+    cd = d["cpu_baseline_detect"]
+    assert cd["kind"] == "oracle" and cd["unit"] == "tokens/s" and 0 < cd["value"] < d["detect_tokens_per_s"]
+    for name, e in d["extra"].items():
+        if isinstance(e, dict) and "frac" in e:
+            assert e["frac"] <= 1.05, (name, e["frac"])
     e = d["e2e"]
     assert e["h2d_bytes_per_step"] >= elems * 2 and e["d2h_bytes_per_step"] == elems * 2
     assert 0 < e["value"] < d["value"]                         # the copies are inside that timed region

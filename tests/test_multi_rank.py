@@ -92,6 +92,9 @@ def _shard_worker(rank: int, world: int, port: int, out_dir: str):
     summ[:, 2] = o["score"]
     summ[:, 3] = (o["tokens"] + lo).astype(np.int32).view(np.float32)
     summ[:, 4] = biased[np.arange(B), o["tokens"]]
+    # the agreement check the multi-GPU benchmark leg uses: equal ids pass, rank-dependent ones do not
+    assert sharded.same_on_every_rank(torch.arange(5, dtype=torch.int32))
+    assert not sharded.same_on_every_rank(torch.arange(5, dtype=torch.int32) + rank)
     gathered = sharded.gather_summaries(torch.from_numpy(summ))
     assert gathered.shape == (world, B, 8)
     assert torch.equal(gathered[rank], torch.from_numpy(summ))           # rank-major layout
