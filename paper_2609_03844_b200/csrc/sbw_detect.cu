@@ -15,17 +15,8 @@
 namespace sbw {
 namespace {
 
-#ifndef SBW_DETECT_THREADS
-#define SBW_DETECT_THREADS 128
-#endif
-#ifndef SBW_DETECT_ILP
-#define SBW_DETECT_ILP 4
-#endif
-#ifndef SBW_DETECT_MIN_BLOCKS
-#define SBW_DETECT_MIN_BLOCKS 1
-#endif
-constexpr int kDetectThreads = SBW_DETECT_THREADS;  // 4 sequences per block: short blocks keep the tail small
-constexpr int kDetectIlp = SBW_DETECT_ILP;
+constexpr int kDetectThreads = 128;  // 4 sequences per block: short blocks keep the tail small
+constexpr int kDetectIlp = 4;        // tokens per lane in a full trip
 constexpr int kScanThreads = 256;
 constexpr int kScanItems = 4;        // lengths per thread
 constexpr int kScanTile = kScanThreads * kScanItems;
@@ -128,13 +119,12 @@ scan_offsets(const int32_t *lengths, int64_t N, const int64_t *tile_sums, int64_
 // sequence.  TAIL = false: every position is inside the sequence, no masking.  WIDTH > 0 fixes the
 // context width at compile time (loops unrolled), WIDTH = 0 reads it from the arguments.
 // load_trip reads the tokens and derives their seeds; score_trip hashes them and counts.
-template <int SCHEME, int WIDTH, bool TAIL>
+template <int SCHEME, int WIDTH, bool TAIL, int ILP = kDetectIlp>
 __device__ __forceinline__ void load_trip(const DetectArgs &a, const int32_t *tok, int base, int len, int lane,
-                                          uint32_t (&v)[kDetectIlp], uint64_t (&r)[kDetectIlp],
-                                          bool (&valid)[kDetectIlp]) {
+                                          uint32_t (&v)[ILP], uint64_t (&r)[ILP], bool (&valid)[ILP]) {
     const int width = WIDTH > 0 ? WIDTH : a.W;
 #pragma unroll
-    for (int u = 0; u < kDetectIlp; ++u) {
+    for (int u = 0; u < ILP; ++u) {
         const int t = base + u * 32 + lane;
         valid[u] = !TAIL || static_cast<unsigned>(t) < static_cast<unsigned>(len);
         const int ts = valid[u] ? t : width;      // any readable position; its result is dropped
@@ -159,29 +149,52 @@ __device__ __forceinline__ void load_trip(const DetectArgs &a, const int32_t *to
     }
 }
 
-template <int SCHEME, int WIDTH, bool TAIL>
+// A trip of ILP * 32 positions: ILP = 4 for the bulk of a sequence, 2 and 1 for what is left at its
+// end, so that at most 31 lanes idle per sequence.  BITS: also keep the ballots (sbw_detect_bits).
+template <int SCHEME, int WIDTH, bool TAIL, bool BITS, int ILP = kDetectIlp>
 __device__ __forceinline__ int score_trip(const DetectArgs &a, const int32_t *tok, int base, int len,
                                           int lane, uint32_t *bits) {
     const int width = WIDTH > 0 ? WIDTH : a.W;
-    uint32_t v[kDetectIlp];
-    uint64_t r[kDetectIlp];
-    bool valid[kDetectIlp];
-    load_trip<SCHEME, WIDTH, TAIL>(a, tok, base, len, lane, v, r, valid);
-    uint32_t x[kDetectIlp];
-    philox_word0_n<kDetectIlp>(v, r, x, a.weyl);
+    uint32_t v[ILP];
+    uint64_t r[ILP];
+    bool valid[ILP];
+    load_trip<SCHEME, WIDTH, TAIL, ILP>(a, tok, base, len, lane, v, r, valid);
+    uint32_t x[ILP];
+    philox_word0_n<ILP>(v, r, x, a.weyl);
     int count = 0;
 #pragma unroll
-    for (int u = 0; u < kDetectIlp; ++u) {
+    for (int u = 0; u < ILP; ++u) {
         const unsigned greens = __ballot_sync(0xffffffffu, valid[u] && x[u] <= a.thr_m1);
         count += __popc(greens);
         // the ballot is the bit mask of 32 consecutive scored positions: keep it if asked to
-        if (bits && lane == 0 && (!TAIL || base + u * 32 < len)) bits[((base - width) >> 5) + u] = greens;
+        if (BITS && lane == 0 && (!TAIL || base + u * 32 < len)) bits[((base - width) >> 5) + u] = greens;
     }
     return count;
 }
 
-template <int SCHEME, int WIDTH>
-__global__ void __launch_bounds__(kDetectThreads, SBW_DETECT_MIN_BLOCKS)
+// All scored positions of one sequence from `base` on, by one warp.
+template <int SCHEME, int WIDTH, bool BITS>
+__device__ __forceinline__ int score_sequence(const DetectArgs &a, const int32_t *tok, int base, int len, int lane,
+                                              uint32_t *bits) {
+    constexpr int kTrip = 32 * kDetectIlp;
+    int count = 0;
+    // written as differences so that lengths near 2^31 cannot overflow the position
+    for (; len - base >= kTrip; base += kTrip)
+        count += score_trip<SCHEME, WIDTH, false, BITS>(a, tok, base, len, lane, bits);
+    if (len - base >= 64) {
+        count += score_trip<SCHEME, WIDTH, false, BITS, 2>(a, tok, base, len, lane, bits);
+        base += 64;
+    }
+    if (len - base >= 32) {
+        count += score_trip<SCHEME, WIDTH, false, BITS, 1>(a, tok, base, len, lane, bits);
+        base += 32;
+    }
+    if (base < len) count += score_trip<SCHEME, WIDTH, true, BITS, 1>(a, tok, base, len, lane, bits);
+    return count;
+}
+
+template <int SCHEME, int WIDTH, bool BITS>
+__global__ void __launch_bounds__(kDetectThreads)
 detect_kernel(const DetectArgs a) {
     const int lane = threadIdx.x & 31;
     const int64_t seq = static_cast<int64_t>(blockIdx.x) * (kDetectThreads / 32) + (threadIdx.x >> 5);
@@ -193,15 +206,8 @@ detect_kernel(const DetectArgs a) {
     const int width = WIDTH > 0 ? WIDTH : a.W;
     const int32_t *tok = a.tokens + off;
     const int len = static_cast<int>(L);
-    constexpr int kTrip = 32 * kDetectIlp;
-
-    int count = 0;
-    int base = width;
-    // written as a difference so that lengths near 2^31 cannot overflow the trip counter
-    uint32_t *bits = a.out_bits ? a.out_bits + (off >> 5) + 2 * seq : nullptr;
-    for (; len - base >= kTrip; base += kTrip)
-        count += score_trip<SCHEME, WIDTH, false>(a, tok, base, len, lane, bits);
-    if (base < len) count += score_trip<SCHEME, WIDTH, true>(a, tok, base, len, lane, bits);
+    uint32_t *bits = BITS ? a.out_bits + (off >> 5) + 2 * seq : nullptr;
+    const int count = len > width ? score_sequence<SCHEME, WIDTH, BITS>(a, tok, width, len, lane, bits) : 0;
 
     if (lane == 0) {
         const int T = len > width ? len - width : 0;
@@ -213,7 +219,7 @@ detect_kernel(const DetectArgs a) {
 
 // Few sequences: one CTA per sequence, its warps taking the trips in turn, so that a handful of
 // long texts still spreads over the GPU (a warp per sequence would walk each text alone).
-template <int SCHEME, int WIDTH>
+template <int SCHEME, int WIDTH, bool BITS>
 __global__ void __launch_bounds__(1024)
 detect_wide_kernel(const DetectArgs a) {
     __shared__ int sh_count[32];
@@ -240,15 +246,15 @@ detect_wide_kernel(const DetectArgs a) {
     const int32_t *tok = a.tokens + off;
     const int len = static_cast<int>(L);
     constexpr int kTrip = 32 * kDetectIlp;
-    uint32_t *bits = a.out_bits ? a.out_bits + (off >> 5) + 2 * seq : nullptr;
+    uint32_t *bits = BITS ? a.out_bits + (off >> 5) + 2 * seq : nullptr;
 
     int count = 0;
     const int full = len > width ? (len - width) / kTrip : 0;         // unmasked trips
     for (int i = warp; i < full; i += nwarps)
-        count += score_trip<SCHEME, WIDTH, false>(a, tok, width + i * kTrip, len, lane, bits);
+        count += score_trip<SCHEME, WIDTH, false, BITS>(a, tok, width + i * kTrip, len, lane, bits);
     const int tail_base = width + full * kTrip;
     if (tail_base < len && warp == full % nwarps)
-        count += score_trip<SCHEME, WIDTH, true>(a, tok, tail_base, len, lane, bits);
+        count += score_trip<SCHEME, WIDTH, true, BITS>(a, tok, tail_base, len, lane, bits);
     if (lane == 0) sh_count[warp] = count;
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -268,23 +274,23 @@ inline int wide_threads(int64_t N, int sm_count) {
     return N * 32 <= resident_warps ? 1024 : N * 16 <= resident_warps ? 512 : N * 8 <= resident_warps ? 256 : 0;
 }
 
-template <int SCHEME>
+template <int SCHEME, bool BITS>
 cudaError_t launch_detect(const DetectArgs &a, int sm_count, cudaStream_t s) {
     const int wide = wide_threads(a.N, sm_count);
     if (wide) {
         const unsigned grid = static_cast<unsigned>(a.N);
         switch (a.W) {
-            case 1: detect_wide_kernel<SCHEME, 1><<<grid, wide, 0, s>>>(a); break;
-            case 4: detect_wide_kernel<SCHEME, 4><<<grid, wide, 0, s>>>(a); break;
-            default: detect_wide_kernel<SCHEME, 0><<<grid, wide, 0, s>>>(a); break;
+            case 1: detect_wide_kernel<SCHEME, 1, BITS><<<grid, wide, 0, s>>>(a); break;
+            case 4: detect_wide_kernel<SCHEME, 4, BITS><<<grid, wide, 0, s>>>(a); break;
+            default: detect_wide_kernel<SCHEME, 0, BITS><<<grid, wide, 0, s>>>(a); break;
         }
         return cudaGetLastError();
     }
     const unsigned grid = static_cast<unsigned>((a.N + kDetectThreads / 32 - 1) / (kDetectThreads / 32));
     switch (a.W) {
-        case 1: detect_kernel<SCHEME, 1><<<grid, kDetectThreads, 0, s>>>(a); break;
-        case 4: detect_kernel<SCHEME, 4><<<grid, kDetectThreads, 0, s>>>(a); break;
-        default: detect_kernel<SCHEME, 0><<<grid, kDetectThreads, 0, s>>>(a); break;
+        case 1: detect_kernel<SCHEME, 1, BITS><<<grid, kDetectThreads, 0, s>>>(a); break;
+        case 4: detect_kernel<SCHEME, 4, BITS><<<grid, kDetectThreads, 0, s>>>(a); break;
+        default: detect_kernel<SCHEME, 0, BITS><<<grid, kDetectThreads, 0, s>>>(a); break;
     }
     return cudaGetLastError();
 }
@@ -362,8 +368,15 @@ int detect_impl(const int32_t *tokens, const int32_t *lengths, const int64_t *of
             a.offsets = ws_offsets;
         }
     }
-    SBW_CUDA_TRY(scheme == SBW_SCHEME_CONTEXT ? launch_detect<SBW_SCHEME_CONTEXT>(a, di.sm_count, s)
-                                              : launch_detect<SBW_SCHEME_SELFSALT>(a, di.sm_count, s));
+    cudaError_t err;
+    if (out_bits) {
+        err = scheme == SBW_SCHEME_CONTEXT ? launch_detect<SBW_SCHEME_CONTEXT, true>(a, di.sm_count, s)
+                                           : launch_detect<SBW_SCHEME_SELFSALT, true>(a, di.sm_count, s);
+    } else {
+        err = scheme == SBW_SCHEME_CONTEXT ? launch_detect<SBW_SCHEME_CONTEXT, false>(a, di.sm_count, s)
+                                           : launch_detect<SBW_SCHEME_SELFSALT, false>(a, di.sm_count, s);
+    }
+    SBW_CUDA_TRY(err);
     return SBW_OK;
 }
 

@@ -25,29 +25,8 @@ constexpr uint32_t kPhiloxW1 = 0xBB67AE85u;
 // register or in the constant bank costs one, and the per-candidate key schedule has 16 adds.
 struct Weyl {
     uint32_t w0, w1;
-    uint32_t w0a, w0b, w1a, w1b;   // w0a + w0b = w0, w1a + w1b = w1 (mod 2^32)
 };
-inline Weyl make_weyl() {
-    return Weyl{kPhiloxW0, kPhiloxW1, kPhiloxW0 - 0x01234567u, 0x01234567u, kPhiloxW1 - 0x089abcdeu, 0x089abcdeu};
-}
-
-#ifndef SBW_KS_ALU_MASK0
-#define SBW_KS_ALU_MASK0 0
-#endif
-#ifndef SBW_KS_ALU_MASK1
-#define SBW_KS_ALU_MASK1 0
-#endif
-// x + a + b as one three-input add (ALU pipe only).
-__device__ __forceinline__ uint32_t add3(uint32_t x, uint32_t a, uint32_t b) {
-    uint32_t d;
-    asm("{ .reg .u32 t; add.u32 t, %1, %2; add.u32 %0, t, %3; }" : "=r"(d) : "r"(x), "r"(a), "r"(b));
-    return d;
-}
-template <int ROUND>
-__device__ __forceinline__ void key_step(uint32_t &k0, uint32_t &k1, const Weyl w) {
-    if constexpr ((SBW_KS_ALU_MASK0 >> ROUND) & 1) k0 = add3(k0, w.w0a, w.w0b); else k0 += w.w0;
-    if constexpr ((SBW_KS_ALU_MASK1 >> ROUND) & 1) k1 = add3(k1, w.w1a, w.w1b); else k1 += w.w1;
-}
+inline Weyl make_weyl() { return Weyl{kPhiloxW0, kPhiloxW1}; }
 
 __device__ __forceinline__ void mulhilo(uint32_t a, uint32_t b, uint32_t &hi, uint32_t &lo) {
     const uint64_t p = static_cast<uint64_t>(a) * b;   // one IMAD.WIDE.U32
@@ -240,16 +219,6 @@ __device__ __forceinline__ void philox_word0_n(uint32_t vbase, const RowKeys &rk
     }
 }
 
-template <int ROUND, int N>
-__device__ __forceinline__ void round_n(uint32_t (&c0)[N], uint32_t (&c1)[N], uint32_t (&c2)[N], uint32_t (&c3)[N],
-                                        uint32_t (&k0)[N], uint32_t (&k1)[N], const Weyl w) {
-#pragma unroll
-    for (int i = 0; i < N; ++i) {
-        key_step<ROUND>(k0[i], k1[i], w);
-        philox_round(c0[i], c1[i], c2[i], c3[i], k0[i], k1[i]);
-    }
-}
-
 // Per-candidate seeds r[i] (self-salt scheme, detection), arbitrary ids v[i].
 template <int N>
 __device__ __forceinline__ void philox_word0_n(const uint32_t (&v)[N], const uint64_t (&r)[N],
@@ -269,28 +238,28 @@ __device__ __forceinline__ void philox_word0_n(const uint32_t (&v)[N], const uin
     }
 #pragma unroll
     for (int i = 0; i < N; ++i) {
-        key_step<1>(k0[i], k1[i], w);
+        k0[i] += w.w0;
+        k1[i] += w.w1;
         uint32_t h1, l1;
         mulhilo(kPhiloxM1, c2[i], h1, l1);
         c2[i] = c0[i] ^ c1[i] ^ k1[i];
         c0[i] = h1 ^ k0[i];
         c1[i] = l1;
     }
-    round_n<2, N>(c0, c1, c2, c3, k0, k1, w);
-    round_n<3, N>(c0, c1, c2, c3, k0, k1, w);
-    round_n<4, N>(c0, c1, c2, c3, k0, k1, w);
-    round_n<5, N>(c0, c1, c2, c3, k0, k1, w);
-    round_n<6, N>(c0, c1, c2, c3, k0, k1, w);
-    round_n<7, N>(c0, c1, c2, c3, k0, k1, w);
+#pragma unroll
+    for (int rd = 2; rd < 8; ++rd) {
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+            k0[i] += w.w0;
+            k1[i] += w.w1;
+            philox_round(c0[i], c1[i], c2[i], c3[i], k0[i], k1[i]);
+        }
+    }
 #pragma unroll
     for (int i = 0; i < N; ++i) {
         const uint32_t n1 = kPhiloxM1 * c2[i];
-        uint32_t k1e;
-        if constexpr ((SBW_KS_ALU_MASK1 >> 8) & 1) k1e = add3(k1[i], w.w1a, w.w1b); else k1e = k1[i] + w.w1;
-        const uint32_t n2 = __umulhi(kPhiloxM0, c0[i]) ^ c3[i] ^ k1e;
-        uint32_t k0e;
-        if constexpr ((SBW_KS_ALU_MASK0 >> 9) & 1) k0e = add3(k0[i], w.w0, w.w0); else k0e = k0[i] + w.w0 + w.w0;
-        out[i] = __umulhi(kPhiloxM1, n2) ^ n1 ^ k0e;
+        const uint32_t n2 = __umulhi(kPhiloxM0, c0[i]) ^ c3[i] ^ (k1[i] + w.w1);
+        out[i] = __umulhi(kPhiloxM1, n2) ^ n1 ^ (k0[i] + w.w0 + w.w0);
     }
 }
 
