@@ -169,6 +169,8 @@ int sbw_bias_sample(const void *logits, int dtype, int64_t B, int64_t V, int64_t
  *   out_shard   device, 16-byte aligned, [B, 8] float: per row (m, Z, best score s, GLOBAL id of
  *               the best candidate as int bits, its biased logit, 0, 0, 0) of this shard.
  *   out_tokens  device [B] int32: the shard-local column of that candidate (required).
+ *   vocab_offset + V may not exceed 2^31 here (the summary holds the global id as a signed
+ *   32-bit value), else SBW_ERR_UNSUPPORTED.
  * sbw_sample_combine merges S such summaries laid out [S, B, 8] (shard-major, e.g. the result of
  * an all-gather): m = max m_r, Z = sum Z_r exp((m_r - m)/tau) in fp64, id = the global id with
  * the largest s (ties -> lowest global id), p = exp((l_id - m)/tau)/Z.  out_max / out_sumexp /
@@ -210,7 +212,8 @@ int sbw_bias_sample_shard_ids(const void *logits, int dtype, int64_t B, int64_t 
  * Arguments and results are exactly those of sbw_bias_sample without `workspace` and
  * `workspace_bytes`; inputs and outputs are still the caller's.  Differences:
  *   - B may be at most SBW_NOALLOC_MAX_ROWS; a larger batch returns SBW_ERR_TOO_LARGE and
- *     enqueues nothing (split it, or use sbw_bias_sample).
+ *     enqueues nothing (split it, or use sbw_bias_sample).  The other arguments are checked
+ *     first, so a call that is wrong in another way as well reports that.
  *   - The first call on each device looks up the array's device address (with that device
  *     current) before launching; make that first call outside any stream capture.
  *   - All calls on a device share the one array.  The library clears what has to start at zero

@@ -6,6 +6,7 @@ to load, importing the symbols raises.
 """
 from __future__ import annotations
 
+import atexit
 import ctypes
 from pathlib import Path
 
@@ -35,6 +36,16 @@ EXPORTS = ("sbw_version", "sbw_last_cuda_error", "sbw_bias_logits",
            "sbw_bias_sample_filtered", "sbw_roc_auc_batched", "sbw_bias_sample_shard_ids")
 
 _lib = None
+
+
+def _drain_at_exit() -> None:
+    """Waits for queued GPU work before the interpreter starts tearing libraries down, so that no
+    kernel of this library is in flight while the CUDA runtime it shares with torch unloads."""
+    try:
+        if torch.cuda.is_available() and torch.cuda.is_initialized():
+            torch.cuda.synchronize()
+    except Exception:
+        pass
 
 
 class SbwError(RuntimeError):
@@ -128,6 +139,7 @@ def lib() -> ctypes.CDLL:
                                                vp, sz, vp]
         L.sbw_int_probe.restype = i32
         L.sbw_int_probe.argtypes = [i32, i32, i32, i32, vp, vp, vp]
+        atexit.register(_drain_at_exit)
         _lib = L
     return _lib
 

@@ -374,6 +374,13 @@ extern "C" int sbw_bias_logits_host(void *logits_host, int dtype, int64_t B, int
     const size_t cbytes = static_cast<size_t>(B) * ctx_width * sizeof(int32_t);
     char *d_logits = static_cast<char *>(staging);
     int32_t *d_ctx = reinterpret_cast<int32_t *>(d_logits + sbw::align_up(lbytes, 256));
+    // every check the device entry makes, before anything is enqueued
+    sbw::BiasArgs probe;
+    bool run = false;
+    if (int rc = sbw::prepare(probe, d_logits, dtype, B, V, ld, vocab_offset, d_ctx, ctx_width, key, gamma, delta,
+                              scheme, &run))
+        return rc;
+    if (!run) return SBW_OK;      // a bias that is zero in the logits' precision changes no bit: no copy needed
     SBW_CUDA_TRY(cudaMemcpyAsync(d_ctx, ctx_tokens_host, cbytes, cudaMemcpyHostToDevice, s));
     SBW_CUDA_TRY(cudaMemcpyAsync(d_logits, logits_host, lbytes, cudaMemcpyHostToDevice, s));
     const int rc = sbw::bias_logits_impl(d_logits, dtype, B, V, ld, vocab_offset, d_ctx, ctx_width, key,

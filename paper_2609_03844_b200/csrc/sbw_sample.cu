@@ -36,10 +36,9 @@
 namespace sbw {
 namespace {
 
-#ifndef SBW_SAMPLE_MIN_BLOCKS
-#define SBW_SAMPLE_MIN_BLOCKS 2
-#endif
 constexpr int kSampleThreads = 256;
+constexpr int kSampleMinBlocks = 2;      // with statistics: two blocks per SM (about 110 registers)
+constexpr int kSampleIdsMinBlocks = 3;   // ids only: the kernel waits on its loads, three blocks per SM
 constexpr int kSampleWarps = kSampleThreads / 32;
 constexpr int kMaxSplit = 512;         // chunks per row at most
 constexpr int kMinSlotsPerItem = 32;   // one full trip of a warp at least
@@ -397,11 +396,8 @@ __global__ void __launch_bounds__(1024) clear_kernel(unsigned *p, unsigned n) {
     if (i < n) p[i] = 0u;
 }
 
-#ifndef SBW_SAMPLE_IDS_MIN_BLOCKS
-#define SBW_SAMPLE_IDS_MIN_BLOCKS 3
-#endif
 template <int DTYPE, int SCHEME, bool VECTOR, bool STATS>
-__global__ void __launch_bounds__(kSampleThreads, STATS ? SBW_SAMPLE_MIN_BLOCKS : SBW_SAMPLE_IDS_MIN_BLOCKS)
+__global__ void __launch_bounds__(kSampleThreads, STATS ? kSampleMinBlocks : kSampleIdsMinBlocks)
 sample_kernel(const SampleArgs a) {
     constexpr int VEC = VECTOR ? (DTYPE == SBW_DTYPE_F32 ? 4 : 8) : 1;
     constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
@@ -701,25 +697,39 @@ int launch(SampleArgs &a, bool vector, int64_t nslot, size_t partial_bytes, floa
 
 // Shared by the two entry points: `workspace_bytes` must cover workspace_min_bytes(B); more
 // lets rows be split into more chunks.
+// The argument checks of every sampling entry, workspace excepted; host only.
+int check_sample_args(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld, int64_t vocab_offset,
+                      const int32_t *ctx_tokens, int ctx_width, double gamma, float delta, int scheme,
+                      float temperature, const int32_t *out_tokens, const float *out_shard, int64_t row_offset) {
+    if (!valid_common(dtype, ctx_width, gamma, scheme)) return SBW_ERR_INVALID_ARG;
+    if (B < 0 || V <= 0 || ld < V || vocab_offset < 0) return SBW_ERR_INVALID_ARG;
+    if (!(temperature > 0.0f) || temperature - temperature != 0.0f) return SBW_ERR_INVALID_ARG;
+    if (!(delta == delta) || delta - delta != 0.0f) return SBW_ERR_INVALID_ARG;
+    if (V > 0x7fffffffLL || vocab_offset + V > (int64_t(1) << 32)) return SBW_ERR_UNSUPPORTED;
+    // a shard summary carries the global id as a signed 32-bit value
+    if (out_shard && vocab_offset + V > (int64_t(1) << 31)) return SBW_ERR_UNSUPPORTED;
+    if (B > 0x7fffffffLL / kMaxSplit) return SBW_ERR_UNSUPPORTED;
+    if (B == 0) return SBW_OK;
+    if (!logits || !ctx_tokens || !out_tokens) return SBW_ERR_INVALID_ARG;
+    if (row_offset < 0 || row_offset + B > (int64_t(1) << 32)) return SBW_ERR_INVALID_ARG;
+    if (out_shard && reinterpret_cast<uintptr_t>(out_shard) % 16 != 0) return SBW_ERR_INVALID_ARG;
+    const float c2_hi = static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
+    if (!(c2_hi * 1e15f < FLT_MAX)) return SBW_ERR_INVALID_ARG;   // temperature too small
+    return SBW_OK;
+}
+
 int bias_sample_impl(const void *logits, int dtype, int64_t B, int64_t V, int64_t ld, int64_t vocab_offset,
                      const int32_t *ctx_tokens, int ctx_width, uint64_t key, double gamma, float delta,
                      int scheme, float temperature, uint64_t rng_seed, uint64_t rng_step, int32_t *out_tokens,
                      float *out_max, float *out_sumexp, float *out_prob, float *out_probs, void *workspace,
                      size_t workspace_bytes, bool need_full_workspace, cudaStream_t s,
                      float *out_shard = nullptr, int64_t row_offset = 0, bool shard_ids_only = false) {
-    if (!valid_common(dtype, ctx_width, gamma, scheme)) return SBW_ERR_INVALID_ARG;
-    if (B < 0 || V <= 0 || ld < V || vocab_offset < 0) return SBW_ERR_INVALID_ARG;
-    if (!(temperature > 0.0f) || temperature - temperature != 0.0f) return SBW_ERR_INVALID_ARG;
-    if (!(delta == delta) || delta - delta != 0.0f) return SBW_ERR_INVALID_ARG;
-    if (V > 0x7fffffffLL || vocab_offset + V > (int64_t(1) << 32)) return SBW_ERR_UNSUPPORTED;
-    if (B > 0x7fffffffLL / kMaxSplit) return SBW_ERR_UNSUPPORTED;
+    if (int rc = check_sample_args(logits, dtype, B, V, ld, vocab_offset, ctx_tokens, ctx_width, gamma, delta, scheme,
+                                   temperature, out_tokens, out_shard, row_offset))
+        return rc;
     if (B == 0) return SBW_OK;
-    if (!logits || !ctx_tokens || !out_tokens) return SBW_ERR_INVALID_ARG;
-    if (row_offset < 0 || row_offset + B > (int64_t(1) << 32)) return SBW_ERR_INVALID_ARG;
-    if (out_shard && reinterpret_cast<uintptr_t>(out_shard) % 16 != 0) return SBW_ERR_INVALID_ARG;
     const double c2 = 1.4426950408889634 / static_cast<double>(temperature);
     const float c2_hi = static_cast<float>(c2);
-    if (!(c2_hi * 1e15f < FLT_MAX)) return SBW_ERR_INVALID_ARG;   // temperature too small
     const size_t need = need_full_workspace ? workspace_full_bytes(B) : workspace_min_bytes(B);
     if (!workspace || workspace_bytes < need || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
         return SBW_ERR_WORKSPACE;
@@ -839,17 +849,20 @@ extern "C" int sbw_bias_sample_noalloc(const void *logits, int dtype, int64_t B,
                                        int32_t *out_tokens, float *out_max, float *out_sumexp,
                                        float *out_prob, float *out_probs, void *stream) {
     using namespace sbw;
+    // host-side argument checks first, as in every other entry; the capacity next; the device is
+    // asked for the array's address only by a call that will launch
+    if (int rc = check_sample_args(logits, dtype, B, V, ld, vocab_offset, ctx_tokens, ctx_width, gamma, delta, scheme,
+                                   temperature, out_tokens, nullptr, 0))
+        return rc;
+    if (B == 0) return SBW_OK;
     if (B > SBW_NOALLOC_MAX_ROWS) return SBW_ERR_TOO_LARGE;
     static_assert(sizeof(double2) * SBW_NOALLOC_MAX_ROWS + 2 * sizeof(unsigned) * SBW_NOALLOC_MAX_ROWS +
                           sizeof(Partial) * SBW_NOALLOC_MAX_ROWS + 3 * 256 <=
                       kNoallocScratchBytes,
                   "the built-in scratch must hold the workspace of SBW_NOALLOC_MAX_ROWS rows");
-    if (B > 0 && workspace_min_bytes(B) > kNoallocScratchBytes) return SBW_ERR_TOO_LARGE;
+    if (workspace_min_bytes(B) > kNoallocScratchBytes) return SBW_ERR_TOO_LARGE;
     void *scratch = nullptr;
-    if (B > 0) {
-        const int rc = noalloc_scratch_address(&scratch);
-        if (rc != SBW_OK) return rc;
-    }
+    if (int rc = noalloc_scratch_address(&scratch)) return rc;
     // The shared array keeps whatever the previous call left in it.  The only part that must
     // start at zero is the per-row ticket counters, and the launch code clears those on the
     // stream before every launch that uses them; everything else is written before it is read.

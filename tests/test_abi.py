@@ -85,6 +85,42 @@ def test_argument_validation_happens_on_the_host():
     assert sample(ws_bytes=16) == binding.SBW_ERR_WORKSPACE
     assert sample(ws=ctypes.c_void_p(0x1008)) == binding.SBW_ERR_WORKSPACE   # not 256-aligned
 
+    def noalloc(**kw):          # the entry without a workspace: same checks, then its capacity, all on the host
+        a = {**ok, "tau": 0.7, **kw}
+        return L.sbw_bias_sample_noalloc(a.get("logits", fake), a["dtype"], a["B"], a["V"], a["ld"], a["off"],
+                                         a.get("ctx", fake), a["W"], a["key"], a["gamma"], a["delta"],
+                                         a["scheme"], a["tau"], 1, 2, a.get("out", fake), None, None, None, None, None)
+
+    assert noalloc(B=0) == binding.SBW_OK
+    big = binding.NOALLOC_MAX_ROWS + 1
+    assert noalloc(B=big) == binding.SBW_ERR_TOO_LARGE
+    for bad in (dict(tau=0.0), dict(gamma=1.5), dict(out=None), dict(logits=None), dict(ld=3), dict(dtype=2),
+                dict(delta=float("nan"))):
+        assert noalloc(**bad) == binding.SBW_ERR_INVALID_ARG, bad
+        assert noalloc(B=big, **bad) == binding.SBW_ERR_INVALID_ARG, bad      # the other fault is reported first
+
+    def host(**kw):             # host-buffer entry: every check before the first copy is enqueued
+        a = {**ok, "staging": ctypes.c_void_p(0x1000), "sb": 1 << 20, **kw}
+        return L.sbw_bias_logits_host(a.get("logits", fake), a["dtype"], a["B"], a["V"], a["ld"], a["off"],
+                                      a.get("ctx", fake), a["W"], a["key"], a["gamma"], a["delta"], a["scheme"],
+                                      a["staging"], a["sb"], None)
+
+    assert host(B=0) == binding.SBW_OK and host(delta=0.0) == binding.SBW_OK
+    for bad in (dict(delta=float("nan")), dict(delta=float("inf")), dict(gamma=0.0), dict(logits=None), dict(ctx=None)):
+        assert host(**bad) == binding.SBW_ERR_INVALID_ARG, bad
+    assert host(off=(1 << 32) - 4) == binding.SBW_ERR_UNSUPPORTED
+    assert host(staging=None) == binding.SBW_ERR_WORKSPACE and host(sb=8) == binding.SBW_ERR_WORKSPACE
+
+    def shard(**kw):            # a shard summary holds the global id in 31 bits
+        a = {**ok, "tau": 0.7, **kw}
+        return L.sbw_bias_sample_shard(fake, a["dtype"], a["B"], a["V"], a["ld"], a["off"], 0, fake, a["W"], a["key"],
+                                       a["gamma"], a["delta"], a["scheme"], a["tau"], 1, 2, a.get("summary", fake), fake,
+                                       fake, 1 << 20, None)
+
+    assert shard(B=0) == binding.SBW_OK
+    assert shard(off=(1 << 31) - 4) == binding.SBW_ERR_UNSUPPORTED
+    assert shard(summary=None) == binding.SBW_ERR_INVALID_ARG
+
     def detect(**kw):
         a = dict(N=4, total=40, W=1, gamma=0.25, scheme=0, ws=fake, ws_bytes=1 << 20, off=None)
         a.update(kw)
