@@ -139,12 +139,31 @@ __device__ __forceinline__ void load_trip(const DetectArgs &a, const int32_t *to
                     if (i <= width) sigma += static_cast<uint32_t>(tok[ts - i]);
                 r[u] = a.key * sigma;
             }
-        } else {
+        }
+    }
+    if constexpr (SCHEME == SBW_SCHEME_SELFSALT) {
+        // Every id of the trip is hashed once: a position's context hashes are its neighbours' own
+        // hashes, fetched by shuffles (position t - i sits i lanes down, or at the top of the group
+        // of 32 before; the group before the trip's first is hashed for the purpose).  A lane whose
+        // position is valid only draws on lanes with smaller, hence valid, positions.
+        uint32_t jv[ILP + 1];                       // jv[u + 1]: group u; jv[0]: the 32 positions before the trip
+        const int before = base - 32 + lane;
+        jv[0] = jenkins(static_cast<uint32_t>(tok[before > 0 ? before : 0]));
+#pragma unroll
+        for (int u = 0; u < ILP; ++u) jv[u + 1] = jenkins(v[u]);
+#pragma unroll
+        for (int u = 0; u < ILP; ++u) {
             uint32_t jmin = 0xFFFFFFFFu;
 #pragma unroll
-            for (int i = 1; i <= (WIDTH > 0 ? WIDTH : SBW_MAX_CTX_WIDTH); ++i)
-                if (i <= width) jmin = min(jmin, jenkins(static_cast<uint32_t>(tok[ts - i])));
-            r[u] = seed_selfsalt(a.key, jmin, v[u]);
+            for (int i = 1; i <= (WIDTH > 0 ? WIDTH : SBW_MAX_CTX_WIDTH); ++i) {
+                if (i <= width) {
+                    // lanes 32 - i .. 31 hand over the group before, the others this group
+                    const uint32_t give = lane >= 32 - i ? jv[u] : jv[u + 1];
+                    jmin = min(jmin, __shfl_sync(0xffffffffu, give, (lane - i) & 31));
+                }
+            }
+            const uint64_t prod = static_cast<uint64_t>(jv[u + 1]) * min(jv[u + 1], jmin);
+            r[u] = a.key * prod;
         }
     }
 }

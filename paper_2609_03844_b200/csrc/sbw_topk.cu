@@ -123,21 +123,31 @@ __device__ __forceinline__ void for_each_vector(const char *row_ptr, uint32_t be
     for (uint32_t c = done + threadIdx.x; c < end; c += kTopkThreads) fone(c, scalar_code<DTYPE>(row_ptr, c));
 }
 
-// Eq. 1 + Eq. 2 on one chosen column.
-template <int DTYPE, int SCHEME>
-__device__ __noinline__ void bias_column(const TopkArgs &a, int64_t row, char *row_ptr, uint32_t col) {
+// What the green test of a row needs from its context tokens: the seed itself (context scheme) or
+// the smallest context hash (self-salt).  Read when the row is started, so that the tokens'
+// latency hides behind the row's first loads.
+template <int SCHEME>
+__device__ __forceinline__ uint64_t row_seed_material(const TopkArgs &a, int64_t row) {
     const int32_t *ctx = a.ctx + row * a.W;
+    if constexpr (SCHEME == SBW_SCHEME_CONTEXT) return seed_context(a.key, ctx, a.W);
+    else return jenkins_min(ctx, a.W);
+}
+
+// Eq. 1 + Eq. 2 on one chosen column whose order code is known: the value is rebuilt from the
+// code (no second read of the logit) and stored only if the column is green.
+template <int DTYPE, int SCHEME>
+__device__ __noinline__ void bias_column(const TopkArgs &a, uint64_t material, char *row_ptr, uint32_t col, uint32_t code) {
     const uint32_t v = a.vocab_offset + col;
     uint64_t r;
-    if constexpr (SCHEME == SBW_SCHEME_CONTEXT) r = seed_context(a.key, ctx, a.W);
-    else r = seed_selfsalt(a.key, jenkins_min(ctx, a.W), v);
+    if constexpr (SCHEME == SBW_SCHEME_CONTEXT) r = material;
+    else r = seed_selfsalt(a.key, static_cast<uint32_t>(material), v);
     if (philox_word0(v, r, a.weyl) > a.thr_m1) return;
     if constexpr (DTYPE == SBW_DTYPE_F32) {
-        float *p = reinterpret_cast<float *>(row_ptr) + col;
-        *p = __fadd_rn(*p, a.delta);
+        reinterpret_cast<float *>(row_ptr)[col] = __fadd_rn(__uint_as_float(order_decode(code)), a.delta);
     } else {
-        __nv_bfloat16 *p = reinterpret_cast<__nv_bfloat16 *>(row_ptr) + col;
-        *p = __float2bfloat16_rn(__fadd_rn(__bfloat162float(*p), a.delta));
+        const uint32_t bits = (code & 0x8000u) ? (code ^ 0x8000u) : (code ^ 0xffffu);
+        reinterpret_cast<__nv_bfloat16 *>(row_ptr)[col] =
+            __float2bfloat16_rn(__fadd_rn(__uint_as_float(bits << 16), a.delta));
     }
 }
 
@@ -170,7 +180,7 @@ topk_kernel(const TopkArgs a) {
     constexpr int kTopkWarps = kTopkThreads / 32;
     constexpr int kGroups = kTopkThreads / 4;   // maxima of disjoint column sets used for the lower bound
     __shared__ uint32_t sh_max[kGroups];
-    __shared__ uint64_t sh_cand[kCap];
+    __shared__ __align__(16) uint64_t sh_cand[kCap + 2];
     __shared__ uint64_t sh_red[kTopkWarps];
     __shared__ uint64_t sh_best;
     __shared__ uint32_t sh_floor;
@@ -188,6 +198,7 @@ topk_kernel(const TopkArgs a) {
 
     for (int64_t row = first_row; row < a.B; row += row_step) {
         char *row_ptr = static_cast<char *>(a.logits) + row * a.ld * ESIZE;
+        const uint64_t material = row_seed_material<SCHEME>(a, row);
 
         // 1. lower bound of the k-th largest code from a prefix of the columns
         const uint32_t prefix_end = min(c_hi, c_lo + static_cast<uint32_t>(kPrefixColumns / CS));
@@ -257,11 +268,21 @@ topk_kernel(const TopkArgs a) {
 
         if (n <= kCap) {
             // 3. rank by counting, bias ranks below k
+            if (threadIdx.x == 0 && (n & 1u)) sh_cand[n] = 0;      // pad to a pair (kCap is even; 0 ranks below all)
+            __syncthreads();
             for (unsigned e = threadIdx.x; e < n; e += kTopkThreads) {
                 const uint64_t mine = sh_cand[e];
-                uint32_t rank = 0;
-                for (unsigned u = 0; u < n; ++u) rank += sh_cand[u] > mine ? 1u : 0u;
-                if (rank < k) bias_column<DTYPE, SCHEME>(a, row, row_ptr, 0xFFFFFFFFu - static_cast<uint32_t>(mine));
+                uint32_t r0 = 0, r1 = 0;
+                const ulonglong2 *pairs = reinterpret_cast<const ulonglong2 *>(sh_cand);
+#pragma unroll 4
+                for (unsigned u = 0; u < (n + 1) / 2; ++u) {          // two composites per shared-memory load
+                    const ulonglong2 q = pairs[u];
+                    r0 += q.x > mine ? 1u : 0u;
+                    r1 += q.y > mine ? 1u : 0u;
+                }
+                if (r0 + r1 < k)
+                    bias_column<DTYPE, SCHEME>(a, material, row_ptr, 0xFFFFFFFFu - static_cast<uint32_t>(mine),
+                                               static_cast<uint32_t>(mine >> 32));
             }
         } else {
             // fallback: k rounds of "largest composite below the previous one" find the composite
@@ -280,7 +301,8 @@ topk_kernel(const TopkArgs a) {
             }
             const uint64_t kth = prev;
             for_each_code<DTYPE, kTopkThreads>(row_ptr, 0u, V, a.vector, [&](uint32_t col, uint32_t code) {
-                if (composite(code, col) >= kth) bias_column<DTYPE, SCHEME>(a, row, row_ptr, col);
+                if (composite(code, col) >= kth)
+                    bias_column<DTYPE, SCHEME>(a, material, row_ptr, col, DTYPE == SBW_DTYPE_F32 ? code : code >> 16);
             });
         }
         __syncthreads();             // shared scratch is reused by the next row
