@@ -376,7 +376,7 @@ def run_ours(args) -> None:
 
     k_steps()                           # one untimed pass: graph upload
     ms1, _, _ = time_region(k_steps, stream, world, dev)
-    replays = max(1, int(MIN_REGION_S * 1.2 / (ms1 * 1e-3)) + 1)
+    replays = max(1, int(args.region_s * 1.2 / (ms1 * 1e-3)) + 1)
     if world > 1:                       # every rank replays the same number of times
         replays = int(max_over_ranks(float(replays), world, dev))
     ms, t0, t1 = time_region(lambda: [k_steps() for _ in range(replays)], stream, world, dev)
@@ -844,6 +844,8 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=16)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches only")
+    ap.add_argument("--region-s", type=float, default=MIN_REGION_S,
+                    help="shortest timed region in seconds (0: exactly --steps steps, for a profiler's launch list)")
     ap.add_argument("--no-extra", action="store_true", help="skip the secondary workloads and the CPU baselines")
     ap.add_argument("--profile-case", choices=PROFILE_CASES, default=None,
                     help="run a few launches of one kernel on a small (> L2) input, for a profiler")
