@@ -28,6 +28,12 @@ def gather_summaries(local: torch.Tensor, group=None) -> torch.Tensor:
     world = dist.get_world_size(group) if dist.is_initialized() else 1
     if world == 1:
         return local.reshape(1, *local.shape).contiguous()
+    if local.is_cuda and dist.get_backend(group) == "gloo":
+        # gloo gathers host tensors only: stage the 32 bytes per row through the host
+        host = local.detach().cpu().contiguous()
+        parts = [torch.empty_like(host) for _ in range(world)]
+        dist.all_gather(parts, host, group=group)
+        return torch.stack(parts).to(local.device)
     out = torch.empty((world, *local.shape), dtype=local.dtype, device=local.device)
     dist.all_gather([out[r] for r in range(world)], local.contiguous(), group=group)
     return out

@@ -101,3 +101,50 @@ def test_ids_only_shards_give_the_same_ids(dtype, scheme, S, B):
     assert np.array_equal(tok.cpu().numpy(), want["tokens"])
     s = summaries.cpu().numpy()
     assert np.isneginf(s[:, :, 0]).all() and (s[:, :, 1] == 0).all()       # no statistics in these summaries
+
+
+def _leg_worker(rank: int, world: int, port: int, out_dir: str):
+    import json
+    import os
+    import sys
+    from pathlib import Path
+
+    import torch.distributed as dist
+
+    root = Path(__file__).resolve().parent.parent
+    sys.path.insert(0, str(root))
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world),
+                      LOCAL_RANK="0")
+    torch.cuda.set_device(0)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    import paper_2609_03844_b200 as lib
+    from paper_2609_03844_b200 import inputs as inp
+
+    out = bench.run_sharded_leg(lib, inp, torch.device("cuda", 0), rank, world)
+    with open(os.path.join(out_dir, f"leg{rank}.json"), "w") as f:
+        json.dump(out, f)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+@pytest.mark.gpu
+def test_benchmark_sharded_leg_with_two_ranks_on_one_gpu(tmp_path):
+    """The N > 1 leg of bench.py end to end: two processes share the one GPU (their kernels never wait
+    on each other), each samples its half of the vocabulary, the summaries are all-gathered (gloo
+    here, NCCL on several GPUs) and combined; both must end with the ids of the unsplit call."""
+    import json
+    import socket
+
+    import torch.multiprocessing as mp
+
+    require_gpu()
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    world = 2
+    mp.spawn(_leg_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    for r in range(world):
+        leg = json.loads((tmp_path / f"leg{r}.json").read_text())
+        assert leg["shards"] == 2 and leg["ids_equal_on_every_rank"] and leg["ids_equal_unsplit_call"]
+        assert leg["sumexp_max_rel_diff_to_unsplit_call"] <= 1e-6 and leg["ms_per_step"] > 0
