@@ -77,6 +77,7 @@ template <int DTYPE, int SCHEME>
 __device__ __noinline__ void bias_scalar(const BiasArgs &a, const RowSeed<SCHEME> &rs, void *row_ptr,
                                          uint32_t c_begin, uint32_t c_end, uint32_t c_step) {
     for (uint32_t col = c_begin; col < c_end; col += c_step) {
+        if (!SBW_CHECKED(col < static_cast<uint32_t>(a.V), SBW_SITE_BIAS_SCALAR)) continue;
         const uint32_t v = a.vocab_offset + col;
         if (rs.word0(v, a.key, a.weyl) > a.thr_m1) continue;
         if constexpr (DTYPE == SBW_DTYPE_F32) {
@@ -173,6 +174,9 @@ bias_kernel(const BiasArgs a) {
             if constexpr (DTYPE == SBW_DTYPE_BF16) {
                 const uint32_t dlo = a.delta_bf16, dhi = a.delta_bf16 << 16;
                 for (uint32_t j = col + threadIdx.x; j < jf_end; j += kBiasThreads) {
+                    if (!SBW_CHECKED(row < a.B && (static_cast<uint64_t>(j) + 1) * 8 <= static_cast<uint64_t>(a.V),
+                                     SBW_SITE_BIAS_VECTOR))
+                        continue;
                     uint4 w = in[j];
                     bool g[8];
                     green8<SCHEME>(a, rs, a.vocab_offset + j * 8, g);
@@ -191,6 +195,9 @@ bias_kernel(const BiasArgs a) {
                 for (uint32_t j = col + threadIdx.x; j < jf_end; j += 2 * kBiasThreads) {
                     const uint32_t j2 = j + kBiasThreads;
                     const bool two = j2 < jf_end;
+                    if (!SBW_CHECKED(row < a.B && (static_cast<uint64_t>(two ? j2 : j) + 1) * 4 <= static_cast<uint64_t>(a.V),
+                                     SBW_SITE_BIAS_VECTOR))
+                        continue;
                     uint4 w0 = in[j];
                     uint4 w1 = two ? in[j2] : make_uint4(0, 0, 0, 0);
                     bool g[8];

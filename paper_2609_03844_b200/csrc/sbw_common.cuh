@@ -8,6 +8,28 @@
 
 #include "../../include/sbw.h"
 
+// Bounds-flag build (-DSBW_DEBUG, relocatable device code): every global access of the three core
+// kernels is preceded by a check of its row / column / position against the call's sizes.  A
+// failed check records its site in a device-side flag word and the access is skipped -- no trap,
+// no device assert -- and sbw_debug_flags() reads the words back.  It stands in for a memory
+// checker on machines where none can be run; release builds compile the checks away.
+#ifdef SBW_DEBUG
+extern __device__ unsigned int g_sbw_debug[4];   // [0]: bit mask of failed sites, [1]: failures, [2]: checks passed
+#define SBW_CHECKED(ok, site)                                                            \
+    ((ok) ? (atomicAdd(&g_sbw_debug[2], 1u), true)                                       \
+          : (atomicOr(&g_sbw_debug[0], 1u << (site)), atomicAdd(&g_sbw_debug[1], 1u), false))
+#else
+#define SBW_CHECKED(ok, site) (true)
+#endif
+// check sites
+#define SBW_SITE_BIAS_VECTOR 0
+#define SBW_SITE_BIAS_SCALAR 1
+#define SBW_SITE_SAMPLE_LOAD 2
+#define SBW_SITE_SAMPLE_WORKSPACE 3
+#define SBW_SITE_SAMPLE_OUTPUT 4
+#define SBW_SITE_DETECT_TOKEN 5
+#define SBW_SITE_DETECT_OUTPUT 6
+
 namespace sbw {
 
 // cudaError_t of the calling thread's last failing runtime call.

@@ -128,6 +128,8 @@ __device__ __forceinline__ void load_trip(const DetectArgs &a, const int32_t *to
         const int t = base + u * 32 + lane;
         valid[u] = !TAIL || static_cast<unsigned>(t) < static_cast<unsigned>(len);
         const int ts = valid[u] ? t : width;      // any readable position; its result is dropped
+        (void)SBW_CHECKED(ts >= width && ts < len && (tok - a.tokens) + ts < a.total_tokens && (tok - a.tokens) + ts - width >= 0,
+                          SBW_SITE_DETECT_TOKEN);
         v[u] = static_cast<uint32_t>(tok[ts]);
         if constexpr (SCHEME == SBW_SCHEME_CONTEXT) {
             if constexpr (WIDTH == 1) {
@@ -230,6 +232,7 @@ detect_kernel(const DetectArgs a) {
 
     if (lane == 0) {
         const int T = len > width ? len - width : 0;
+        (void)SBW_CHECKED(seq >= 0 && seq < a.N && count >= 0 && count <= T, SBW_SITE_DETECT_OUTPUT);
         a.out_counts[seq] = count;
         if (a.out_T) a.out_T[seq] = T;
         a.out_z[seq] = zscore(count, T, a.gamma);

@@ -277,6 +277,7 @@ __device__ void finish_row(const SampleArgs &a, int64_t row, const Partial *part
     if (lane == 0) {
         if (id == INT_MAX) id = 0;                       // every score was -inf: lowest id
         const double md = static_cast<double>(m);
+        (void)SBW_CHECKED(row >= 0 && row < a.B && id >= 0 && id < a.V, SBW_SITE_SAMPLE_OUTPUT);
         a.out_tokens[row] = id;
         if (a.out_max) a.out_max[row] = m;
         if (a.out_sumexp) a.out_sumexp[row] = static_cast<float>(Z);
@@ -296,6 +297,7 @@ __device__ __forceinline__ void load_biased(const SampleArgs &a, const RowSeedS<
                                             uint32_t j, uint32_t cb, uint32_t V, float (&lp)[VEC]) {
     const uint32_t vg = a.vocab_offset + cb;
     if (VECTOR && cb + VEC <= V) {
+        (void)SBW_CHECKED(static_cast<uint64_t>(j) * VEC + VEC <= static_cast<uint64_t>(a.V), SBW_SITE_SAMPLE_LOAD);
         const uint4 w = __ldg(reinterpret_cast<const uint4 *>(row_ptr) + j);
         const uint32_t *e = reinterpret_cast<const uint32_t *>(&w);
         uint32_t x[VEC];
@@ -546,7 +548,7 @@ sample_kernel(const SampleArgs a) {
             Partial p;
             p.m = m_w; p.z = z_t; p.s = best.s; p.id = best.id; p.l = best.l;
             p.pad[0] = p.pad[1] = p.pad[2] = 0.0f;
-            a.partials[item] = p;
+            if (SBW_CHECKED(item >= 0 && item < a.n_items && row < a.B, SBW_SITE_SAMPLE_WORKSPACE)) a.partials[item] = p;
             __threadfence();                           // partial visible before the ticket is taken
             if (a.split > 1) ticket = atomicAdd(&a.tickets[row], 1u);
         }
