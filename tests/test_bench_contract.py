@@ -69,3 +69,45 @@ def test_gpu_arm_prints_the_contract_line():
     assert c["sm_mhz"] > 0 and c["sm_max_mhz"] >= c["sm_mhz"] and isinstance(c["reasons"], list)
     cb = d["cpu_baseline"]
     assert cb["kind"] == "oracle" and cb["cores"] >= 1 and 0 < cb["value"] < d["value"]
+
+
+def test_roofline_model_arithmetic():
+    """bench.place on hand-made rates: the ceiling is the slowest of the multiplier pipe, the ALU pipe,
+    both pipes sharing the work, the issue slots and HBM; frac = ceiling time / measured time."""
+    sys.path.insert(0, str(ROOT))
+    import bench
+
+    rates = {"r_wide": 30.0, "r_wide_isolated": 32.0, "r_imad": 64.0, "r_alu": 64.0, "r_issue": 128.0}
+    w = bench.WORK["bias_context"]
+    clocks = bench.unit_clocks(w, rates)
+    assert abs(clocks["multiplier pipe"] - (w["wide"] / 30.0 + w["imad"] / 64.0)) < 1e-12
+    assert abs(clocks["alu pipe"] - w["alu"] / 64.0) < 1e-12
+    assert abs(clocks["both integer pipes"] - (w["wide"] * 64.0 / 30.0 + w["imad"] + w["alu"]) / 128.0) < 1e-12
+    assert abs(clocks["issue slots"] - (w["wide"] + w["imad"] + w["alu"] + w["fp"]) / 128.0) < 1e-12
+    units, mhz = 64 * 128256, 1965.0
+    t_mul = clocks["multiplier pipe"] * units / (bench.SMS * mhz * 1e6)
+    r = bench.place("bias_context", units, 4 * units, 2.0 * t_mul, rates, mhz, 6553.6)
+    assert r["bound"] == "alu" and r["limiter"] == "multiplier pipe" and abs(r["frac"] - 0.5) < 1e-9
+    assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-12 and r["frac_isolated"] < r["frac"]
+    assert r["plain_eval"]["frac"] > r["frac"]                      # the plain count holds more products
+    # a launch that moves so many bytes per unit that HBM is the ceiling
+    r = bench.place("bias_context", units, 4000 * units, 1.0, rates, mhz, 6553.6)
+    assert r["bound"] == "hbm" and abs(r["frac"] - 4000 * units / 6553.6e9) < 1e-9
+    # least-work counts never exceed the plain-evaluation counts
+    for kind, plain in bench.PLAIN_EVAL.items():
+        least = bench.WORK[kind]
+        assert least["wide"] <= plain["wide"] and least["wide"] + least["imad"] + least["alu"] <= \
+            plain["wide"] + plain["imad"] + plain["alu"]
+
+
+def test_clock_summary_uses_only_samples_inside_the_region():
+    sys.path.insert(0, str(ROOT))
+    import bench
+
+    s = bench.ClockSampler.__new__(bench.ClockSampler)
+    s.nv, s.max_mhz = object(), 1965.0
+    s.samples = [(0.5, 1000.0, 0x1), (1.1, 1965.0, 0x0), (1.2, 1950.0, 0x4), (1.3, 1965.0, 0x0), (2.5, 300.0, 0x8)]
+    out = s.summary(1.0, 2.0)
+    assert out["samples"] == 3 and out["sm_mhz"] == 1965.0 and out["sm_min_mhz"] == 1950.0
+    assert out["reasons"] == ["sw_power_cap"]                        # the slowdown outside the region is not reported
+    assert s.summary(3.0, 4.0)["samples"] == 0 and s.summary(3.0, 4.0)["sm_mhz"] is None
