@@ -86,7 +86,12 @@ PLAIN_EVAL = {
 # DRAM bytes per bias launch of the headline workload: dram__bytes_read.sum + dram__bytes_write.sum
 # of one ncu capture of the same kernel on B=512 (131.38 MB + 91.60 MB, profiles/), divided by 8
 # because a bench launch processes 1/8 of those units and the traffic grows with the units.
-NCU_TRAFFIC_BYTES = (131.38e6 + 91.60e6) / 8
+NCU_TRAFFIC_BYTES = (131.38e6 + 91.76e6) / 8
+# DRAM bytes of one detection launch on the config-5 shape (the bench's own workload, one ncu capture
+# each, profiles/detect_kernel_...md) and of one sampling launch with statistics (captured at B = 512,
+# doubled for the B = 1024 launch the bench times, profiles/sample_kernel_...md).
+NCU_TRAFFIC_DETECT = {"context": 218.95e6 + 4.23e6, "selfsalt": 218.86e6 + 4.16e6}
+NCU_TRAFFIC_SAMPLE_B1024 = 2 * 131.42e6
 
 
 def measured_peaks() -> dict:
@@ -628,7 +633,8 @@ def run_detect(sbw, inputs, dev, peaks, rates, sampler) -> dict:
                                                          workspace=ws), 30, min_s=0.25)
         mhz = sampler.mhz(t0, t1) or sampler.max_mhz or 1965.0
         r = place(f"detect_{name}", ntok, 4 * ntok + 24 * N, s, rates, mhz, peaks["hbm_gbs"])
-        r.update({"tokens_per_s": ntok / s, "ms": s * 1e3, "tokens": ntok, "sequences": N,
+        r.update({"traffic": NCU_TRAFFIC_DETECT[name], "tokens_per_s": ntok / s, "ms": s * 1e3, "tokens": ntok,
+                  "sequences": N,
                   "workload": "config 5 shape: 100000 sequences of uniform ids, lengths uniform in [64, 1024], "
                               f"V=128256, {name} scheme, gamma 0.25; 218 MB of ids, larger than L2"})
         out[name] = r
@@ -737,7 +743,7 @@ def run_extra(sbw, inputs, dev, peaks, rates, sampler) -> dict:
                 out[f"sample_bf16_{name}_B{B}"]["graph_ms"] = s * 1e3
                 s = _time_graph(lambda i: sbw.sbw_bias_sample(x, c, KEY, 0.25, 2.0, scheme, 0.7, 0xC4, i, ids, wsb), 16)
                 out[f"sample_ids_only_bf16_{name}_B{B}"]["graph_ms"] = s * 1e3
-    out["roofline_sample"] = {**out["sample_bf16_context_B1024"],
+    out["roofline_sample"] = {**out["sample_bf16_context_B1024"], "traffic": NCU_TRAFFIC_SAMPLE_B1024,
                               "workload": "config 4: sbw_bias_sample with the softmax sum, B=1024, V=128256, "
                                           "bf16, context scheme, gamma 0.25, delta 2, tau 0.7 (263 MB, larger than L2)"}
     # Appendix F's sampling setting (temperature 0.7, top_p 0.8) and a top-k one, through the truncated sampler
