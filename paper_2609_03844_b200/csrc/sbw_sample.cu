@@ -36,10 +36,11 @@
 namespace sbw {
 namespace {
 
-constexpr int kSampleThreads = 256;
-constexpr int kSampleMinBlocks = 2;      // with statistics: two blocks per SM (about 110 registers)
-constexpr int kSampleIdsMinBlocks = 3;   // ids only: the kernel waits on its loads, three blocks per SM
-constexpr int kSampleWarps = kSampleThreads / 32;
+// Block shape.  With statistics: one block of 16 warps per SM at about 110 registers (3 % ahead of
+// two blocks of 8 warps, as in the bias kernel).  Ids only: the kernel waits on its loads and does
+// best with three blocks of 8 warps (85 registers).
+__host__ __device__ constexpr int sample_threads(bool stats) { return stats ? 512 : 256; }
+__host__ __device__ constexpr int sample_min_blocks(bool stats) { return stats ? 1 : 3; }
 constexpr int kMaxSplit = 512;         // chunks per row at most
 constexpr int kMinSlotsPerItem = 32;   // one full trip of a warp at least
 constexpr int kMaxExtraParts = 40960;  // partials beyond one per row never needed: ~16 waves of warps
@@ -399,8 +400,9 @@ __global__ void __launch_bounds__(1024) clear_kernel(unsigned *p, unsigned n) {
 }
 
 template <int DTYPE, int SCHEME, bool VECTOR, bool STATS>
-__global__ void __launch_bounds__(kSampleThreads, STATS ? kSampleMinBlocks : kSampleIdsMinBlocks)
+__global__ void __launch_bounds__(sample_threads(STATS), sample_min_blocks(STATS))
 sample_kernel(const SampleArgs a) {
+    constexpr int kSampleWarps = sample_threads(STATS) / 32;
     constexpr int VEC = VECTOR ? (DTYPE == SBW_DTYPE_F32 ? 4 : 8) : 1;
     constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
     const int lane = threadIdx.x & 31;
@@ -641,6 +643,7 @@ int launch_one(SampleArgs &a, int64_t nslot, size_t partial_bytes, cudaStream_t 
     DeviceInfo di;
     const int rc = current_device_info(&di);
     if (rc != SBW_OK) return rc;
+    constexpr int kSampleThreads = sample_threads(STATS), kSampleWarps = kSampleThreads / 32;
     static std::atomic<int> blocks_per_sm{0};  // a property of the compiled kernel, equal on every sm_100a device
     if (blocks_per_sm == 0) {
         int n = 0;
@@ -650,10 +653,10 @@ int launch_one(SampleArgs &a, int64_t nslot, size_t partial_bytes, cudaStream_t 
     }
     const int64_t ctas = static_cast<int64_t>(di.sm_count) * blocks_per_sm;
     const int64_t warps = ctas * kSampleWarps;
-    // small batches: no more chunks per row than fill two CTAs per SM, even when more CTAs fit --
+    // small batches: no more chunks per row than fill sixteen warps per SM, even when more fit --
     // beyond that the extra partials cost more in the final merge than the extra warps bring
     int64_t max_parts = static_cast<int64_t>(partial_bytes / sizeof(Partial));
-    const int64_t two_per_sm = static_cast<int64_t>(di.sm_count) * 2 * kSampleWarps;
+    const int64_t two_per_sm = static_cast<int64_t>(di.sm_count) * 16;
     if (two_per_sm / a.B >= 32 && max_parts > two_per_sm) max_parts = two_per_sm;
     a.split = choose_split(a.B, nslot, warps, max_parts);
     a.n_items = a.B * a.split;
