@@ -406,7 +406,9 @@ sample_kernel(const SampleArgs a) {
     constexpr int VEC = VECTOR ? (DTYPE == SBW_DTYPE_F32 ? 4 : 8) : 1;
     constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
     const int lane = threadIdx.x & 31;
-    const int64_t warp_id = static_cast<int64_t>(blockIdx.x) * kSampleWarps + (threadIdx.x >> 5);
+    // warp w of block b takes items b + w * gridDim.x, ...: consecutive items go to different blocks, so
+    // a small batch (fewer items than warps) spreads over all SMs instead of filling a few
+    const int64_t warp_id = static_cast<int64_t>(threadIdx.x >> 5) * gridDim.x + blockIdx.x;
     const int64_t n_warps = static_cast<int64_t>(gridDim.x) * kSampleWarps;
     const uint32_t V = static_cast<uint32_t>(a.V);
     // the kernel that clears tickets and bounds may still be running (see launch_one)
@@ -661,7 +663,11 @@ int launch_one(SampleArgs &a, int64_t nslot, size_t partial_bytes, cudaStream_t 
     a.split = choose_split(a.B, nslot, warps, max_parts);
     a.n_items = a.B * a.split;
     a.slots_per_chunk = static_cast<uint32_t>((nslot + a.split - 1) / a.split);
-    const int64_t want_ctas = (a.n_items + kSampleWarps - 1) / kSampleWarps;
+    // as many blocks as the items fill, but at least one per SM while items last (the kernel hands
+    // consecutive items to different blocks)
+    int64_t want_ctas = (a.n_items + kSampleWarps - 1) / kSampleWarps;
+    const int64_t one_per_sm = a.n_items < di.sm_count ? a.n_items : di.sm_count;
+    if (want_ctas < one_per_sm) want_ctas = one_per_sm;
     const unsigned grid = static_cast<unsigned>(want_ctas < ctas ? want_ctas : ctas);
     // Tickets and bounds start at zero.  Inside a stream capture (where the device-side gap between
     // the two nodes is what counts) they are cleared by a small kernel that releases its dependents
