@@ -106,6 +106,13 @@ __device__ __forceinline__ float ex2_approx(float x) {
     asm("ex2.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// The same with results below 2^-126 flushed to zero (one instruction instead of a scaled
+// sequence): for terms of a sum whose largest term is 1.
+__device__ __forceinline__ float ex2_approx_ftz(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
 // exp2(d * c) for d <= 0 with c = c_hi + c_lo: returns e = exp2(round(d c_hi)) and the residual
 // `lo` such that the true value is e * 2^lo ~ e * (1 + lo ln 2).
@@ -113,7 +120,7 @@ __device__ __forceinline__ float exp2_split(float d, float c_hi, float c_lo, flo
     d = fmaxf(d, -1e15f);                       // keeps -inf logits finite below
     const float hi = __fmul_rn(d, c_hi);
     lo = __fmaf_rn(d, c_lo, __fmaf_rn(d, c_hi, -hi));
-    return ex2_approx(hi);
+    return ex2_approx_ftz(hi);
 }
 __device__ __forceinline__ float exp2_scaled(float d, float c_hi, float c_lo) {
     float lo;
