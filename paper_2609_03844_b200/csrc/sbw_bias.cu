@@ -145,24 +145,30 @@ bias_kernel(const BiasArgs a) {
     constexpr int ESIZE = DTYPE == SBW_DTYPE_F32 ? 4 : 2;
     // let the next kernel in the stream start launching; wait for the previous ones to finish
     asm volatile("griddepcontrol.launch_dependents;");
-    const int64_t s_begin = a.total / gridDim.x * blockIdx.x +
-                            (a.total % gridDim.x) * blockIdx.x / gridDim.x;
-    const int64_t s_end = a.total / gridDim.x * (blockIdx.x + 1) +
-                          (a.total % gridDim.x) * (blockIdx.x + 1) / gridDim.x;
-    int64_t row = s_begin / a.nslot;
-    uint32_t col = static_cast<uint32_t>(s_begin - row * a.nslot);
-    int64_t left = s_end - s_begin;
+    // The rows are cut into units of one trip of the whole block (kBiasThreads slots, twice that
+    // for fp32); a row's last unit may be partly empty.  Every block takes the same number of
+    // units (to within one) of the B * units_per_row there are, so a range that crosses a row
+    // boundary costs no extra trip.
+    constexpr uint32_t kUnitSlots = VECTOR ? kBiasThreads * (DTYPE == SBW_DTYPE_F32 ? 2 : 1) : kBiasThreads;
     const uint32_t nslot = static_cast<uint32_t>(a.nslot);
+    const uint32_t units_per_row = (nslot + kUnitSlots - 1) / kUnitSlots;
+    const int64_t units = a.B * units_per_row;
+    const int64_t u_begin = units / gridDim.x * blockIdx.x + (units % gridDim.x) * blockIdx.x / gridDim.x;
+    const int64_t u_end = units / gridDim.x * (blockIdx.x + 1) + (units % gridDim.x) * (blockIdx.x + 1) / gridDim.x;
+    int64_t row = u_begin / units_per_row;
+    uint32_t unit = static_cast<uint32_t>(u_begin - row * units_per_row);
+    int64_t left = u_end - u_begin;
     const uint32_t V = static_cast<uint32_t>(a.V);
     const uint32_t nfull = V / VEC;       // slots of the row that are complete vectors
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
     while (left > 0) {
-        const uint32_t seg = static_cast<uint32_t>(min(static_cast<int64_t>(nslot - col), left));
+        const uint32_t seg_units = static_cast<uint32_t>(min(static_cast<int64_t>(units_per_row - unit), left));
         RowSeed<SCHEME> rs;
         rs.init(a.key, a.ctx + row * a.W, a.W);
         char *row_ptr = static_cast<char *>(a.logits) + row * a.ld * ESIZE;
-        const uint32_t j_end = col + seg;
+        const uint32_t col = unit * kUnitSlots;
+        const uint32_t j_end = min(nslot, col + seg_units * kUnitSlots);
         if constexpr (!VECTOR) {
             bias_scalar<DTYPE, SCHEME>(a, rs, row_ptr, col + threadIdx.x, j_end, kBiasThreads);
         } else {
@@ -224,9 +230,9 @@ bias_kernel(const BiasArgs a) {
                 bias_scalar<DTYPE, SCHEME>(a, rs, row_ptr, nfull * VEC, V, 1);
             }
         }
-        left -= seg;
+        left -= seg_units;
         ++row;
-        col = 0;
+        unit = 0;
     }
 }
 
@@ -242,7 +248,8 @@ int launch(const BiasArgs &a, cudaStream_t stream) {
                                                                    kBiasThreads, 0));
         blocks_per_sm = n > 0 ? n : 1;
     }
-    const int64_t want = (a.total + kBiasThreads - 1) / kBiasThreads;
+    constexpr int64_t kUnitSlots = VECTOR ? kBiasThreads * (DTYPE == SBW_DTYPE_F32 ? 2 : 1) : kBiasThreads;
+    const int64_t want = a.B * ((a.nslot + kUnitSlots - 1) / kUnitSlots);
     const int64_t cap = static_cast<int64_t>(di.sm_count) * blocks_per_sm;
     const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
     SBW_CUDA_TRY(launch_pdl(bias_kernel<DTYPE, SCHEME, VECTOR, COPY>, dim3(grid), dim3(kBiasThreads), stream, a));
