@@ -30,7 +30,6 @@ struct BiasArgs {
     void *logits;
     int64_t B, V, ld;
     int64_t nslot;          // slots per row
-    int64_t total;          // B * nslot
     const int32_t *ctx;
     int W;
     uint32_t vocab_offset;  // global id of column 0 (mod 2^32)
@@ -312,7 +311,6 @@ int bias_logits_impl(void *logits, int dtype, int64_t B, int64_t V, int64_t ld, 
     const bool vector = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && ((ld * esize) % 16 == 0);
     const int vec = vector ? 16 / esize : 1;
     a.nslot = (V + vec - 1) / vec;
-    a.total = B * a.nslot;
 
     if (dtype == SBW_DTYPE_F32) {
         return scheme == SBW_SCHEME_CONTEXT
@@ -345,7 +343,6 @@ int bias_copy_impl(const void *src, int64_t ld_src, void *dst, int dtype, int64_
     a.ld_src = ld_src;
     const int vec = 16 / esize;
     a.nslot = (V + vec - 1) / vec;
-    a.total = B * a.nslot;
     *done = true;
     if (dtype == SBW_DTYPE_F32) {
         return scheme == SBW_SCHEME_CONTEXT ? launch<SBW_DTYPE_F32, SBW_SCHEME_CONTEXT, true, true>(a, stream)
