@@ -181,6 +181,9 @@ topk_kernel(const TopkArgs a) {
     constexpr int kGroups = kTopkThreads / 4;   // maxima of disjoint column sets used for the lower bound
     __shared__ uint32_t sh_max[kGroups];
     __shared__ __align__(16) uint64_t sh_cand[kCap + 2];
+    __shared__ __align__(16) uint64_t sh_keep[kCap + 2];
+    __shared__ unsigned sh_hist[256];
+    __shared__ unsigned sh_kept, sh_cut;
     __shared__ uint64_t sh_red[kTopkWarps];
     __shared__ uint64_t sh_best;
     __shared__ uint32_t sh_floor;
@@ -267,13 +270,60 @@ topk_kernel(const TopkArgs a) {
         }
 
         if (n <= kCap) {
+            uint64_t *list = sh_cand;
+            if (n > 2 * k + 64) {
+                // Counting costs n^2, so a long list is cut first: a histogram of the codes over
+                // [bound, largest code] in 256 bins of equal width; the bin in which the count from
+                // the top reaches k holds the k-th largest code, and everything in a lower bin has
+                // k larger codes above it.
+                if (threadIdx.x < 256) sh_hist[threadIdx.x] = 0;
+                if (threadIdx.x == 0) {
+                    sh_kept = 0;
+                    sh_cut = 0;
+                }
+                uint64_t top = 0;
+                for (unsigned i = threadIdx.x; i < n; i += kTopkThreads) top = sh_cand[i] > top ? sh_cand[i] : top;
+                top = block_max_u64<kTopkWarps>(top, sh_red, &sh_best);
+                const uint32_t span = static_cast<uint32_t>(top >> 32) - floor_code;
+                const int shift = span < 256u ? 0 : 32 - __clz(span) - 8;
+                for (unsigned i = threadIdx.x; i < n; i += kTopkThreads)
+                    atomicAdd(&sh_hist[(static_cast<uint32_t>(sh_cand[i] >> 32) - floor_code) >> shift], 1u);
+                __syncthreads();
+                if (threadIdx.x < 32) {
+                    unsigned mine = 0;                            // entries in this lane's 8 bins
+                    for (int b = 0; b < 8; ++b) mine += sh_hist[threadIdx.x * 8 + b];
+                    unsigned above = mine;                        // entries in this lane's bins and all higher ones
+                    for (int d = 1; d < 32; d <<= 1) {
+                        const unsigned o = __shfl_down_sync(0xffffffffu, above, d);
+                        if (threadIdx.x + d < 32) above += o;
+                    }
+                    if (above >= k && above - mine < k) {         // one lane: the count from the top reaches k in its bins
+                        unsigned run = above - mine;
+                        int b = 7;
+                        for (; b > 0; --b) {
+                            run += sh_hist[threadIdx.x * 8 + b];
+                            if (run >= k) break;
+                        }
+                        sh_cut = threadIdx.x * 8 + b;
+                    }
+                }
+                __syncthreads();
+                const unsigned cut = sh_cut;
+                for (unsigned i = threadIdx.x; i < n; i += kTopkThreads) {
+                    const uint64_t e = sh_cand[i];
+                    if (((static_cast<uint32_t>(e >> 32) - floor_code) >> shift) >= cut) sh_keep[atomicAdd(&sh_kept, 1u)] = e;
+                }
+                __syncthreads();
+                list = sh_keep;
+                n = sh_kept;
+            }
             // 3. rank by counting, bias ranks below k
-            if (threadIdx.x == 0 && (n & 1u)) sh_cand[n] = 0;      // pad to a pair (kCap is even; 0 ranks below all)
+            if (threadIdx.x == 0 && (n & 1u)) list[n] = 0;         // pad to a pair (kCap is even; 0 ranks below all)
             __syncthreads();
             for (unsigned e = threadIdx.x; e < n; e += kTopkThreads) {
-                const uint64_t mine = sh_cand[e];
+                const uint64_t mine = list[e];
                 uint32_t r0 = 0, r1 = 0;
-                const ulonglong2 *pairs = reinterpret_cast<const ulonglong2 *>(sh_cand);
+                const ulonglong2 *pairs = reinterpret_cast<const ulonglong2 *>(list);
 #pragma unroll 4
                 for (unsigned u = 0; u < (n + 1) / 2; ++u) {          // two composites per shared-memory load
                     const ulonglong2 q = pairs[u];

@@ -2,6 +2,8 @@
 entry point (the paper's Section 5.1 "in-place, zero allocation" and the 0 MB column of its memory
 table, Appendix E), the softmax sum keeps its accuracy on rows built to stress it, and the
 host-buffer entry point matches the oracle at the size the benchmark's end-to-end figure uses."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -87,6 +89,7 @@ def test_no_entry_point_allocates_device_memory():
     torch.cuda.synchronize()
 
     def one_pass():
+        gc.collect()                                           # tensors left by earlier tests go now, not mid-pass
         free0, _ = torch.cuda.mem_get_info(dev)
         torch0 = torch.cuda.memory_allocated(dev), torch.cuda.memory_reserved(dev)
         for name, fn in calls.items():
