@@ -4,10 +4,10 @@
 //
 // One CTA per row.  "Largest" is the total order on order-encoded bit patterns with ties to the
 // lowest column, expressed as one 64-bit composite (code << 32 | ~column).
-//   1. A pass over a prefix of the row (32 columns per thread): every thread keeps the largest code
+//   1. A pass over a prefix of the row (its first 128 KB): every thread keeps the largest code
 //      it has seen; groups of four threads give 256 maxima of disjoint column sets.  Their k-th
 //      largest value L is a lower bound of the row's k-th largest logit (k distinct columns reach
-//      it), and it is known after a fifth of the row.
+//      it), and it is known after a fifth (fp32, V = 151936) to a half (bf16, V = 128256) of the row.
 //   2. One pass over the whole row: columns with code >= L -- a few hundred for ordinary logits --
 //      go into a shared-memory candidate list.  The common path is one compare per 16-byte vector.
 //   3. Candidates are ranked by counting larger composites; ranks below k are hashed and biased.
@@ -32,7 +32,7 @@ namespace {
 // CTA size: 1024 threads (one CTA per SM) when there are fewer rows than SMs can take two of,
 // 512 threads (two CTAs per SM, twice the rows in flight) for larger batches.
 constexpr int kCap = 2048;                  // candidate list entries
-constexpr int kPrefixColumns = 32768;        // leading columns read by the pass that finds the bound
+constexpr int kPrefixBytes = 131072;         // leading part of the row read by the pass that finds the bound
 
 struct TopkArgs {
     void *logits;
@@ -204,7 +204,7 @@ topk_kernel(const TopkArgs a) {
         const uint64_t material = row_seed_material<SCHEME>(a, row);
 
         // 1. lower bound of the k-th largest code from a prefix of the columns
-        const uint32_t prefix_end = min(c_hi, c_lo + static_cast<uint32_t>(kPrefixColumns / CS));
+        const uint32_t prefix_end = min(c_hi, c_lo + static_cast<uint32_t>(kPrefixBytes / ESIZE / CS));
         uint32_t mx = 0;
         for_each_vector<DTYPE, kTopkThreads>(
             row_ptr, c_lo, prefix_end, a.vector,
