@@ -32,6 +32,7 @@ namespace {
 // CTA size: 1024 threads (one CTA per SM) when there are fewer rows than SMs can take two of,
 // 512 threads (two CTAs per SM, twice the rows in flight) for larger batches.
 constexpr int kCap = 2048;                  // candidate list entries
+constexpr int kHitCap = 2048;                // vectors noted by the gather pass for a closer look
 constexpr int kPrefixBytes = 131072;         // leading part of the row read by the pass that finds the bound
 
 struct TopkArgs {
@@ -182,6 +183,8 @@ topk_kernel(const TopkArgs a) {
     __shared__ uint32_t sh_max[kGroups];
     __shared__ __align__(16) uint64_t sh_cand[kCap + 2];
     __shared__ __align__(16) uint64_t sh_keep[kCap + 2];
+    __shared__ uint32_t sh_hitvec[kHitCap];
+    __shared__ unsigned sh_nhit;
     __shared__ unsigned sh_hist[256];
     __shared__ unsigned sh_kept, sh_cut;
     __shared__ uint64_t sh_red[kTopkWarps];
@@ -216,6 +219,7 @@ topk_kernel(const TopkArgs a) {
         if (threadIdx.x == 0) {
             sh_floor = 0;            // k_part > kGroups: no bound, everything is a candidate
             sh_count = 0;
+            sh_nhit = 0;
         }
         __syncthreads();
         if (k_part <= kGroups && threadIdx.x < kGroups) {
@@ -242,14 +246,41 @@ topk_kernel(const TopkArgs a) {
                 if (pos < kCap) sh_cand[pos] = composite(code, col);
             }
         };
-        for_each_vector<DTYPE, kTopkThreads>(
-            row_ptr, c_lo, c_hi, a.vector,
-            [&](uint32_t col0, const uint4 &w) {
-                if (vector_max_code<DTYPE>(w) < floor_code) return;   // the common case: one compare per vector
+        // bf16 (eight logits per vector): a vector that reaches the bound is only noted here (the
+        // common case is one compare per vector, the rare one an atomic add and a store) and its
+        // logits are looked at afterwards by one thread each, so that no warp walks a vector's
+        // elements with a single lane active.  fp32 (four logits) looks at them on the spot: the
+        // extra barrier and the second read cost more than they save there.
+        if constexpr (DTYPE == SBW_DTYPE_BF16) {
+            for_each_vector<DTYPE, kTopkThreads>(
+                row_ptr, c_lo, c_hi, a.vector,
+                [&](uint32_t col0, const uint4 &w) {
+                    if (vector_max_code<DTYPE>(w) < floor_code) return;
+                    const unsigned pos = atomicAdd(&sh_nhit, 1u);
+                    if (pos < static_cast<unsigned>(kHitCap)) sh_hitvec[pos] = col0;
+                },
+                push);
+            __syncthreads();
+            constexpr unsigned kVec = 16 / ESIZE;
+            const unsigned nhit = sh_nhit;
+            if (nhit <= static_cast<unsigned>(kHitCap)) {
+                for (unsigned t = threadIdx.x; t < nhit * kVec; t += kTopkThreads) {
+                    const uint32_t col = sh_hitvec[t / kVec] + t % kVec;
+                    push(col, scalar_code<DTYPE>(row_ptr, col));
+                }
+            } else if (threadIdx.x == 0) {
+                sh_count = kCap + 1;             // too many to note: the exact fallback takes the row
+            }
+        } else {
+            for_each_vector<DTYPE, kTopkThreads>(
+                row_ptr, c_lo, c_hi, a.vector,
+                [&](uint32_t col0, const uint4 &w) {
+                    if (vector_max_code<DTYPE>(w) < floor_code) return;   // the common case: one compare per vector
 #pragma unroll
-                for (int i = 0; i < 16 / ESIZE; ++i) push(col0 + i, element_code<DTYPE>(w, i));
-            },
-            push);
+                    for (int i = 0; i < 16 / ESIZE; ++i) push(col0 + i, element_code<DTYPE>(w, i));
+                },
+                push);
+        }
         __syncthreads();
         unsigned n = sh_count;
         if constexpr (CS > 1) {
