@@ -189,7 +189,7 @@ topk_kernel(const TopkArgs a) {
     __shared__ unsigned sh_kept, sh_cut;
     __shared__ uint64_t sh_red[kTopkWarps];
     __shared__ uint64_t sh_best;
-    __shared__ uint32_t sh_floor;
+    __shared__ uint32_t sh_floor, sh_top;
     __shared__ unsigned sh_count;
     namespace cg = cooperative_groups;
     const uint32_t V = static_cast<uint32_t>(a.V);
@@ -218,6 +218,7 @@ topk_kernel(const TopkArgs a) {
         if ((threadIdx.x & 3) == 0) sh_max[threadIdx.x >> 2] = mx;
         if (threadIdx.x == 0) {
             sh_floor = 0;            // k_part > kGroups: no bound, everything is a candidate
+            sh_top = 0xffffffffu;    // and no largest prefix code either
             sh_count = 0;
             sh_nhit = 0;
         }
@@ -230,6 +231,7 @@ topk_kernel(const TopkArgs a) {
                 rank += (o > mine || (o == mine && u < static_cast<int>(threadIdx.x))) ? 1u : 0u;
             }
             if (rank == k_part - 1) sh_floor = mine;
+            if (rank == 0) sh_top = mine;            // the largest code of the prefix
         }
         __syncthreads();
         uint32_t floor_code = sh_floor;
@@ -304,7 +306,7 @@ topk_kernel(const TopkArgs a) {
             uint64_t *list = sh_cand;
             if (n > 2 * k + 64) {
                 // Counting costs n^2, so a long list is cut first: a histogram of the codes over
-                // [bound, largest code] in 256 bins of equal width; the bin in which the count from
+                // [bound, largest code of the prefix] in 256 bins of equal width; the bin in which the count from
                 // the top reaches k holds the k-th largest code, and everything in a lower bin has
                 // k larger codes above it.
                 if (threadIdx.x < 256) sh_hist[threadIdx.x] = 0;
@@ -312,13 +314,16 @@ topk_kernel(const TopkArgs a) {
                     sh_kept = 0;
                     sh_cut = 0;
                 }
-                uint64_t top = 0;
-                for (unsigned i = threadIdx.x; i < n; i += kTopkThreads) top = sh_cand[i] > top ? sh_cand[i] : top;
-                top = block_max_u64<kTopkWarps>(top, sh_red, &sh_best);
-                const uint32_t span = static_cast<uint32_t>(top >> 32) - floor_code;
+                __syncthreads();                                  // the histogram is clear
+                // bins over [bound, largest code of the prefix]; codes above that share the top bin
+                const uint32_t top = sh_top > floor_code ? sh_top : floor_code;
+                const uint32_t span = top - floor_code;
                 const int shift = span < 256u ? 0 : 32 - __clz(span) - 8;
-                for (unsigned i = threadIdx.x; i < n; i += kTopkThreads)
-                    atomicAdd(&sh_hist[(static_cast<uint32_t>(sh_cand[i] >> 32) - floor_code) >> shift], 1u);
+                auto bin_of = [&](uint64_t e) -> unsigned {
+                    const uint32_t b = (static_cast<uint32_t>(e >> 32) - floor_code) >> shift;
+                    return b < 255u ? b : 255u;
+                };
+                for (unsigned i = threadIdx.x; i < n; i += kTopkThreads) atomicAdd(&sh_hist[bin_of(sh_cand[i])], 1u);
                 __syncthreads();
                 if (threadIdx.x < 32) {
                     unsigned mine = 0;                            // entries in this lane's 8 bins
@@ -342,7 +347,7 @@ topk_kernel(const TopkArgs a) {
                 const unsigned cut = sh_cut;
                 for (unsigned i = threadIdx.x; i < n; i += kTopkThreads) {
                     const uint64_t e = sh_cand[i];
-                    if (((static_cast<uint32_t>(e >> 32) - floor_code) >> shift) >= cut) sh_keep[atomicAdd(&sh_kept, 1u)] = e;
+                    if (bin_of(e) >= cut) sh_keep[atomicAdd(&sh_kept, 1u)] = e;
                 }
                 __syncthreads();
                 list = sh_keep;
