@@ -97,14 +97,14 @@ __device__ __forceinline__ void for_each_code(const char *row_ptr, uint32_t begi
 // Calls fvec(first column, vector) for the aligned 16-byte vectors of the columns [begin, end) that
 // this thread owns and fone(column, code) for the columns left over (all of them when the rows
 // are not aligned); begin is a multiple of 8 columns.
-template <int DTYPE, int kTopkThreads, typename FV, typename F1>
+template <int DTYPE, int kTopkThreads, int kInFlight = 8, typename FV, typename F1>
 __device__ __forceinline__ void for_each_vector(const char *row_ptr, uint32_t begin, uint32_t end, bool vector,
                                                 FV fvec, F1 fone) {
     constexpr int VEC = DTYPE == SBW_DTYPE_F32 ? 4 : 8;
     uint32_t done = begin;
     if (vector) {
         const uint32_t nfull = end / VEC;
-        constexpr int kInFlight = 8;   // independent 128-bit loads per thread before the first use
+        // kInFlight independent 128-bit loads per thread before the first use
         for (uint32_t j0 = begin / VEC + threadIdx.x; j0 < nfull; j0 += kInFlight * kTopkThreads) {
             uint4 w[kInFlight];
 #pragma unroll
@@ -274,7 +274,9 @@ topk_kernel(const TopkArgs a) {
                 sh_count = kCap + 1;             // too many to note: the exact fallback takes the row
             }
         } else {
-            for_each_vector<DTYPE, kTopkThreads>(
+            // ten loads in flight fit the 64 registers that two 512-thread CTAs per SM leave a thread
+            // (the cluster variants would spill); bf16, with more work per vector, is faster with eight
+            for_each_vector<DTYPE, kTopkThreads, (CS == 1 ? 10 : 8)>(
                 row_ptr, c_lo, c_hi, a.vector,
                 [&](uint32_t col0, const uint4 &w) {
                     if (vector_max_code<DTYPE>(w) < floor_code) return;   // the common case: one compare per vector
